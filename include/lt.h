@@ -1,0 +1,207 @@
+/*
+ * lt.h - C ABI of liblt: the hybrid decode-attention path of LightTransfer on
+ * one NVIDIA B200 (sm_100a).
+ *
+ * The method (LightTransfer-Test, Section 5.1 of the paper): after the prompt
+ * has been prefilled, every layer gets a "lazy ratio" (Eq. 1) - the share of
+ * attention that its last w_last prompt queries put on the first n_sink keys
+ * and on the last n_recent keys.  The layers with the highest ratios become
+ * "lazy": they keep only those keys/values (a constant-size cache) and decode
+ * with streaming attention; every other layer keeps its whole cache and
+ * decodes with full attention.
+ *
+ * Conventions
+ *   - Every function returns an lt_status; nothing aborts, throws or traps.
+ *   - The caller owns all memory.  The library allocates nothing on the
+ *     device, keeps no state between calls and never synchronises the device
+ *     unless a function says so.  All device work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - "dev" marks a device pointer, "host" a host pointer.
+ *   - Layer tables (k_full, v_full, k_stream, v_stream) are HOST arrays of
+ *     n_layers DEVICE pointers, read during the call only.  An entry may be
+ *     NULL when that layer never takes that role (a layer's role is known
+ *     only after lt_select_lazy, so a caller may allocate both kinds for all
+ *     layers, or re-allocate after selection).  A NULL entry that the device
+ *     mask selects is skipped and reported through the error word.
+ *   - Layouts are dense row-major, last index fastest:
+ *       full cache of one layer    [batch][n_kv_heads][full_capacity][head_dim]
+ *       stream cache of one layer  [batch][n_kv_heads][n_sink+n_recent][head_dim]
+ *     Every cache pointer must be 16-byte aligned.
+ *   - layer_mask is uint8[n_layers] on the device, 1 = lazy (streaming).
+ *   - seq_lens is int32[batch] on the device: tokens already in the cache of
+ *     that batch row = position of the next token.
+ *   - A decode step is "append, then attend": the new token attends to itself
+ *     (causal mask with i >= j, Appendix E).
+ *   - GQA: query head hq reads kv head hq / (n_q_heads / n_kv_heads).
+ */
+#ifndef LT_H_
+#define LT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t lt_status;
+enum {
+  LT_OK = 0,
+  LT_ERR_INVALID_ARG = 1, /* null pointer, bad size, n_lazy outside [0, L], ... */
+  LT_ERR_UNSUPPORTED = 2, /* head_dim not in {64,128}, unknown dtype, too many layers */
+  LT_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  LT_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error) */
+  LT_ERR_TIMEOUT = 5,     /* reserved: no kernel of this library waits on another */
+  LT_ERR_DEVICE_RANGE = 6 /* reported by lt_check: a position left its cache */
+};
+
+enum { LT_F32 = 0, LT_BF16 = 1 };
+
+#define LT_MAX_LAYERS 128
+
+/* Bits of the device error word (see lt_check). */
+#define LT_DEVERR_POS_OUT_OF_RANGE 1u /* append: seq_len >= full_capacity; store skipped */
+#define LT_DEVERR_NULL_LAYER 2u       /* mask selected a layer whose table entry is NULL */
+#define LT_DEVERR_LEN_CLAMPED 4u      /* attend: seq_len > full_capacity; clamped */
+
+typedef struct lt_shape {
+  int32_t n_layers;      /* L, 1..LT_MAX_LAYERS */
+  int32_t batch;         /* B >= 1 */
+  int32_t n_q_heads;     /* Hq, multiple of n_kv_heads */
+  int32_t n_kv_heads;    /* Hkv >= 1 */
+  int32_t head_dim;      /* D, 64 or 128 */
+  int32_t n_sink;        /* w_sink >= 0 (0 = pure sliding window) */
+  int32_t n_recent;      /* w_recent >= 1 */
+  int32_t full_capacity; /* rows per (batch, kv head) of a full cache */
+  int32_t dtype;         /* LT_F32 or LT_BF16: q, k, v and both caches */
+  float softmax_scale;   /* <= 0 means 1/sqrt(head_dim) */
+} lt_shape;
+
+/* Text for a status code (static storage, never NULL). */
+const char* lt_status_string(lt_status s);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t lt_version(void);
+
+/*
+ * Slot of token position `pos` in a lazy layer's cache (Section 5.1: a lazy
+ * layer retains only the KV of {X_initial, X_recent}): pos itself while
+ * pos < n_sink, else n_sink + (pos - n_sink) mod n_recent.  Pure host function;
+ * returns -1 on pos < 0, n_sink < 0 or n_recent < 1.
+ */
+int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent);
+
+/*
+ * Bytes of workspace that lt_lazy_scores (prompt length up to n_ctx_max, up to
+ * w_last_max tail queries) and lt_hybrid_decode_attn (any seq_len up to
+ * max(full_capacity, n_sink + n_recent)) need for this shape.  Host only.
+ * The workspace is device memory, 256-byte aligned, owned by the caller; its
+ * first 256 bytes hold the device error word and must be zeroed once with
+ * lt_workspace_init.  Two calls that overlap on the device must not share it.
+ */
+lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max,
+                             size_t* bytes_out /* host */);
+
+/* Zero the workspace header (async on `stream`). */
+lt_status lt_workspace_init(void* ws /* dev */, size_t ws_bytes, void* stream);
+
+/*
+ * Copy the device error word to *flags_out and clear it.  SYNCHRONISES the
+ * stream.  Returns LT_ERR_DEVICE_RANGE when any bit is set, LT_OK otherwise.
+ */
+lt_status lt_check(void* ws /* dev */, uint32_t* flags_out /* host, may be NULL */, void* stream);
+
+/*
+ * Lazy ratio (Eq. 1; Table 1 for the log-sum-exp identity it equals).
+ *   q_tail  dev [L][B][Hq][w_last][D]: queries of prompt positions
+ *           n_ctx - w_last .. n_ctx - 1
+ *   k_full  host table of dev pointers; rows 0 .. n_ctx-1 of every (b, kv head)
+ *           hold the prompt keys.  Every entry must be non-NULL.
+ *   scores  dev float [L][B][Hq]: for each query head the mean over the w_last
+ *           tail queries of the causal-softmax mass on keys j < n_sink or
+ *           j >= n_ctx - n_recent (a set union; 1.0 when the window covers all).
+ * The mean over heads and batch rows that completes Eq. 1 is taken by
+ * lt_select_lazy.  Requires 1 <= w_last <= n_ctx <= full_capacity.
+ */
+lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
+                         const void* const* k_full /* host table */, int32_t n_ctx, int32_t w_last,
+                         float* scores /* dev */, void* ws /* dev */, size_t ws_bytes, void* stream);
+
+/*
+ * Selection (Section 5.1, the max-priority queue of size P = L - n_lazy; Fig. 3):
+ * r_l = mean over [B][Hq] of scores[l] (accumulated in double, fixed order);
+ * layer_mask[l] = 1 for the n_lazy layers with the largest r_l, ties to the
+ * lower layer index - the same set the streaming priority queue leaves lazy.
+ *   layer_ratio  dev float [L] or NULL: r_l rounded to float.
+ * Runs on the device; no host round trip.
+ */
+lt_status lt_select_lazy(const float* scores /* dev [L][B][Hq] */, int32_t n_layers, int32_t batch,
+                         int32_t n_q_heads, int32_t n_lazy, uint8_t* layer_mask /* dev [L] */,
+                         float* layer_ratio /* dev [L] or NULL */, void* stream);
+
+/*
+ * Prefill -> decode compaction of the lazy layers (Section 5.1: "retain only
+ * the KV caches corresponding to {X_initial, X_recent} and discard others";
+ * Fig. 3).  For every layer with mask 1 and every (b, kv head), prompt rows
+ * p in {0 .. min(n_sink,n)-1} U {max(n_sink, n - n_recent) .. n-1}, n = seq_lens[b],
+ * are copied bit for bit from the full cache to row lt_ring_slot(p) of the
+ * stream cache, so later appends continue the ring.  Layers with mask 0 are
+ * untouched.
+ */
+lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask /* dev */,
+                         const void* const* k_full, const void* const* v_full /* host tables */,
+                         const int32_t* seq_lens /* dev [B] */, void* const* k_stream,
+                         void* const* v_stream /* host tables */, void* ws /* dev, for the error word; may be NULL */,
+                         void* stream);
+
+/*
+ * Per-step KV append (Section 3: decoding "saves their KV cache"; Section 5.1
+ * for the lazy layers).  With p = seq_lens[b]:
+ *   mask 0: k_new[l][b][h][:] -> full cache row p        (skipped and flagged
+ *           LT_DEVERR_POS_OUT_OF_RANGE when p >= full_capacity)
+ *   mask 1: -> stream cache row lt_ring_slot(p): sinks are never overwritten,
+ *           later tokens overwrite the oldest ring row.
+ * Then seq_lens[b] += 1 for every b (once per call, not per layer).
+ *   k_new, v_new  dev [L][B][Hkv][D]
+ *   layers [layer_begin, layer_begin + layer_count) are written; pass 0 and
+ *   n_layers for the whole stack.  seq_lens is advanced only when
+ *   advance_seq_lens != 0 (a per-layer caller advances on its last layer).
+ */
+lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask /* dev */,
+                       const void* k_new /* dev */, const void* v_new /* dev */,
+                       int32_t* seq_lens /* dev [B] */, void* const* k_full, void* const* v_full,
+                       void* const* k_stream, void* const* v_stream /* host tables */,
+                       int32_t layer_begin, int32_t layer_count, int32_t advance_seq_lens,
+                       void* ws /* dev, for the error word; may be NULL */, void* stream);
+
+/*
+ * One decode step of attention for the whole stack (Appendix E: MHA with the
+ * causal mask in layers outside I, with M_lazy in layers inside I; Section 3).
+ * With n = seq_lens[b] (the new token already appended):
+ *   mask 0: out[l][b][hq] = softmax(scale * q . K[0..n-1]^T) V[0..n-1]  over the
+ *           full cache;
+ *   mask 1: the same over the min(n, n_sink + n_recent) valid rows of the stream
+ *           cache (order of rows is irrelevant to softmax, so the ring is read
+ *           linearly).
+ *   q    dev [L][B][Hq][D], dtype of the shape
+ *   out  dev [L][B][Hq][D], LT_F32 or LT_BF16 (out_dtype); zeros where n = 0
+ *   max_seq_len_hint  host upper bound on max_b seq_lens[b], used only to size
+ *           the launch; <= 0 means full_capacity.  A seq_len above the hint is
+ *           still handled correctly only up to the hint rounded up to the
+ *           split size, so pass a true bound (or 0).
+ *   layers [layer_begin, layer_begin + layer_count).
+ * Split-KV: partial (max, sum, weighted values) per KV chunk go to the
+ * workspace and a second kernel merges them.
+ */
+lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q /* dev */,
+                                const void* const* k_full, const void* const* v_full,
+                                const void* const* k_stream, const void* const* v_stream /* host tables */,
+                                const uint8_t* layer_mask /* dev */, const int32_t* seq_lens /* dev */,
+                                void* out /* dev */, int32_t out_dtype, int32_t max_seq_len_hint,
+                                int32_t layer_begin, int32_t layer_count, void* ws /* dev */,
+                                size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LT_H_ */

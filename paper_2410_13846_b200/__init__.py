@@ -1,0 +1,11 @@
+"""B200-native hybrid decode attention (LightTransfer hot path).
+
+The work is done by liblt.so (hand-written CUDA for sm_100a behind a C ABI,
+declared in include/lt.h).  This package is the thin Python binding: argument
+marshalling only.  There is no CPU or PyTorch fallback: calls raise when the
+library is missing or a CUDA device is absent.
+"""
+from .binding import (  # noqa: F401
+    LT_BF16, LT_F32, LayerTables, LtError, Shape, check, hybrid_decode_attn, kv_append, lazy_scores, lib, lib_path,
+    ring_slot, select_lazy, status_string, stream_init, version, workspace_bytes, workspace_init,
+)

@@ -1,0 +1,210 @@
+"""ctypes binding of liblt.so.  Same names as the C ABI minus the ``lt_`` prefix.
+
+Tensors are torch CUDA tensors used only as device memory: the binding passes
+``data_ptr()`` and the current CUDA stream.  Layer tables are Python lists of
+tensors (or None entries).  Nothing here computes anything.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+LT_F32, LT_BF16 = 0, 1
+LT_MAX_LAYERS = 128
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+class LtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: lt_status {status} ({status_string(status)})")
+
+
+class _CShape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_sink", "n_recent",
+                 "full_capacity", "dtype")] + [("softmax_scale", C.c_float)]
+
+
+@dataclass
+class Shape:
+    n_layers: int
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    n_sink: int
+    n_recent: int
+    full_capacity: int
+    dtype: int = LT_BF16
+    softmax_scale: float = 0.0
+
+    def c(self) -> _CShape:
+        return _CShape(self.n_layers, self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_sink,
+                       self.n_recent, self.full_capacity, self.dtype, self.softmax_scale)
+
+    @property
+    def stream_capacity(self) -> int:
+        return self.n_sink + self.n_recent
+
+
+def lib_path() -> str:
+    return os.path.join(_PKG_DIR, "liblt.so")
+
+
+def lib() -> C.CDLL:
+    """Load liblt.so (once).  Raises if it has not been built."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2410_13846_b200.build` "
+                           "(there is no fallback path)")
+    L = C.CDLL(path)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    shp = C.POINTER(_CShape)
+    tab = C.POINTER(C.c_void_p)
+    L.lt_status_string.restype = C.c_char_p
+    L.lt_status_string.argtypes = [i32]
+    L.lt_version.restype = i32
+    L.lt_version.argtypes = []
+    L.lt_ring_slot.restype = i32
+    L.lt_ring_slot.argtypes = [i32, i32, i32]
+    L.lt_workspace_bytes.restype = i32
+    L.lt_workspace_bytes.argtypes = [shp, i32, i32, C.POINTER(sz)]
+    L.lt_workspace_init.restype = i32
+    L.lt_workspace_init.argtypes = [vp, sz, vp]
+    L.lt_check.restype = i32
+    L.lt_check.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    L.lt_lazy_scores.restype = i32
+    L.lt_lazy_scores.argtypes = [shp, vp, tab, i32, i32, vp, vp, sz, vp]
+    L.lt_select_lazy.restype = i32
+    L.lt_select_lazy.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    L.lt_stream_init.restype = i32
+    L.lt_stream_init.argtypes = [shp, vp, tab, tab, vp, tab, tab, vp, vp]
+    L.lt_kv_append.restype = i32
+    L.lt_kv_append.argtypes = [shp, vp, vp, vp, vp, tab, tab, tab, tab, i32, i32, i32, vp, vp]
+    L.lt_hybrid_decode_attn.restype = i32
+    L.lt_hybrid_decode_attn.argtypes = [shp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
+    _LIB = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().lt_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().lt_version())
+
+
+def ring_slot(pos: int, n_sink: int, n_recent: int) -> int:
+    return int(lib().lt_ring_slot(pos, n_sink, n_recent))
+
+
+# ---- marshalling helpers ----------------------------------------------------
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("liblt works on CUDA tensors only (no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _table(tensors, n_layers):
+    """Host array of device pointers from a list of tensors / None; None -> NULL table."""
+    if tensors is None:
+        return None
+    if len(tensors) != n_layers:
+        raise ValueError("layer table must have n_layers entries")
+    arr = (C.c_void_p * n_layers)()
+    for i, t in enumerate(tensors):
+        if t is None:
+            arr[i] = None
+        else:
+            if not t.is_cuda or not t.is_contiguous():
+                raise ValueError("layer table entries must be contiguous CUDA tensors")
+            arr[i] = t.data_ptr()
+    return arr
+
+
+def _stream(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ok(status: int, where: str):
+    if status != 0:
+        raise LtError(status, where)
+
+
+class LayerTables:
+    """Pre-marshalled host tables for one set of caches (build once, reuse every step)."""
+
+    def __init__(self, shape: Shape, k_full=None, v_full=None, k_stream=None, v_stream=None):
+        L = shape.n_layers
+        self.keep = (k_full, v_full, k_stream, v_stream)     # keep the tensors alive
+        self.k_full, self.v_full = _table(k_full, L), _table(v_full, L)
+        self.k_stream, self.v_stream = _table(k_stream, L), _table(v_stream, L)
+
+
+# ---- the calls --------------------------------------------------------------
+def workspace_bytes(shape: Shape, n_ctx_max: int = 0, w_last_max: int = 0) -> int:
+    out = C.c_size_t(0)
+    _ok(lib().lt_workspace_bytes(C.byref(shape.c()), n_ctx_max, w_last_max, C.byref(out)), "lt_workspace_bytes")
+    return int(out.value)
+
+
+def workspace_init(ws, stream=None):
+    _ok(lib().lt_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "lt_workspace_init")
+
+
+def check(ws, stream=None, raise_on_error: bool = True) -> int:
+    flags = C.c_uint32(0)
+    st = lib().lt_check(_ptr(ws), C.byref(flags), _stream(stream))
+    if st != 0 and (raise_on_error or st != 6):
+        raise LtError(st, f"lt_check (flags={flags.value:#x})")
+    return int(flags.value)
+
+
+def lazy_scores(shape: Shape, q_tail, k_full, n_ctx: int, w_last: int, scores, ws, stream=None):
+    tab = k_full.k_full if isinstance(k_full, LayerTables) else _table(k_full, shape.n_layers)
+    _ok(lib().lt_lazy_scores(C.byref(shape.c()), _ptr(q_tail), tab, n_ctx, w_last, _ptr(scores), _ptr(ws),
+                             ws.numel() * ws.element_size(), _stream(stream)), "lt_lazy_scores")
+
+
+def select_lazy(scores, n_layers: int, batch: int, n_q_heads: int, n_lazy: int, layer_mask, layer_ratio=None,
+                stream=None):
+    _ok(lib().lt_select_lazy(_ptr(scores), n_layers, batch, n_q_heads, n_lazy, _ptr(layer_mask),
+                             _ptr(layer_ratio), _stream(stream)), "lt_select_lazy")
+
+
+def stream_init(shape: Shape, layer_mask, tables: LayerTables, seq_lens, ws=None, stream=None):
+    _ok(lib().lt_stream_init(C.byref(shape.c()), _ptr(layer_mask), tables.k_full, tables.v_full, _ptr(seq_lens),
+                             tables.k_stream, tables.v_stream, _ptr(ws), _stream(stream)), "lt_stream_init")
+
+
+def kv_append(shape: Shape, layer_mask, k_new, v_new, seq_lens, tables: LayerTables, layer_begin: int = 0,
+              layer_count: int | None = None, advance_seq_lens: bool = True, ws=None, stream=None):
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_kv_append(C.byref(shape.c()), _ptr(layer_mask), _ptr(k_new), _ptr(v_new), _ptr(seq_lens),
+                           tables.k_full, tables.v_full, tables.k_stream, tables.v_stream, layer_begin, cnt,
+                           1 if advance_seq_lens else 0, _ptr(ws), _stream(stream)), "lt_kv_append")
+
+
+def hybrid_decode_attn(shape: Shape, q, tables: LayerTables, layer_mask, seq_lens, out, ws, out_dtype: int | None = None,
+                       max_seq_len_hint: int = 0, layer_begin: int = 0, layer_count: int | None = None, stream=None):
+    import torch
+    if out_dtype is None:
+        out_dtype = LT_F32 if out.dtype == torch.float32 else LT_BF16
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_hybrid_decode_attn(C.byref(shape.c()), _ptr(q), tables.k_full, tables.v_full, tables.k_stream,
+                                    tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
+                                    max_seq_len_hint, layer_begin, cnt, _ptr(ws), ws.numel() * ws.element_size(),
+                                    _stream(stream)), "lt_hybrid_decode_attn")

@@ -1,0 +1,267 @@
+// C-ABI entry points of liblt: argument validation, workspace carving and
+// stream-ordered launches.  No device memory is allocated here and no state
+// survives a call.
+#include <math.h>
+#include <string.h>
+
+#include "lt_internal.h"
+
+namespace lt {
+
+lt_status validate_shape(const lt_shape* s) {
+  if (!s) return LT_ERR_INVALID_ARG;
+  if (s->n_layers < 1 || s->batch < 1 || s->n_kv_heads < 1 || s->n_q_heads < 1) return LT_ERR_INVALID_ARG;
+  if (s->n_q_heads % s->n_kv_heads != 0) return LT_ERR_INVALID_ARG;
+  if (s->n_sink < 0 || s->n_recent < 1 || s->full_capacity < 1) return LT_ERR_INVALID_ARG;
+  if ((int64_t)s->n_sink + s->n_recent > (1 << 30)) return LT_ERR_INVALID_ARG;
+  if (s->n_layers > LT_MAX_LAYERS) return LT_ERR_UNSUPPORTED;
+  if (s->head_dim != 64 && s->head_dim != 128) return LT_ERR_UNSUPPORTED;
+  if (s->dtype != LT_F32 && s->dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
+  if (!(s->softmax_scale == s->softmax_scale)) return LT_ERR_INVALID_ARG;  // NaN
+  return LT_OK;
+}
+
+DecodePlan make_decode_plan(const lt_shape& s) {
+  DecodePlan p;
+  const int64_t n_max = (int64_t)((s.full_capacity > s.n_sink + s.n_recent) ? s.full_capacity
+                                                                            : s.n_sink + s.n_recent);
+  const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
+  const int64_t target = 148 * 4;  // a few CTAs per SM even for small stacks
+  int ck = 2048;
+  while (ck > 256 && units * ((n_max + ck - 1) / ck) < target) ck /= 2;
+  p.chunk_keys = ck;
+  p.n_chunks_max = (int)((n_max + ck - 1) / ck);
+  const int G = s.n_q_heads / s.n_kv_heads;
+  p.ml_floats = (size_t)units * p.n_chunks_max * G * 2;
+  p.o_floats = (size_t)units * p.n_chunks_max * G * s.head_dim;
+  return p;
+}
+
+ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last) {
+  ScorePlan p;
+  const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
+  int64_t want = (148 * 4 + units - 1) / units;
+  int64_t most = (n_ctx + 1023) / 1024;
+  if (want > most) want = most;
+  if (want < 1) want = 1;
+  p.n_splits = (int)want;
+  p.stat_floats = (size_t)s.n_layers * s.batch * s.n_q_heads * w_last * p.n_splits * 3;
+  return p;
+}
+
+static lt_status fill_table(LayerTable* t, const void* const* host, int L, bool require_all) {
+  memset(t, 0, sizeof(*t));
+  if (!host) return require_all ? LT_ERR_INVALID_ARG : LT_OK;
+  for (int l = 0; l < L; ++l) {
+    t->p[l] = host[l];
+    if (require_all && !host[l]) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)host[l] & 15u) != 0) return LT_ERR_INVALID_ARG;
+  }
+  return LT_OK;
+}
+
+static lt_status check_layer_range(const lt_shape* s, int begin, int count) {
+  if (begin < 0 || count < 1 || begin + count > s->n_layers) return LT_ERR_INVALID_ARG;
+  return LT_OK;
+}
+
+static inline uint32_t* err_word(void* ws) { return reinterpret_cast<uint32_t*>(ws); }
+
+}  // namespace lt
+
+using namespace lt;
+
+extern "C" {
+
+const char* lt_status_string(lt_status s) {
+  switch (s) {
+    case LT_OK: return "ok";
+    case LT_ERR_INVALID_ARG: return "invalid argument";
+    case LT_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case LT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case LT_ERR_CUDA: return "CUDA runtime error";
+    case LT_ERR_TIMEOUT: return "device wait timed out";
+    case LT_ERR_DEVICE_RANGE: return "device error word set (position or length out of range)";
+    default: return "unknown status";
+  }
+}
+
+int32_t lt_version(void) { return 100; }
+
+int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent) {
+  if (pos < 0 || n_sink < 0 || n_recent < 1) return -1;
+  if (pos < n_sink) return pos;
+  return n_sink + (pos - n_sink) % n_recent;
+}
+
+lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max, size_t* bytes_out) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!bytes_out || n_ctx_max < 0 || w_last_max < 0) return LT_ERR_INVALID_ARG;
+  DecodePlan dp = make_decode_plan(*shape);
+  size_t decode_bytes = round_up(dp.ml_floats * 4, kWsAlign) + round_up(dp.o_floats * 4, kWsAlign);
+  size_t score_bytes = 0;
+  if (n_ctx_max > 0 && w_last_max > 0) {
+    ScorePlan sp = make_score_plan(*shape, n_ctx_max, w_last_max);
+    score_bytes = round_up(sp.stat_floats * 4, kWsAlign);
+  }
+  *bytes_out = kWsHeaderBytes + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
+  return LT_OK;
+}
+
+lt_status lt_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+  if (!ws || ws_bytes < kWsHeaderBytes || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
+  cudaError_t e = cudaMemsetAsync(ws, 0, kWsHeaderBytes, (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_check(void* ws, uint32_t* flags_out, void* stream) {
+  if (!ws) return LT_ERR_WORKSPACE;
+  uint32_t flags = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(&flags, ws, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LT_ERR_CUDA;
+  if (cudaMemsetAsync(ws, 0, sizeof(flags), st) != cudaSuccess) return LT_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LT_ERR_CUDA;
+  if (flags_out) *flags_out = flags;
+  return flags ? LT_ERR_DEVICE_RANGE : LT_OK;
+}
+
+lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* const* k_full, int32_t n_ctx,
+                         int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
+  if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
+  if (((uintptr_t)q_tail & 15u) != 0) return LT_ERR_INVALID_ARG;
+  LayerTable kf;
+  if ((st = fill_table(&kf, k_full, shape->n_layers, true)) != LT_OK) return st;
+  ScorePlan sp = make_score_plan(*shape, n_ctx, w_last);
+  if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
+  if (ws_bytes < kWsHeaderBytes + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
+  ScoreArgs a;
+  a.s = *shape;
+  a.q_tail = q_tail;
+  a.n_ctx = n_ctx;
+  a.w_last = w_last;
+  a.n_splits = sp.n_splits;
+  a.stats = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
+  a.scores = scores;
+  a.cs = resolved_scale(*shape) * 1.4426950408889634f;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e = scores_mma_supported(*shape, w_last) ? launch_scores_mma(a, kf, cs)
+                                                       : launch_scores_generic(a, kf, cs);
+  if (e != cudaSuccess) return LT_ERR_CUDA;
+  e = launch_scores_finish(a, cs);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_select_lazy(const float* scores, int32_t n_layers, int32_t batch, int32_t n_q_heads, int32_t n_lazy,
+                         uint8_t* layer_mask, float* layer_ratio, void* stream) {
+  if (!scores || !layer_mask) return LT_ERR_INVALID_ARG;
+  if (n_layers < 1 || batch < 1 || n_q_heads < 1) return LT_ERR_INVALID_ARG;
+  if (n_layers > LT_MAX_LAYERS) return LT_ERR_UNSUPPORTED;
+  if (n_lazy < 0 || n_lazy > n_layers) return LT_ERR_INVALID_ARG;
+  cudaError_t e = launch_select(scores, n_layers, batch, n_q_heads, n_lazy, layer_mask, layer_ratio,
+                                (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask, const void* const* k_full,
+                         const void* const* v_full, const int32_t* seq_lens, void* const* k_stream,
+                         void* const* v_stream, void* ws, void* stream) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!layer_mask || !k_full || !v_full || !seq_lens || !k_stream || !v_stream) return LT_ERR_INVALID_ARG;
+  if (ws && ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
+  LayerTable kf, vf, ks, vs;
+  const int L = shape->n_layers;
+  if ((st = fill_table(&kf, k_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vf, v_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&ks, (const void* const*)k_stream, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vs, (const void* const*)v_stream, L, false)) != LT_OK) return st;
+  cudaError_t e = launch_stream_init(*shape, layer_mask, kf, vf, seq_lens, ks, vs, ws ? err_word(ws) : nullptr,
+                                     (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask, const void* k_new, const void* v_new,
+                       int32_t* seq_lens, void* const* k_full, void* const* v_full, void* const* k_stream,
+                       void* const* v_stream, int32_t layer_begin, int32_t layer_count, int32_t advance_seq_lens,
+                       void* ws, void* stream) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!layer_mask || !k_new || !v_new || !seq_lens) return LT_ERR_INVALID_ARG;
+  if (!k_full && !k_stream) return LT_ERR_INVALID_ARG;
+  if ((k_full == nullptr) != (v_full == nullptr) || (k_stream == nullptr) != (v_stream == nullptr))
+    return LT_ERR_INVALID_ARG;
+  if ((((uintptr_t)k_new | (uintptr_t)v_new) & 15u) != 0) return LT_ERR_INVALID_ARG;
+  if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
+  if (ws && ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
+  LayerTable kf, vf, ks, vs;
+  const int L = shape->n_layers;
+  if ((st = fill_table(&kf, (const void* const*)k_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vf, (const void* const*)v_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&ks, (const void* const*)k_stream, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vs, (const void* const*)v_stream, L, false)) != LT_OK) return st;
+  cudaError_t e = launch_append(*shape, layer_mask, k_new, v_new, seq_lens, kf, vf, ks, vs, layer_begin, layer_count,
+                                advance_seq_lens, ws ? err_word(ws) : nullptr, (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q, const void* const* k_full,
+                                const void* const* v_full, const void* const* k_stream, const void* const* v_stream,
+                                const uint8_t* layer_mask, const int32_t* seq_lens, void* out, int32_t out_dtype,
+                                int32_t max_seq_len_hint, int32_t layer_begin, int32_t layer_count, void* ws,
+                                size_t ws_bytes, void* stream) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!q || !layer_mask || !seq_lens || !out) return LT_ERR_INVALID_ARG;
+  if (!k_full && !k_stream) return LT_ERR_INVALID_ARG;
+  if ((k_full == nullptr) != (v_full == nullptr) || (k_stream == nullptr) != (v_stream == nullptr))
+    return LT_ERR_INVALID_ARG;
+  if (out_dtype != LT_F32 && out_dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
+  if ((((uintptr_t)q | (uintptr_t)out) & 15u) != 0) return LT_ERR_INVALID_ARG;
+  if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
+  LayerTable kf, vf, ks, vs;
+  const int L = shape->n_layers;
+  if ((st = fill_table(&kf, k_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vf, v_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&ks, k_stream, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&vs, v_stream, L, false)) != LT_OK) return st;
+
+  DecodePlan dp = make_decode_plan(*shape);
+  const size_t ml_bytes = round_up(dp.ml_floats * 4, kWsAlign);
+  const size_t o_bytes = round_up(dp.o_floats * 4, kWsAlign);
+  if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
+  if (ws_bytes < kWsHeaderBytes + ml_bytes + o_bytes) return LT_ERR_WORKSPACE;
+
+  DecodeArgs a;
+  a.s = *shape;
+  a.q = q;
+  a.mask = layer_mask;
+  a.seq_lens = seq_lens;
+  a.out = out;
+  a.out_dtype = out_dtype;
+  a.layer_begin = layer_begin;
+  a.layer_count = layer_count;
+  a.chunk_keys = dp.chunk_keys;
+  a.n_chunks_max = dp.n_chunks_max;
+  a.n_chunks_launch = dp.n_chunks_max;
+  if (max_seq_len_hint > 0) {
+    int c = (max_seq_len_hint + dp.chunk_keys - 1) / dp.chunk_keys;
+    if (c < a.n_chunks_launch) a.n_chunks_launch = c;
+  }
+  a.part_ml = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
+  a.part_o = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes + ml_bytes);
+  a.dev_err = err_word(ws);
+  a.cs = resolved_scale(*shape) * 1.4426950408889634f;
+
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e = decode_mma_supported(*shape) ? launch_decode_mma(a, kf, vf, ks, vs, cs)
+                                               : launch_decode_generic(a, kf, vf, ks, vs, cs);
+  if (e != cudaSuccess) return LT_ERR_CUDA;
+  e = launch_decode_combine(a, cs);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+}  // extern "C"

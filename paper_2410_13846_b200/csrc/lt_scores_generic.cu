@@ -1,0 +1,158 @@
+// Lazy ratio (Eq. 1), reference-quality CUDA-core path (any dtype, head_dim 64
+// or 128), the merge kernel shared by all scoring paths, and the selection.
+//
+// Partial statistics of one tail row (layer, b, hq, t) over one key split, log2
+// domain with t_j = scale * log2(e) * (q . k_j):
+//   M = max_j t_j,  A = sum_j 2^(t_j - M),  W = sum_{j in window} 2^(t_j - M)
+// over the visible keys j <= n_ctx - w_last + t of the split; the window is
+// {j < n_sink} U {j >= n_ctx - n_recent}.
+#include <cuda_bf16.h>
+
+#include "lt_internal.h"
+
+namespace lt {
+
+template <typename T>
+__device__ __forceinline__ float ld_f32(const T* p);
+template <>
+__device__ __forceinline__ float ld_f32<float>(const float* p) {
+  return *p;
+}
+template <>
+__device__ __forceinline__ float ld_f32<__nv_bfloat16>(const __nv_bfloat16* p) {
+  return __bfloat162float(*p);
+}
+
+__host__ __device__ inline int score_split_len(int n_ctx, int n_splits) {
+  int len = (n_ctx + n_splits - 1) / n_splits;
+  return (len + 63) / 64 * 64;
+}
+
+// grid (w_last * n_splits, B * Hq, L); block 128.
+template <typename T, int D>
+__global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
+  const lt_shape& s = a.s;
+  const int t = blockIdx.x / a.n_splits, sp = blockIdx.x % a.n_splits;
+  const int b = blockIdx.y / s.n_q_heads, hq = blockIdx.y % s.n_q_heads;
+  const int l = blockIdx.z;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  const int h = hq / G;
+  __shared__ float qs[D];
+  __shared__ float red[3][128];
+  const T* qp = (const T*)a.q_tail + ((((long long)l * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * D;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) qs[d] = ld_f32<T>(qp + d);
+  __syncthreads();
+  const int i = a.n_ctx - a.w_last + t;  // position of this query; sees keys 0..i
+  const int len = score_split_len(a.n_ctx, a.n_splits);
+  const int j0 = sp * len;
+  const int j1 = min(i + 1, j0 + len);
+  const T* Kb = (const T*)kf.p[l] + ((long long)(b * s.n_kv_heads + h) * s.full_capacity) * D;
+  float M = -INFINITY, A = 0.f, W = 0.f;
+  for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
+    const T* kr = Kb + (long long)j * D;
+    float dot = 0.f;
+#pragma unroll 8
+    for (int d = 0; d < D; ++d) dot += qs[d] * ld_f32<T>(kr + d);
+    const float tj = dot * a.cs;
+    const float Mn = fmaxf(M, tj);
+    const float corr = exp2f(M - Mn), p = exp2f(tj - Mn);
+    A = A * corr + p;
+    W = W * corr + ((j < s.n_sink || j >= a.n_ctx - s.n_recent) ? p : 0.f);
+    M = Mn;
+  }
+  red[0][threadIdx.x] = M;
+  red[1][threadIdx.x] = A;
+  red[2][threadIdx.x] = W;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float Mx = -INFINITY;
+    for (int k = 0; k < 128; ++k) Mx = fmaxf(Mx, red[0][k]);
+    float As = 0.f, Ws = 0.f;
+    if (Mx > -INFINITY) {
+      for (int k = 0; k < 128; ++k) {
+        const float w = exp2f(red[0][k] - Mx);
+        As += w * red[1][k];
+        Ws += w * red[2][k];
+      }
+    }
+    float* st = a.stats +
+                ((((((long long)l * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * a.n_splits) + sp) * 3;
+    st[0] = Mx;
+    st[1] = As;
+    st[2] = Ws;
+  }
+}
+
+cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
+  dim3 grid(a.w_last * a.n_splits, a.s.batch * a.s.n_q_heads, a.s.n_layers);
+  const bool bf = a.s.dtype == LT_BF16;
+  if (a.s.head_dim == 128) {
+    if (bf) scores_generic_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(a, kf);
+    else scores_generic_kernel<float, 128><<<grid, 128, 0, st>>>(a, kf);
+  } else {
+    if (bf) scores_generic_kernel<__nv_bfloat16, 64><<<grid, 128, 0, st>>>(a, kf);
+    else scores_generic_kernel<float, 64><<<grid, 128, 0, st>>>(a, kf);
+  }
+  return cudaGetLastError();
+}
+
+// One thread per (layer, b, hq): merge the splits of every tail row, take the
+// row's mass W/A, average over the w_last rows in row order.
+__global__ void scores_finish_kernel(ScoreArgs a) {
+  const lt_shape& s = a.s;
+  const long long total = (long long)s.n_layers * s.batch * s.n_q_heads;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  float sum = 0.f;
+  for (int t = 0; t < a.w_last; ++t) {
+    const float* st = a.stats + ((idx * a.w_last + t) * a.n_splits) * 3;
+    float Mx = -INFINITY;
+    for (int sp = 0; sp < a.n_splits; ++sp) Mx = fmaxf(Mx, st[sp * 3]);
+    float A = 0.f, W = 0.f;
+    for (int sp = 0; sp < a.n_splits; ++sp) {
+      const float w = exp2f(st[sp * 3] - Mx);
+      A += w * st[sp * 3 + 1];
+      W += w * st[sp * 3 + 2];
+    }
+    sum += W / A;
+  }
+  a.scores[idx] = sum / (float)a.w_last;
+}
+
+cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st) {
+  const long long total = (long long)a.s.n_layers * a.s.batch * a.s.n_q_heads;
+  scores_finish_kernel<<<(unsigned)((total + 127) / 128), 128, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+// Selection: one CTA.  Thread l sums its layer's scores in double in index
+// order, then ranks itself by counting the layers that beat it under the total
+// order (ratio descending, index ascending).
+__global__ void select_kernel(const float* __restrict__ scores, int L, int per_layer, int n_lazy,
+                              uint8_t* __restrict__ mask, float* __restrict__ ratio) {
+  __shared__ double r[LT_MAX_LAYERS];
+  const int l = threadIdx.x;
+  if (l < L) {
+    double acc = 0.0;
+    const float* p = scores + (long long)l * per_layer;
+    for (int k = 0; k < per_layer; ++k) acc += (double)p[k];
+    r[l] = acc / (double)per_layer;
+  }
+  __syncthreads();
+  if (l < L) {
+    int rank = 0;
+    for (int m = 0; m < L; ++m) rank += (r[m] > r[l]) || (r[m] == r[l] && m < l);
+    mask[l] = rank < n_lazy ? 1 : 0;
+    if (ratio) ratio[l] = (float)r[l];
+  }
+}
+
+cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,
+                          cudaStream_t st) {
+  select_kernel<<<1, LT_MAX_LAYERS, 0, st>>>(scores, L, B * Hq, n_lazy, mask, ratio);
+  return cudaGetLastError();
+}
+
+// Tensor-core scoring path: provided by lt_scores_mma.cu.
+
+}  // namespace lt

@@ -1,0 +1,83 @@
+"""GPU parity: lt_lazy_scores (Eq. 1) and lt_select_lazy against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2410_13846_b200 as lt
+from oracle import lt_oracle as O
+from tests.gpu_util import SCORE_ABS, Stack, f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_scores(st, q_tail, n_ctx, T):
+    s = st.shape
+    scores = torch.full((s.n_layers, s.batch, s.n_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    lt.lazy_scores(s, q_tail, st.tables, n_ctx, T, scores, st.ws)
+    return scores
+
+
+def _oracle_scores(st, q_tail, n_ctx):
+    s = st.shape
+    scale = s.softmax_scale if s.softmax_scale > 0 else None
+    ref = np.zeros((s.n_layers, s.batch, s.n_q_heads))
+    for l in range(s.n_layers):
+        for b in range(s.batch):
+            ref[l, b] = O.lazy_scores(f64(q_tail[l, b]), f64(st.k_full[l][b, :, :n_ctx]), s.n_sink, s.n_recent, scale)
+    return ref
+
+
+CASES = [
+    # dtype, D, Hq, Hkv, S, R, n_ctx, T, scale
+    (torch.float32, 64, 4, 2, 4, 60, 512, 16, 0.0),        # toy
+    (torch.bfloat16, 128, 8, 2, 4, 60, 777, 64, 0.0),      # GQA 4, odd length
+    (torch.bfloat16, 128, 5, 1, 4, 28, 1300, 8, 0.0),      # GQA 5
+    (torch.bfloat16, 128, 2, 2, 0, 16, 130, 64, 0.2),      # MHA, no sink, T > R, custom scale
+    (torch.bfloat16, 128, 4, 1, 4, 2044, 2500, 64, 0.0),   # paper defaults
+    (torch.bfloat16, 128, 4, 1, 4, 60, 40, 40, 0.0),       # window covers everything -> 1.0
+    (torch.bfloat16, 64, 4, 2, 2, 9, 300, 5, 0.0),         # D=64
+    (torch.bfloat16, 128, 8, 2, 6, 252, 4100, 32, 0.0),    # several key splits
+]
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv,S,R,n_ctx,T,scale", CASES)
+def test_scores_match_oracle(dtype, D, Hq, Hkv, S, R, n_ctx, T, scale):
+    torch.manual_seed(5)
+    L, B = 2, 2
+    cap = n_ctx + 3
+    st = Stack(L, B, Hq, Hkv, D, S, R, cap, dtype, scale, n_ctx_max=n_ctx, w_last_max=T)
+    for l in range(L):
+        st.k_full[l][:, :, :n_ctx] = torch.randn(B, Hkv, n_ctx, D).to(dtype).cuda()
+        st.k_full[l][:, :, n_ctx:] = float("nan")               # never read
+    q_tail = (1.3 * torch.randn(L, B, Hq, T, D)).to(dtype).cuda()
+    got = f64(_run_scores(st, q_tail, n_ctx, T))
+    ref = _oracle_scores(st, q_tail, n_ctx)
+    assert np.isfinite(got).all()
+    assert np.max(np.abs(got - ref)) <= SCORE_ABS, np.max(np.abs(got - ref))
+    if S + R >= n_ctx:
+        assert np.max(np.abs(got - 1.0)) <= 1e-5
+    assert torch.equal(_run_scores(st, q_tail, n_ctx, T), torch.from_numpy(got).float().cuda())   # deterministic
+
+
+def test_select_fed_oracle_scores_is_bit_exact():
+    g = np.random.default_rng(6)
+    for L, B, Hq in [(2, 1, 4), (32, 8, 32), (64, 4, 40), (7, 3, 5), (128, 1, 1)]:
+        sc = g.random((L, B, Hq)).astype(np.float32)
+        d = torch.from_numpy(sc).cuda()
+        for n_lazy in sorted({0, 1, L // 4, L // 2, L - 1, L}):
+            mask = torch.full((L,), 9, dtype=torch.uint8, device="cuda")
+            ratio = torch.zeros(L, dtype=torch.float32, device="cuda")
+            lt.select_lazy(d, L, B, Hq, n_lazy, mask, ratio)
+            em, er = O.select_lazy(sc, n_lazy)
+            assert np.array_equal(mask.cpu().numpy(), em)
+            assert np.allclose(ratio.cpu().numpy(), er, rtol=0, atol=1e-7)
+            assert np.array_equal(O.select_lazy_priority_queue(er, L - n_lazy), em)
+
+
+def test_select_ties_go_to_lower_index():
+    sc = np.array([0.5, 0.9, 0.5, 0.9, 0.1, 0.9], dtype=np.float32).reshape(6, 1, 1).repeat(3, axis=2)
+    d = torch.from_numpy(sc).cuda()
+    for n_lazy in range(7):
+        mask = torch.zeros(6, dtype=torch.uint8, device="cuda")
+        lt.select_lazy(d, 6, 1, 3, n_lazy, mask)
+        assert np.array_equal(mask.cpu().numpy(), O.select_lazy(sc, n_lazy)[0])
