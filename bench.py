@@ -447,6 +447,26 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_profile_case(args):
+    """Small case of the same kernels for profiler captures: 4 layers (2 lazy) of
+    the benchmark's stack (about 5 GB on the device, K/V per step far above the
+    L2), one warm-up pass and one pass of a few decode steps, nothing else."""
+    assert torch.cuda.is_available()
+    torch.cuda.set_device(0)
+    from paper_2410_13846_b200 import build
+    build.build_library()
+    from synth import CONFIGS
+    cfg = CONFIGS[WORKLOAD].scaled(n_layers=4, n_lazy=2, steps=args.profile_case)
+    wl = Workload(cfg, torch.device("cuda", 0))
+    wl.full_pass()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    wl.full_pass()
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": cfg.name, "layers": cfg.n_layers, "decode_steps": cfg.steps,
+                      "pass_s": time.perf_counter() - t0, "mask": wl.mask.cpu().tolist()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -454,8 +474,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-case", type=int, default=0, metavar="DECODE_STEPS",
+                    help="run the 4-layer small case with this many decode steps per pass (for ncu) and exit")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_case > 0:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
