@@ -201,6 +201,39 @@ lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q /* dev */,
                                 int32_t layer_begin, int32_t layer_count, void* ws /* dev */,
                                 size_t ws_bytes, void* stream);
 
+/*
+ * The decode-attention step for callers that cannot allocate device memory.
+ * (No counterpart in the paper: this is a deployment convenience of the library.)
+ *
+ * Some hosts are handed pointers but no allocator - a serving engine that has
+ * already given all free HBM to its KV-cache pool, a plug-in inside another
+ * program's memory plan, a loop in which cudaMalloc would stall the device.
+ * This call is lt_hybrid_decode_attn without the workspace arguments: the
+ * split-KV partials live in a fixed array of LT_STATIC_SCRATCH_BYTES inside the
+ * library image, resident on every GPU that loads the library until the process
+ * exits.  The call allocates and frees nothing.
+ *
+ *   - Same arguments, layouts and result as lt_hybrid_decode_attn.
+ *   - dev_error (dev, may be NULL): receives this call's error word (the
+ *     LT_DEVERR_* bits), stream-ordered; there is no workspace to lt_check.
+ *   - A shape whose lt_workspace_bytes(shape, 0, 0, ..) exceeds
+ *     LT_STATIC_SCRATCH_BYTES returns LT_ERR_WORKSPACE before any device work.
+ *   - The first call on each device looks up the array's device address; make
+ *     that call before beginning any stream capture.
+ *   - All calls on a device share the array, which still holds the previous
+ *     call's partials.  The error word is cleared at the start of every call and
+ *     partials are written before they are read, so calls in stream order are
+ *     independent; calls that overlap on the GPU race and must be serialised.
+ */
+#define LT_STATIC_SCRATCH_BYTES (16u << 20)
+lt_status lt_hybrid_decode_attn_static(const lt_shape* shape, const void* q /* dev */,
+                                       const void* const* k_full, const void* const* v_full,
+                                       const void* const* k_stream, const void* const* v_stream /* host tables */,
+                                       const uint8_t* layer_mask /* dev */, const int32_t* seq_lens /* dev */,
+                                       void* out /* dev */, int32_t out_dtype, int32_t max_seq_len_hint,
+                                       int32_t layer_begin, int32_t layer_count,
+                                       uint32_t* dev_error /* dev, may be NULL */, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -208,3 +208,31 @@ def hybrid_decode_attn(shape: Shape, q, tables: LayerTables, layer_mask, seq_len
                                     tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
                                     max_seq_len_hint, layer_begin, cnt, _ptr(ws), ws.numel() * ws.element_size(),
                                     _stream(stream)), "lt_hybrid_decode_attn")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def hybrid_decode_attn_static(shape: Shape, q, tables: LayerTables, layer_mask, seq_lens, out, out_dtype: int | None = None,
+                              max_seq_len_hint: int = 0, layer_begin: int = 0, layer_count: int | None = None,
+                              dev_error=None, stream=None):
+    """lt_hybrid_decode_attn_static: the decode step for callers that cannot
+    allocate device memory (the scratch is a fixed array inside the library).
+    ``dev_error`` is an optional uint32/int32 CUDA tensor of one element that
+    receives the call's error word."""
+    import torch
+    L = lib()
+    if not hasattr(L.lt_hybrid_decode_attn_static, "_lt_typed"):
+        vp, i32 = C.c_void_p, C.c_int32
+        tab = C.POINTER(C.c_void_p)
+        L.lt_hybrid_decode_attn_static.restype = i32
+        L.lt_hybrid_decode_attn_static.argtypes = [C.POINTER(_CShape), vp, tab, tab, tab, tab, vp, vp, vp, i32, i32,
+                                                   i32, i32, vp, vp]
+        L.lt_hybrid_decode_attn_static._lt_typed = True
+    if out_dtype is None:
+        out_dtype = LT_F32 if out.dtype == torch.float32 else LT_BF16
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(L.lt_hybrid_decode_attn_static(C.byref(shape.c()), _ptr(q), tables.k_full, tables.v_full, tables.k_stream,
+                                       tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
+                                       max_seq_len_hint, layer_begin, cnt, _ptr(dev_error), _stream(stream)),
+        "lt_hybrid_decode_attn_static")
