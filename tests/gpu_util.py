@@ -68,3 +68,22 @@ def attn_errors(got: np.ndarray, ref: np.ndarray):
 ATTN_MAX_ABS = 1e-2
 ATTN_REL_L2 = 2e-3
 SCORE_ABS = 1e-3
+
+
+def build_stack(cfg, steps=None):
+    """Device state of a synth workload: prompt K/V in the full caches of every
+    layer, tail queries, seq_lens at the prompt length.  Returns (stack, q_tail,
+    planted layers)."""
+    from synth import make_layer, planted_layers, torch_dtype
+    dt = torch_dtype(cfg)
+    cap = cfg.n_ctx + (cfg.steps if steps is None else steps)
+    st = Stack(cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_sink, cfg.n_recent, cap,
+               dt, 0.0, n_ctx_max=cfg.n_ctx, w_last_max=cfg.w_last)
+    planted = planted_layers(cfg)
+    q_tail = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.w_last, cfg.head_dim), dtype=dt, device="cuda")
+    for l in range(cfg.n_layers):
+        qt, K, V = make_layer(cfg, l, l in planted, "cuda", capacity=cap)
+        q_tail[l].copy_(qt); st.k_full[l].copy_(K); st.v_full[l].copy_(V)
+        del qt, K, V
+    st.set_seq_lens([cfg.n_ctx] * cfg.batch)
+    return st, q_tail, planted

@@ -8,25 +8,10 @@ import torch
 
 import paper_2410_13846_b200 as lt
 from oracle import lt_oracle as O
-from synth import CONFIGS, decode_inputs, make_layer, planted_layers, torch_dtype
-from tests.gpu_util import ATTN_MAX_ABS, ATTN_REL_L2, SCORE_ABS, Stack, attn_errors, bits, f64
+from synth import CONFIGS, decode_inputs
+from tests.gpu_util import ATTN_MAX_ABS, ATTN_REL_L2, SCORE_ABS, attn_errors, bits, build_stack as _build, f64
 
 pytestmark = pytest.mark.gpu
-
-
-def _build(cfg, steps=None):
-    dt = torch_dtype(cfg)
-    cap = cfg.n_ctx + (cfg.steps if steps is None else steps)
-    st = Stack(cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_sink, cfg.n_recent, cap,
-               dt, 0.0, n_ctx_max=cfg.n_ctx, w_last_max=cfg.w_last)
-    planted = planted_layers(cfg)
-    q_tail = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.w_last, cfg.head_dim), dtype=dt, device="cuda")
-    for l in range(cfg.n_layers):
-        qt, K, V = make_layer(cfg, l, l in planted, "cuda", capacity=cap)
-        q_tail[l].copy_(qt); st.k_full[l].copy_(K); st.v_full[l].copy_(V)
-        del qt, K, V
-    st.set_seq_lens([cfg.n_ctx] * cfg.batch)
-    return st, q_tail, planted
 
 
 def test_toy_stack_every_element():
