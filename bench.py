@@ -55,6 +55,35 @@ def _dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+def init_replicas(world: int, backend: str = "nccl", device=None):
+    """Process group of the replicas (None for a single process).  The path has
+    no exchange step: the group is used for the barrier around the timed region
+    and for the max-over-ranks of the measured time, never for data."""
+    if world <= 1:
+        return None
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=device)
+    else:
+        dist.init_process_group(backend)
+    return dist
+
+
+def max_over_ranks(x: float, dist, device=None) -> float:
+    """Slowest rank's time: every replica must have finished its steps."""
+    if dist is None:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, tokens_per_rank: int, ms: float) -> float:
+    """tokens/s of all replicas together over the slowest rank's time."""
+    return world * tokens_per_rank / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------
 # clocks sampling during the timed region
 # ----------------------------------------------------------------------------
@@ -192,10 +221,7 @@ def run_ours(args):
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
+    dist = init_replicas(world, "nccl", device)
 
     from paper_2410_13846_b200 import build
     build.build_library()
@@ -240,16 +266,13 @@ def run_ours(args):
     clocks = sampler.stop()
     total_ms = t0.elapsed_time(t1)
     launches = wl.launches
-    if dist is not None:
-        tt = torch.tensor([total_ms], device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms, dist, device)
     attn_ms = np.array([[a.elapsed_time(b) for a, b in ev] for ev in events])          # [K, T]
     ident_ms = np.array([a.elapsed_time(b) for a, b in e_id])
     decode_ms_total = total_ms - float(ident_ms.sum())
 
     # ---- derived numbers ----------------------------------------------------------
-    value = world * B * T * K / (total_ms * 1e-3)
+    value = whole_job_value(world, B * T * K, total_ms)
     bytes_per_step = np.array([algorithmic_bytes_decode(cfg, cfg.n_ctx + i + 1, cfg.n_lazy) for i in range(T)])
     attn_gbs = float(bytes_per_step.sum() * K / (attn_ms.sum() * 1e-3) / 1e9)
     peak, peak_kind = _peaks()
@@ -273,11 +296,8 @@ def run_ours(args):
 
     # ---- end to end through the public API with host buffers ----------------------
     e2e = run_e2e(wl, passes=max(1, min(K, 2)))
-    if dist is not None:
-        te = torch.tensor([e2e["ms_per_pass"]], device=device)
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e["ms_per_pass"] = float(te.item())
-    e2e_value = world * B * T / (e2e["ms_per_pass"] * 1e-3)
+    e2e["ms_per_pass"] = max_over_ranks(e2e["ms_per_pass"], dist, device)
+    e2e_value = whole_job_value(world, B * T, e2e["ms_per_pass"])
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
