@@ -63,6 +63,7 @@ enum { LT_F32 = 0, LT_BF16 = 1 };
 #define LT_DEVERR_POS_OUT_OF_RANGE 1u /* append: seq_len >= full_capacity; store skipped */
 #define LT_DEVERR_NULL_LAYER 2u       /* mask selected a layer whose table entry is NULL */
 #define LT_DEVERR_LEN_CLAMPED 4u      /* attend: seq_len > full_capacity; clamped */
+#define LT_DEVERR_TIMEOUT 8u          /* scoring: a bounded wait inside a kernel expired; scores invalid */
 
 typedef struct lt_shape {
   int32_t n_layers;      /* L, 1..LT_MAX_LAYERS */

@@ -2,6 +2,7 @@
 // stream-ordered launches.  No device memory is allocated here and no state
 // survives a call.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "lt_internal.h"
@@ -147,9 +148,16 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* 
   a.stats = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
   a.scores = scores;
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
+  a.dev_err = err_word(ws);
   cudaStream_t cs = (cudaStream_t)stream;
-  cudaError_t e = scores_mma_supported(*shape, w_last) ? launch_scores_mma(a, kf, cs)
-                                                       : launch_scores_generic(a, kf, cs);
+  // LT_SCORES_IMPL = umma | mma | generic picks a path explicitly (for A/B measurements).
+  const char* impl = getenv("LT_SCORES_IMPL");
+  cudaError_t e;
+  if (impl && !strcmp(impl, "generic")) e = launch_scores_generic(a, kf, cs);
+  else if (impl && !strcmp(impl, "mma") && scores_mma_supported(*shape, w_last)) e = launch_scores_mma(a, kf, cs);
+  else if (scores_umma_supported(*shape, w_last)) e = launch_scores_umma(a, kf, cs);
+  else if (scores_mma_supported(*shape, w_last)) e = launch_scores_mma(a, kf, cs);
+  else e = launch_scores_generic(a, kf, cs);
   if (e != cudaSuccess) return LT_ERR_CUDA;
   e = launch_scores_finish(a, cs);
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;

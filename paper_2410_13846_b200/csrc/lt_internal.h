@@ -84,10 +84,14 @@ struct ScoreArgs {
   float cs;      // softmax scale * log2(e)
   float* stats;  // workspace
   float* scores;
+  uint32_t* dev_err;
 };
 cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
 bool scores_mma_supported(const lt_shape& s, int w_last);
 cudaError_t launch_scores_mma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
+// bf16, head_dim 128: tcgen05 / TMEM path.
+bool scores_umma_supported(const lt_shape& s, int w_last);
+cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
 cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st);
 
 cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask,

@@ -60,6 +60,8 @@ def test_toy_stack_every_element():
 
 def test_llama3_8b_32k_sampled_units():
     """Full-size target configuration (about 40 GB on the device)."""
+    import gc
+    gc.collect(); torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 60 * 2**30:
         pytest.skip("needs ~40 GB of free device memory")

@@ -15,6 +15,8 @@ pytestmark = pytest.mark.gpu
 
 
 def _need_gb(gb):
+    import gc
+    gc.collect(); torch.cuda.empty_cache()          # earlier tests' blocks sit in torch's cache
     free, _ = torch.cuda.mem_get_info()
     if free < gb * 2**30:
         pytest.skip(f"needs ~{gb} GB of free device memory")
