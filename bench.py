@@ -5,7 +5,8 @@ sink 4 + window 2044, 16 lazy layers, 128 decode steps).
 
 One "step" of this benchmark is one whole pass of the hot path over one batch:
 lazy scores over the last 64 prompt queries -> device top-k -> compaction of the
-lazy layers -> 128 x (KV append + hybrid decode attention over all 32 layers).
+lazy layers -> 128 x (one fused launch: KV append + hybrid decode attention over
+all 32 layers + seq_lens advance).
 `value` = decode tokens of all ranks / time of the timed passes.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
@@ -195,13 +196,13 @@ class Workload:
     def decode_step(self, i, ev=None):
         lt = self.lt
         q, k, v = self.step_inputs[i % len(self.step_inputs)]
-        lt.kv_append(self.shape, self.mask, k, v, self.seq, self.tables, ws=self.ws)
         if ev is not None:
             ev[0].record()
-        lt.hybrid_decode_attn(self.shape, q, self.tables, self.mask, self.seq, self.out, self.ws)
+        # append + attend + merge + seq_lens advance: one launch
+        lt.decode_step(self.shape, q, k, v, self.tables, self.mask, self.seq, self.out, self.ws)
         if ev is not None:
             ev[1].record()
-        self.launches += 4
+        self.launches += 1
 
     def full_pass(self, events=None):
         self.identify()
@@ -313,7 +314,7 @@ def run_ours(args):
                        "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim, "batch": B, "context": cfg.n_ctx,
                        "n_sink": cfg.n_sink, "n_recent": cfg.n_recent, "w_last": cfg.w_last, "n_lazy": cfg.n_lazy,
                        "decode_steps_per_pass": T,
-                       "step": "scores+select+compaction+128x(append+attend)",
+                       "step": "scores+select+compaction+128x(fused append+attend)",
                        "l2": "inputs (17 GiB per decode step) exceed the 126 MB L2; no flush needed",
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
@@ -322,7 +323,7 @@ def run_ours(args):
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peak, "unit": "GB/s", "frac": attn_gbs / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": attn_gbs / NOMINAL_HBM_GBS,
-                         "kernel": "lt_hybrid_decode_attn (split-KV kernel + combine), hybrid mask",
+                         "kernel": "lt_decode_step (persistent split-KV kernel: append + attend + merge), hybrid mask",
                          "algorithmic_bytes_per_launch": float(bytes_per_step.mean()),
                          "ms_per_launch": float(attn_ms.mean()),
                          "traffic": (float(bytes_per_step.mean()) * NCU_TRAFFIC_RATIO) if NCU_TRAFFIC_RATIO else None},
@@ -367,8 +368,7 @@ def run_e2e(wl, passes):
         for i in range(cfg.steps):
             hq, hk, hv = h_steps[i % len(h_steps)]
             d_q.copy_(hq, non_blocking=True); d_k.copy_(hk, non_blocking=True); d_v.copy_(hv, non_blocking=True)
-            lt.kv_append(wl.shape, wl.mask, d_k, d_v, wl.seq, wl.tables, ws=wl.ws)
-            lt.hybrid_decode_attn(wl.shape, d_q, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
+            lt.decode_step(wl.shape, d_q, d_k, d_v, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
             h_out.copy_(wl.out, non_blocking=True)
             torch.cuda.current_stream().synchronize()       # the caller consumes the step's result
 

@@ -96,14 +96,15 @@ int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent);
  * Bytes of workspace that lt_lazy_scores (prompt length up to n_ctx_max, up to
  * w_last_max tail queries) and lt_hybrid_decode_attn (any seq_len up to
  * max(full_capacity, n_sink + n_recent)) need for this shape.  Host only.
- * The workspace is device memory, 256-byte aligned, owned by the caller; its
- * first 256 bytes hold the device error word and must be zeroed once with
- * lt_workspace_init.  Two calls that overlap on the device must not share it.
+ * The workspace is device memory, 256-byte aligned, owned by the caller; it
+ * starts with the device error word and the counters of the decode step, which
+ * must be zeroed once with lt_workspace_init (every call leaves them zero).
+ * Two calls that overlap on the device must not share it.
  */
 lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max,
                              size_t* bytes_out /* host */);
 
-/* Zero the workspace header (async on `stream`). */
+/* Zero the workspace (async on `stream`); once, before its first use. */
 lt_status lt_workspace_init(void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
@@ -186,13 +187,12 @@ lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask /* dev *
  *           linearly).
  *   q    dev [L][B][Hq][D], dtype of the shape
  *   out  dev [L][B][Hq][D], LT_F32 or LT_BF16 (out_dtype); zeros where n = 0
- *   max_seq_len_hint  host upper bound on max_b seq_lens[b], used only to size
- *           the launch; <= 0 means full_capacity.  A seq_len above the hint is
- *           still handled correctly only up to the hint rounded up to the
- *           split size, so pass a true bound (or 0).
+ *   max_seq_len_hint  ignored (kept for source compatibility): the launch
+ *           sizes itself from the device-side lengths.
  *   layers [layer_begin, layer_begin + layer_count).
  * Split-KV: partial (max, sum, weighted values) per KV chunk go to the
- * workspace and a second kernel merges them.
+ * workspace; the last chunk of each (layer, b, kv head) to finish merges them
+ * in chunk order inside the same launch.  batch <= 2048.
  */
 lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q /* dev */,
                                 const void* const* k_full, const void* const* v_full,
@@ -201,6 +201,30 @@ lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q /* dev */,
                                 void* out /* dev */, int32_t out_dtype, int32_t max_seq_len_hint,
                                 int32_t layer_begin, int32_t layer_count, void* ws /* dev */,
                                 size_t ws_bytes, void* stream);
+
+/*
+ * One whole decode step in a single launch: lt_kv_append followed by
+ * lt_hybrid_decode_attn (Section 3: each decoding step saves the new token's KV
+ * and attends over the cache; the experimental setup of Appendix A runs that as
+ * one cache-updating attention call).  With p = seq_lens[b]:
+ *   - k_new / v_new [L][B][Hkv][D] are stored at row p of the full cache
+ *     (mask 0) or row lt_ring_slot(p) of the stream cache (mask 1), exactly as
+ *     lt_kv_append does; p >= full_capacity in a full layer skips the store
+ *     and raises LT_DEVERR_POS_OUT_OF_RANGE;
+ *   - out [L][B][Hq][D] is the attention of q over the p + 1 tokens (full
+ *     layers) or the min(p + 1, n_sink + n_recent) retained tokens (lazy
+ *     layers), exactly as lt_hybrid_decode_attn would return after the append;
+ *   - seq_lens[b] += 1 at the end of the launch when advance_seq_lens != 0
+ *     (a per-layer caller passes 0 except for its last layer).
+ * The workspace must have been zeroed once by lt_workspace_init.  Results are
+ * bit-identical to the two separate calls.
+ */
+lt_status lt_decode_step(const lt_shape* shape, const void* q /* dev */, const void* k_new /* dev */,
+                         const void* v_new /* dev */, void* const* k_full, void* const* v_full,
+                         void* const* k_stream, void* const* v_stream /* host tables */,
+                         const uint8_t* layer_mask /* dev */, int32_t* seq_lens /* dev [B] */, void* out /* dev */,
+                         int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int32_t advance_seq_lens,
+                         void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
  * The decode-attention step for callers that cannot allocate device memory.

@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
     L.lt_kv_append.argtypes = [shp, vp, vp, vp, vp, tab, tab, tab, tab, i32, i32, i32, vp, vp]
     L.lt_hybrid_decode_attn.restype = i32
     L.lt_hybrid_decode_attn.argtypes = [shp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
+    L.lt_decode_step.restype = i32
+    L.lt_decode_step.argtypes = [shp, vp, vp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
     _LIB = L
     return L
 
@@ -208,6 +210,20 @@ def hybrid_decode_attn(shape: Shape, q, tables: LayerTables, layer_mask, seq_len
                                     tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
                                     max_seq_len_hint, layer_begin, cnt, _ptr(ws), ws.numel() * ws.element_size(),
                                     _stream(stream)), "lt_hybrid_decode_attn")
+
+
+def decode_step(shape: Shape, q, k_new, v_new, tables: LayerTables, layer_mask, seq_lens, out, ws,
+                out_dtype: int | None = None, layer_begin: int = 0, layer_count: int | None = None,
+                advance_seq_lens: bool = True, stream=None):
+    """lt_decode_step: KV append + hybrid attention (+ seq_lens advance) in one launch."""
+    import torch
+    if out_dtype is None:
+        out_dtype = LT_F32 if out.dtype == torch.float32 else LT_BF16
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_decode_step(C.byref(shape.c()), _ptr(q), _ptr(k_new), _ptr(v_new), tables.k_full, tables.v_full,
+                             tables.k_stream, tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
+                             layer_begin, cnt, 1 if advance_seq_lens else 0, _ptr(ws),
+                             ws.numel() * ws.element_size(), _stream(stream)), "lt_decode_step")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

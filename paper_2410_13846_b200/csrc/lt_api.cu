@@ -50,6 +50,26 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last) {
   return p;
 }
 
+size_t ws_prefix_bytes(const lt_shape& s) {
+  const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads + 2) * sizeof(int);
+  return kWsHeaderBytes + round_up(counters, kWsAlign);
+}
+
+int persistent_grid(const DecodeArgs& a, int ctas_per_sm) {
+  static int sm_count[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  if (sm_count[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    sm_count[dev] = n;
+  }
+  const long long most = (long long)a.layer_count * a.s.batch * a.s.n_kv_heads * a.n_chunks_max;
+  long long grid = (long long)sm_count[dev] * ctas_per_sm;
+  if (grid > most) grid = most;
+  return (int)(grid < 1 ? 1 : grid);
+}
+
 static lt_status fill_table(LayerTable* t, const void* const* host, int L, bool require_all) {
   memset(t, 0, sizeof(*t));
   if (!host) return require_all ? LT_ERR_INVALID_ARG : LT_OK;
@@ -87,7 +107,7 @@ const char* lt_status_string(lt_status s) {
   }
 }
 
-int32_t lt_version(void) { return 100; }
+int32_t lt_version(void) { return 200; }
 
 int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent) {
   if (pos < 0 || n_sink < 0 || n_recent < 1) return -1;
@@ -106,13 +126,14 @@ lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w
     ScorePlan sp = make_score_plan(*shape, n_ctx_max, w_last_max);
     score_bytes = round_up(sp.stat_floats * 4, kWsAlign);
   }
-  *bytes_out = kWsHeaderBytes + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
+  *bytes_out = ws_prefix_bytes(*shape) + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
   return LT_OK;
 }
 
 lt_status lt_workspace_init(void* ws, size_t ws_bytes, void* stream) {
   if (!ws || ws_bytes < kWsHeaderBytes || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
-  cudaError_t e = cudaMemsetAsync(ws, 0, kWsHeaderBytes, (cudaStream_t)stream);
+  // error word and the decode step's counters start at zero; the rest is scratch
+  cudaError_t e = cudaMemsetAsync(ws, 0, ws_bytes, (cudaStream_t)stream);
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 
@@ -138,14 +159,15 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* 
   if ((st = fill_table(&kf, k_full, shape->n_layers, true)) != LT_OK) return st;
   ScorePlan sp = make_score_plan(*shape, n_ctx, w_last);
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
-  if (ws_bytes < kWsHeaderBytes + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
+  const size_t prefix = ws_prefix_bytes(*shape);
+  if (ws_bytes < prefix + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
   ScoreArgs a;
   a.s = *shape;
   a.q_tail = q_tail;
   a.n_ctx = n_ctx;
   a.w_last = w_last;
   a.n_splits = sp.n_splits;
-  a.stats = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
+  a.stats = reinterpret_cast<float*>((char*)ws + prefix);
   a.scores = scores;
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
   a.dev_err = err_word(ws);
@@ -216,20 +238,23 @@ lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask, const v
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 
-lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q, const void* const* k_full,
-                                const void* const* v_full, const void* const* k_stream, const void* const* v_stream,
-                                const uint8_t* layer_mask, const int32_t* seq_lens, void* out, int32_t out_dtype,
-                                int32_t max_seq_len_hint, int32_t layer_begin, int32_t layer_count, void* ws,
-                                size_t ws_bytes, void* stream) {
+// Shared body of lt_hybrid_decode_attn (k_new == NULL) and lt_decode_step.
+static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+                             const void* const* k_full, const void* const* v_full, const void* const* k_stream,
+                             const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
+                             int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
+                             void* ws, size_t ws_bytes, void* stream) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q || !layer_mask || !seq_lens || !out) return LT_ERR_INVALID_ARG;
+  if (fused && (!k_new || !v_new)) return LT_ERR_INVALID_ARG;
   if (!k_full && !k_stream) return LT_ERR_INVALID_ARG;
   if ((k_full == nullptr) != (v_full == nullptr) || (k_stream == nullptr) != (v_stream == nullptr))
     return LT_ERR_INVALID_ARG;
   if (out_dtype != LT_F32 && out_dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
-  if ((((uintptr_t)q | (uintptr_t)out) & 15u) != 0) return LT_ERR_INVALID_ARG;
+  if ((((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15u) != 0) return LT_ERR_INVALID_ARG;
   if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
+  if (shape->batch > kMaxWorkEntries) return LT_ERR_UNSUPPORTED;
   LayerTable kf, vf, ks, vs;
   const int L = shape->n_layers;
   if ((st = fill_table(&kf, k_full, L, false)) != LT_OK) return st;
@@ -238,38 +263,67 @@ lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q, const void
   if ((st = fill_table(&vs, v_stream, L, false)) != LT_OK) return st;
 
   DecodePlan dp = make_decode_plan(*shape);
+  const size_t prefix = ws_prefix_bytes(*shape);
   const size_t ml_bytes = round_up(dp.ml_floats * 4, kWsAlign);
   const size_t o_bytes = round_up(dp.o_floats * 4, kWsAlign);
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
-  if (ws_bytes < kWsHeaderBytes + ml_bytes + o_bytes) return LT_ERR_WORKSPACE;
+  if (ws_bytes < prefix + ml_bytes + o_bytes) return LT_ERR_WORKSPACE;
 
   DecodeArgs a;
   a.s = *shape;
   a.q = q;
+  a.k_new = k_new;
+  a.v_new = v_new;
   a.mask = layer_mask;
   a.seq_lens = seq_lens;
+  a.seq_lens_rw = seq_lens;
   a.out = out;
   a.out_dtype = out_dtype;
-  a.layer_begin = layer_begin;
-  a.layer_count = layer_count;
   a.chunk_keys = dp.chunk_keys;
   a.n_chunks_max = dp.n_chunks_max;
-  a.n_chunks_launch = dp.n_chunks_max;
-  if (max_seq_len_hint > 0) {
-    int c = (max_seq_len_hint + dp.chunk_keys - 1) / dp.chunk_keys;
-    if (c < a.n_chunks_launch) a.n_chunks_launch = c;
-  }
-  a.part_ml = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
-  a.part_o = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes + ml_bytes);
+  a.fused = fused;
+  a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
+  a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;
+  a.work_counter = a.done_counter + 1;
+  a.part_ml = reinterpret_cast<float*>((char*)ws + prefix);
+  a.part_o = reinterpret_cast<float*>((char*)ws + prefix + ml_bytes);
   a.dev_err = err_word(ws);
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
 
+  // One launch takes at most kMaxWorkEntries (layer, batch row) pairs; a larger
+  // stack goes in consecutive launches by layers (only the last one advances).
   cudaStream_t cs = (cudaStream_t)stream;
-  cudaError_t e = decode_mma_supported(*shape) ? launch_decode_mma(a, kf, vf, ks, vs, cs)
-                                               : launch_decode_generic(a, kf, vf, ks, vs, cs);
-  if (e != cudaSuccess) return LT_ERR_CUDA;
-  e = launch_decode_combine(a, cs);
-  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+  const int layers_per_launch = kMaxWorkEntries / shape->batch;
+  const bool mma = decode_mma_supported(*shape);
+  for (int done = 0; done < layer_count; done += layers_per_launch) {
+    a.layer_begin = layer_begin + done;
+    a.layer_count = layer_count - done < layers_per_launch ? layer_count - done : layers_per_launch;
+    a.advance = (advance && done + a.layer_count == layer_count) ? 1 : 0;
+    cudaError_t e = mma ? launch_decode_mma(a, kf, vf, ks, vs, cs) : launch_decode_generic(a, kf, vf, ks, vs, cs);
+    if (e != cudaSuccess) return LT_ERR_CUDA;
+  }
+  return LT_OK;
+}
+
+lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q, const void* const* k_full,
+                                const void* const* v_full, const void* const* k_stream, const void* const* v_stream,
+                                const uint8_t* layer_mask, const int32_t* seq_lens, void* out, int32_t out_dtype,
+                                int32_t max_seq_len_hint, int32_t layer_begin, int32_t layer_count, void* ws,
+                                size_t ws_bytes, void* stream) {
+  (void)max_seq_len_hint;  // the persistent launch sizes itself from the device-side lengths
+  return decode_impl(shape, q, nullptr, nullptr, k_full, v_full, k_stream, v_stream, layer_mask,
+                     const_cast<int32_t*>(seq_lens), out, out_dtype, layer_begin, layer_count, 0, 0, ws, ws_bytes,
+                     stream);
+}
+
+lt_status lt_decode_step(const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+                         void* const* k_full, void* const* v_full, void* const* k_stream, void* const* v_stream,
+                         const uint8_t* layer_mask, int32_t* seq_lens, void* out, int32_t out_dtype,
+                         int32_t layer_begin, int32_t layer_count, int32_t advance_seq_lens, void* ws,
+                         size_t ws_bytes, void* stream) {
+  return decode_impl(shape, q, k_new, v_new, (const void* const*)k_full, (const void* const*)v_full,
+                     (const void* const*)k_stream, (const void* const*)v_stream, layer_mask, seq_lens, out, out_dtype,
+                     layer_begin, layer_count, 1, advance_seq_lens ? 1 : 0, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -1,0 +1,262 @@
+// Pieces shared by the decode-step kernels (tensor-core and CUDA-core paths):
+// the flattened work list of a persistent launch, the fused KV append, and the
+// in-kernel merge of the split-KV partials by the last CTA of each unit.
+//
+// A decode step over a hybrid stack is very uneven: a full layer at 32K context
+// has sixteen 2048-key chunks per (batch row, kv head), a lazy layer has one.
+// Which layers are lazy is known on the device only (layer_mask), so instead of
+// a rectangular grid with mostly empty CTAs for the lazy layers, the kernels
+// launch a fixed number of CTAs (a multiple of the SM count) and every CTA walks
+// the same work list:
+//   entry e = (layer, batch row)      n_e = visible keys, nc_e = chunks
+//   items of e = n_kv_heads * nc_e    item -> (kv head, chunk)
+// The prefix sum over entries lives in shared memory; an item index is turned
+// into (entry, kv head, chunk) by binary search.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "lt_internal.h"
+
+namespace lt {
+
+struct WorkItem {
+  int l, b, h, c;  // layer, batch row, kv head, chunk
+  int nc;          // chunks of this (layer, batch row)
+  int n;           // visible keys of this (layer, batch row), clamped to the cache
+  int j0, j1;      // key rows [j0, j1) of this chunk
+  int rows;        // rows per (b, kv head) of the cache that is read
+  int new_row;     // fused append: row taken from k_new / v_new (and stored) by this item, else -1
+  bool lazy;
+};
+
+__device__ __forceinline__ int ring_slot_of(int p, int S, int R) { return p < S ? p : S + (p - S) % R; }
+
+// Shared-memory footprint of the work list (bytes) for `entries` (layer, b) pairs.
+__host__ __device__ inline int worklist_smem_bytes(int entries, int batch) {
+  return ((entries + 1 + batch) * 4 + 128 + 15) / 16 * 16;
+}
+
+struct WorkList {
+  int* prefix;    // [entries + 1]
+  int* seq;       // [batch]   seq_lens as read at kernel start
+  uint8_t* kind;  // [layer_count]  bit 0 lazy, bit 1 table entry missing
+  int entries;
+
+  __device__ __forceinline__ void carve(uint8_t* mem, int layer_count, int batch) {
+    entries = layer_count * batch;
+    prefix = reinterpret_cast<int*>(mem);
+    seq = prefix + entries + 1;
+    kind = reinterpret_cast<uint8_t*>(seq + batch);
+  }
+
+  // visible keys of (layer kind, batch row) after clamping; raises the error bits
+  __device__ __forceinline__ int visible(const DecodeArgs& a, int lr, int b, bool report) const {
+    const lt_shape& s = a.s;
+    const bool lazy = kind[lr] & 1;
+    const int rows = lazy ? s.n_sink + s.n_recent : s.full_capacity;
+    int n = seq[b] + (a.fused ? 1 : 0);
+    if (n < 0) n = 0;
+    if (n > rows) {
+      if (!lazy && report) atomicOr(a.dev_err, a.fused ? LT_DEVERR_POS_OUT_OF_RANGE : LT_DEVERR_LEN_CLAMPED);
+      n = rows;
+    }
+    return n;
+  }
+
+  // Called by every thread of the CTA.  Ends with a barrier.
+  __device__ void build(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
+                        const LayerTable& vs) {
+    const lt_shape& s = a.s;
+    const int B = s.batch;
+    for (int b = threadIdx.x; b < B; b += blockDim.x) seq[b] = a.seq_lens[b];
+    for (int lr = threadIdx.x; lr < a.layer_count; lr += blockDim.x) {
+      const int l = a.layer_begin + lr;
+      const bool lazy = a.mask[l] != 0;
+      const bool missing = lazy ? (!ks.p[l] || !vs.p[l]) : (!kf.p[l] || !vf.p[l]);
+      kind[lr] = (lazy ? 1 : 0) | (missing ? 2 : 0);
+      if (missing && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_NULL_LAYER);
+    }
+    __syncthreads();
+    // items per entry, then an exclusive scan: thread t owns a contiguous run of entries
+    const int per = (entries + blockDim.x - 1) / blockDim.x;
+    const int e0 = min(entries, (int)threadIdx.x * per), e1 = min(entries, e0 + per);
+    int run = 0;
+    for (int e = e0; e < e1; ++e) {
+      const int lr = e / B, b = e - lr * B;
+      int items = 0;
+      if (!(kind[lr] & 2)) {
+        const int n = visible(a, lr, b, blockIdx.x == 0);
+        const int nc = max(1, (n + a.chunk_keys - 1) / a.chunk_keys);
+        items = s.n_kv_heads * nc;
+      }
+      prefix[e + 1] = items;  // turned into the prefix below
+      run += items;
+    }
+    __shared__ int thread_sum[256];  // blockDim.x <= 256
+    thread_sum[threadIdx.x] = run;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int acc = 0;
+      for (int t = 0; t < (int)blockDim.x; ++t) {
+        const int v = thread_sum[t];
+        thread_sum[t] = acc;
+        acc += v;
+      }
+      prefix[0] = 0;
+    }
+    __syncthreads();
+    int acc = thread_sum[threadIdx.x];
+    for (int e = e0; e < e1; ++e) {
+      acc += prefix[e + 1];
+      prefix[e + 1] = acc;
+    }
+    __syncthreads();
+  }
+
+  __device__ __forceinline__ int total() const { return prefix[entries]; }
+
+  __device__ __forceinline__ WorkItem item(const DecodeArgs& a, int idx) const {
+    const lt_shape& s = a.s;
+    int lo = 0, hi = entries;  // largest e with prefix[e] <= idx
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (prefix[mid] <= idx) lo = mid;
+      else hi = mid;
+    }
+    WorkItem w;
+    const int lr = lo / s.batch;
+    w.b = lo - lr * s.batch;
+    w.l = a.layer_begin + lr;
+    w.lazy = kind[lr] & 1;
+    w.rows = w.lazy ? s.n_sink + s.n_recent : s.full_capacity;
+    w.n = visible(a, lr, w.b, false);
+    w.nc = max(1, (w.n + a.chunk_keys - 1) / a.chunk_keys);
+    const int rem = idx - prefix[lo];
+    w.h = rem / w.nc;
+    w.c = rem - w.h * w.nc;
+    const int len = (w.n + w.nc - 1) / w.nc;  // balanced chunks: no tiny last chunk
+    w.j0 = min(w.n, w.c * len);
+    w.j1 = min(w.n, w.j0 + len);
+    w.new_row = -1;
+    if (a.fused) {
+      const int pos = seq[w.b];
+      const int slot = w.lazy ? ring_slot_of(pos, s.n_sink, s.n_recent) : pos;
+      if (pos >= 0 && slot < w.rows && slot >= w.j0 && slot < w.j1) w.new_row = slot;
+    }
+    return w;
+  }
+};
+
+// Index of the partials of (layer, b, kv head, chunk).
+__device__ __forceinline__ long long partial_unit(const DecodeArgs& a, const WorkItem& w) {
+  return ((((long long)w.l * a.s.batch + w.b) * a.s.n_kv_heads + w.h) * a.n_chunks_max) + w.c;
+}
+
+// Staging buffer (shared memory) for the (max, sum) pairs of a unit's chunks
+// while they are merged; units with more pairs read them from global memory.
+constexpr int kCombineStagePairs = 512;
+
+// After a CTA has written the partials of its item (one thread's fence after a
+// CTA barrier publishes them all): count the item in; true for every thread of
+// the CTA that finished the last chunk of its (layer, b, kv head).  Two CTA
+// barriers.  A unit with a single chunk needs no count.
+__device__ __forceinline__ bool count_item_in(const DecodeArgs& a, const WorkItem& w, int* s_flag) {
+  if (w.nc <= 1) {
+    __syncthreads();
+    return true;
+  }
+  const long long unit = ((long long)w.l * a.s.batch + w.b) * a.s.n_kv_heads + w.h;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();  // cumulative: the partials written before the barrier are visible device-wide
+    const int prev = atomicAdd(a.unit_counters + unit, 1);
+    const int last = prev == w.nc - 1;
+    if (last) {
+      a.unit_counters[unit] = 0;  // ready for the next launch
+      __threadfence();            // acquire side: the other chunks' partials are visible to this CTA
+    }
+    *s_flag = last;
+  }
+  __syncthreads();
+  return *s_flag != 0;
+}
+
+// Merge the chunk partials of w's (layer, b, kv head) in chunk order (fixed
+// order => run-to-run identical bits) and write the outputs of the group's
+// query heads.  Called by every thread of the CTA; one thread owns four
+// consecutive d of one head and keeps eight chunk loads in flight.
+__device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem& w, float2* s_ml) {
+  const lt_shape& s = a.s;
+  const int G = s.n_q_heads / s.n_kv_heads, D = s.head_dim;
+  const long long unit = ((long long)w.l * s.batch + w.b) * s.n_kv_heads + w.h;
+  const long long unit0 = unit * a.n_chunks_max;
+  const int pairs = w.nc * G;
+  const bool staged = pairs <= kCombineStagePairs;
+  const float2* ml_g = reinterpret_cast<const float2*>(a.part_ml) + unit0 * G;  // [c][g]
+  if (staged) {
+    for (int i = threadIdx.x; i < pairs; i += blockDim.x) s_ml[i] = __ldcg(ml_g + i);
+  }
+  __syncthreads();
+  const int dq = D / 4;
+  for (int idx = threadIdx.x; idx < G * dq; idx += blockDim.x) {
+    const int g = idx / dq, d = (idx - g * dq) * 4;
+    float M = -INFINITY;
+    for (int c = 0; c < w.nc; ++c) M = fmaxf(M, staged ? s_ml[c * G + g].x : __ldcg(ml_g + c * G + g).x);
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    if (M > -INFINITY) {
+      const float4* po = reinterpret_cast<const float4*>(a.part_o + (unit0 * G + g) * D + d);
+      const long long cstride = (long long)G * D / 4;  // float4s between chunks
+      for (int c0 = 0; c0 < w.nc; c0 += 8) {
+        float4 ov[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (c0 + i < w.nc) ov[i] = __ldcg(po + (c0 + i) * cstride);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (c0 + i < w.nc) {
+            const float2 ml = staged ? s_ml[(c0 + i) * G + g] : __ldcg(ml_g + (c0 + i) * G + g);
+            const float wgt = exp2f(ml.x - M);
+            den += wgt * ml.y;
+            num.x += wgt * ov[i].x;
+            num.y += wgt * ov[i].y;
+            num.z += wgt * ov[i].z;
+            num.w += wgt * ov[i].w;
+          }
+        }
+      }
+    }
+    const float r0 = den > 0.f ? num.x / den : 0.f, r1 = den > 0.f ? num.y / den : 0.f;
+    const float r2 = den > 0.f ? num.z / den : 0.f, r3 = den > 0.f ? num.w / den : 0.f;
+    const long long oi = (((long long)w.l * s.batch + w.b) * s.n_q_heads + w.h * G + g) * D + d;
+    if (a.out_dtype == LT_F32) {
+      *reinterpret_cast<float4*>((float*)a.out + oi) = make_float4(r0, r1, r2, r3);
+    } else {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>((__nv_bfloat16*)a.out + oi) = pk;
+    }
+  }
+}
+
+// End of a persistent launch: the last CTA to finish re-arms the launch's
+// counters and, for a fused step that advances, increments seq_lens (every CTA
+// has read them by then).  Called by every thread.
+__device__ __forceinline__ void finish_launch(const DecodeArgs& a) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const int prev = atomicAdd(a.done_counter, 1);
+    if (prev == (int)gridDim.x - 1) {
+      *a.done_counter = 0;
+      *a.work_counter = 0;
+      if (a.fused && a.advance)
+        for (int b = 0; b < a.s.batch; ++b) a.seq_lens_rw[b] += 1;
+    }
+  }
+}
+
+}  // namespace lt

@@ -1,11 +1,23 @@
-// Decode attention, bandwidth path: bf16, head_dim 128, GQA group <= 8.
+// Decode step, bandwidth path: bf16, head_dim 128, GQA group <= 8.
 //
-// One CTA per (layer, batch row, kv head, KV chunk) serves every query head of
-// the group, so each cached K and V byte is read from HBM exactly once per step.
-// Each warp streams its own tiles of the chunk through a private multi-stage
-// cp.async ring in shared memory (16-byte vectors, fully coalesced rows, XOR
-// swizzle of the 16-byte column so that ldmatrix is conflict-free) and needs no
-// CTA-wide barrier until the final merge.
+// A persistent launch (two CTAs per SM) walks the flattened work list of
+// (layer, batch row, kv head, KV chunk) items; items are handed out through a
+// device counter so that faster SMs take more of them.  One item serves every
+// query head of the group, so each cached K and V byte is read from HBM exactly
+// once per step.
+//
+// Each warp streams its own 16-key tiles of the chunk through a private
+// multi-stage cp.async ring in shared memory (16-byte vectors, fully coalesced
+// rows, XOR swizzle of the 16-byte column so that ldmatrix is conflict-free).
+// The ring never drains between items: while a warp finishes the tiles of one
+// item its look-ahead already fetches the first tiles of the CTA's next item,
+// so the merge of the four warps, the hand-off of the partials and the merge of
+// a finished (layer, b, kv head) all happen with loads in flight.
+//
+// Fused append: the item that owns the new token's row takes that row from
+// k_new / v_new and stores it into the cache.  The last item of a (layer, batch
+// row, kv head) to finish merges the chunk partials and writes the output, so a
+// whole decode step is one launch.
 //
 // Tensor-core mapping (mma.sync m16n8k16, bf16 in, fp32 accumulate):
 //   S^T[key][head]  = K[key][d] . Q^T[d][head]      keys are M (16), heads are N (8)
@@ -16,6 +28,7 @@
 // bf16 residual (two MMAs) so that the probabilities keep ~16 bits.
 #include <cuda_bf16.h>
 
+#include "lt_decode_common.cuh"
 #include "lt_internal.h"
 
 namespace lt {
@@ -67,229 +80,387 @@ constexpr int kRowBytes = kD * 2;  // one K or V row
 
 }  // namespace
 
-// Shared memory of one warp and one stage: K half-tiles [2][TILE][128 B] then V
-// half-tiles [2][TILE][128 B]; inside a half-tile the 16-byte column c of row r
-// sits at column c ^ (r & 7).
+// What a warp needs to fetch tiles of one item.
+struct TileSrc {
+  const uint8_t* Kb;         // rows of this (b, kv head) in the cache that is read
+  const uint8_t* Vb;
+  const uint8_t* k_new_row;  // fused append: source of row new_row
+  const uint8_t* v_new_row;
+  int j0, j1;                // key rows of the chunk
+  int new_row;               // -1 when the chunk does not hold the new token
+  int my_tiles;              // tiles of this warp (tiles warp, warp + WARPS, ... of the chunk)
+};
+
+// Shared memory: [rings: WARPS x NSTAGE x stage][merge: two 8 x 128 fp32 buffers,
+// (max, sum) of every warp][work list].  A stage holds K half-tiles
+// [2][TILE][128 B] then V half-tiles [2][TILE][128 B]; inside a half-tile the
+// 16-byte column c of row r sits at column c ^ (r & 7).
 template <int TILE, int NSTAGE, int WARPS, int MINB>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
+  static_assert(WARPS == 4, "the merge tree below is written for four warps");
   constexpr int MT = TILE / 16;                // 16-key MMA tiles per pipeline tile
   constexpr int HALF_BYTES = TILE * 128;       // one half-tile
   constexpr int STAGE_BYTES = 4 * HALF_BYTES;  // K halves + V halves
+  constexpr int RING_BYTES = WARPS * NSTAGE * STAGE_BYTES;
+  constexpr int MERGE_BYTES = 2 * 8 * kD * 4 + 2 * WARPS * 8 * 4;
   extern __shared__ __align__(1024) uint8_t smem[];
+  __shared__ int s_flag, s_next;
 
   const lt_shape& s = a.s;
-  const int l = a.layer_begin + blockIdx.z;
-  const int bh = blockIdx.y;
-  const int b = bh / s.n_kv_heads, h = bh - b * s.n_kv_heads;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const bool lazy = a.mask[l] != 0;
-  const uint8_t* K = (const uint8_t*)(lazy ? ks.p[l] : kf.p[l]);
-  const uint8_t* V = (const uint8_t*)(lazy ? vs.p[l] : vf.p[l]);
-  const int rows = lazy ? s.n_sink + s.n_recent : s.full_capacity;
-  int n = a.seq_lens[b];
-  if (!K || !V) {
-    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_NULL_LAYER);
-    return;
-  }
-  if (n > rows) {
-    if (!lazy && threadIdx.x == 0 && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_LEN_CLAMPED);
-    n = rows;
-  }
-  if (n > a.n_chunks_launch * a.chunk_keys) {
-    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_LEN_CLAMPED);
-    n = a.n_chunks_launch * a.chunk_keys;
-  }
-  const int j0 = blockIdx.x * a.chunk_keys;
-  const int j1 = min(n, j0 + a.chunk_keys);
-  if (j0 >= j1) return;
+  float* sm_buf = reinterpret_cast<float*>(smem + RING_BYTES);  // [2][8][128]
+  float* sm_m = sm_buf + 2 * 8 * kD;                            // [WARPS][8]
+  float* sm_l = sm_m + WARPS * 8;                               // [WARPS][8]
+  WorkList wl;
+  wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
+  wl.build(a, kf, vf, ks, vs);
+  const int n_items = wl.total();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
-  const uint8_t* Kb = K + (long long)bh * rows * kRowBytes;
-  const uint8_t* Vb = V + (long long)bh * rows * kRowBytes;
   const uint32_t wsm = smem_u32(smem) + warp * (NSTAGE * STAGE_BYTES);
-
-  // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
-  uint32_t qf[8][2];
-  {
-    const __nv_bfloat16* qp =
-        (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + gp) * kD;
-#pragma unroll
-    for (int ks8 = 0; ks8 < 8; ++ks8) {
-      if (gp < G) {
-        qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
-        qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
-      } else {
-        qf[ks8][0] = 0u;
-        qf[ks8][1] = 0u;
-      }
-    }
-  }
-
-  const int n_tiles = (j1 - j0 + TILE - 1) / TILE;  // tiles of this chunk
-  // warp w owns tiles w, w + WARPS, ...
-  auto issue_tile = [&](int my_idx) {
-    const int t = warp + my_idx * WARPS;
-    if (t < n_tiles) {
-      const int key_base = j0 + t * TILE;
-      const uint32_t st = wsm + (my_idx % NSTAGE) * STAGE_BYTES;
-#pragma unroll
-      for (int i = 0; i < TILE / 2; ++i) {
-        const int r = 2 * i + (lane >> 4);
-        const int p = lane & 15;
-        const int row = key_base + r;
-        const bool valid = row < j1;
-        const long long goff = (long long)(valid ? row : (j1 - 1)) * kRowBytes + p * 16;
-        const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
-        cp_async16(st + soff, Kb + goff, valid ? 16 : 0);
-        cp_async16(st + 2 * HALF_BYTES + soff, Vb + goff, valid ? 16 : 0);
-      }
-    }
-    cp_async_commit();
-  };
-
-  float o[8][4];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
-  float M0 = -INFINITY, M1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2c and 2c+1
-
-  const int my_tiles = (n_tiles > warp) ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
-#pragma unroll
-  for (int i = 0; i < NSTAGE - 1; ++i) issue_tile(i);
-
   // lane-constant parts of the ldmatrix addresses
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8;  // K (A operand, not transposed)
   const int k_chk = lane >> 4;
   const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8;  // V (A operand, transposed)
   const int v_chk = (lane >> 3) & 1;
 
-  for (int it = 0; it < my_tiles; ++it) {
-    __syncwarp();              // every lane is done reading the stage that is refilled next
-    issue_tile(it + NSTAGE - 1);
-    cp_async_wait<NSTAGE - 1>();
-    __syncwarp();              // all lanes' copies of tile `it` have landed
-    const uint32_t st = wsm + (it % NSTAGE) * STAGE_BYTES;
-    const int key_base = j0 + (warp + it * WARPS) * TILE;
-
-    // ---- S^T = K Q^T ------------------------------------------------------
-    float sc[MT][4];
+  auto make_src = [&](const WorkItem& w) {
+    TileSrc t;
+    const long long bh = (long long)w.b * s.n_kv_heads + w.h;
+    t.Kb = (const uint8_t*)(w.lazy ? ks.p[w.l] : kf.p[w.l]) + bh * w.rows * kRowBytes;
+    t.Vb = (const uint8_t*)(w.lazy ? vs.p[w.l] : vf.p[w.l]) + bh * w.rows * kRowBytes;
+    t.j0 = w.j0;
+    t.j1 = w.j1;
+    t.new_row = w.new_row;
+    t.k_new_row = nullptr;
+    t.v_new_row = nullptr;
+    if (w.new_row >= 0) {
+      const long long src = (((long long)w.l * s.batch + w.b) * s.n_kv_heads + w.h) * kRowBytes;
+      t.k_new_row = (const uint8_t*)a.k_new + src;
+      t.v_new_row = (const uint8_t*)a.v_new + src;
+    }
+    const int n_tiles = (w.j1 - w.j0 + TILE - 1) / TILE;
+    t.my_tiles = (n_tiles > warp) ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
+    return t;
+  };
+  // copy this warp's idx-th tile of `t` into ring stage `stage` (no commit)
+  auto fetch_tile = [&](const TileSrc& t, int idx, int stage) {
+    const int key_base = t.j0 + (warp + idx * WARPS) * TILE;
+    const uint32_t st = wsm + stage * STAGE_BYTES;
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      sc[mt][0] = sc[mt][1] = sc[mt][2] = sc[mt][3] = 0.f;
-      const int row = mt * 16 + k_row;
+    for (int i = 0; i < TILE / 2; ++i) {
+      const int r = 2 * i + (lane >> 4);
+      const int p = lane & 15;
+      const int row = key_base + r;
+      const bool valid = row < t.j1;
+      const long long goff = (long long)(valid ? row : (t.j1 - 1)) * kRowBytes + p * 16;
+      const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
+      const bool fresh = row == t.new_row;
+      cp_async16(st + soff, fresh ? t.k_new_row + p * 16 : t.Kb + goff, valid ? 16 : 0);
+      cp_async16(st + 2 * HALF_BYTES + soff, fresh ? t.v_new_row + p * 16 : t.Vb + goff, valid ? 16 : 0);
+    }
+  };
+
+  // The CTA's first two items are fixed; later ones come from the device counter.
+  int cur = blockIdx.x, nxt = blockIdx.x + gridDim.x;
+  WorkItem w;
+  TileSrc src_cur, src_nxt;
+  src_cur.my_tiles = 0;
+  src_nxt.my_tiles = 0;
+  if (cur < n_items) {
+    w = wl.item(a, cur);
+    src_cur = make_src(w);
+  }
+  if (nxt < n_items) src_nxt = make_src(wl.item(a, nxt));
+
+  // Every cp.async group is one "slot" of the warp's tile stream (a tile, or
+  // nothing once the stream has run dry); slot k lives in ring stage k % NSTAGE.
+  uint32_t issued = 0, consumed = 0;
+  int la_in_next = 0;  // look-ahead cursor: 0 = in the current item, 1 = in the next one
+  int la_idx = 0;      // tile index of the cursor inside that item
+  int skip_after = 0;  // empty slots that follow the current item's tiles
+  auto issue_slot = [&]() {
+    if (la_in_next == 0 && la_idx >= src_cur.my_tiles) {
+      la_in_next = 1;
+      la_idx = 0;
+    }
+    const int stage = issued % NSTAGE;
+    if (la_in_next == 0) fetch_tile(src_cur, la_idx, stage);
+    else if (la_idx < src_nxt.my_tiles) fetch_tile(src_nxt, la_idx, stage);
+    ++la_idx;
+    ++issued;
+    cp_async_commit();
+  };
+
+  while (cur < n_items) {
+    const int l = w.l, b = w.b, h = w.h;
+    const int j1 = src_cur.j1;
+    int fetched_next = 0;
+    if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
+
+    // fused append: store the new token's row into the cache
+    if (src_cur.new_row >= 0 && warp == 0) {
+      const uint8_t* sp = (lane < 16 ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 15) * 16;
+      uint8_t* dp = const_cast<uint8_t*>(lane < 16 ? src_cur.Kb : src_cur.Vb) +
+                    (long long)src_cur.new_row * kRowBytes + (lane & 15) * 16;
+      *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
+    }
+
+    // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
+    uint32_t qf[8][2];
+    {
+      const __nv_bfloat16* qp =
+          (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + gp) * kD;
 #pragma unroll
       for (int ks8 = 0; ks8 < 8; ++ks8) {
-        uint32_t af[4];
-        const int chunk = 2 * (ks8 & 3) + k_chk;
-        ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-        mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+        if (gp < G) {
+          qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
+          qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
+        } else {
+          qf[ks8][0] = 0u;
+          qf[ks8][1] = 0u;
+        }
       }
     }
-    // ---- scale, mask the ragged tail, tile max per head ---------------------
-    float mx0 = -INFINITY, mx1 = -INFINITY;
+
+    float o[8][4];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      const int key_lo = key_base + mt * 16 + gp;
-      const bool v_lo = key_lo < j1, v_hi = key_lo + 8 < j1;
-      sc[mt][0] = v_lo ? sc[mt][0] * a.cs : -INFINITY;
-      sc[mt][1] = v_lo ? sc[mt][1] * a.cs : -INFINITY;
-      sc[mt][2] = v_hi ? sc[mt][2] * a.cs : -INFINITY;
-      sc[mt][3] = v_hi ? sc[mt][3] * a.cs : -INFINITY;
-      mx0 = fmaxf(mx0, fmaxf(sc[mt][0], sc[mt][2]));
-      mx1 = fmaxf(mx1, fmaxf(sc[mt][1], sc[mt][3]));
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
+    float M0 = -INFINITY, M1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2c and 2c+1
+
+    while (issued - consumed < NSTAGE - 1) issue_slot();
+    for (int it = 0; it < src_cur.my_tiles; ++it) {
+      __syncwarp();              // every lane is done reading the stage that is refilled next
+      issue_slot();
+      cp_async_wait<NSTAGE - 1>();
+      __syncwarp();              // all lanes' copies of this tile have landed
+      const uint32_t st = wsm + (consumed % NSTAGE) * STAGE_BYTES;
+      ++consumed;
+      const int key_base = src_cur.j0 + (warp + it * WARPS) * TILE;
+
+      // ---- S^T = K Q^T ------------------------------------------------------
+      float sc[MT][4];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        sc[mt][0] = sc[mt][1] = sc[mt][2] = sc[mt][3] = 0.f;
+        const int row = mt * 16 + k_row;
+#pragma unroll
+        for (int ks8 = 0; ks8 < 8; ++ks8) {
+          uint32_t af[4];
+          const int chunk = 2 * (ks8 & 3) + k_chk;
+          ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
+          mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+        }
+      }
+      // ---- scale, mask the ragged tail, tile max per head ---------------------
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const int key_lo = key_base + mt * 16 + gp;
+        const bool v_lo = key_lo < j1, v_hi = key_lo + 8 < j1;
+        sc[mt][0] = v_lo ? sc[mt][0] * a.cs : -INFINITY;
+        sc[mt][1] = v_lo ? sc[mt][1] * a.cs : -INFINITY;
+        sc[mt][2] = v_hi ? sc[mt][2] * a.cs : -INFINITY;
+        sc[mt][3] = v_hi ? sc[mt][3] * a.cs : -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(sc[mt][0], sc[mt][2]));
+        mx1 = fmaxf(mx1, fmaxf(sc[mt][1], sc[mt][3]));
+      }
+#pragma unroll
+      for (int off = 4; off < 32; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+      }
+      const float Mn0 = fmaxf(M0, mx0), Mn1 = fmaxf(M1, mx1);
+      const float corr0 = exp2f(M0 - Mn0), corr1 = exp2f(M1 - Mn1);
+      M0 = Mn0;
+      M1 = Mn1;
+      l0 *= corr0;
+      l1 *= corr1;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        o[i][0] *= corr0;
+        o[i][1] *= corr1;
+        o[i][2] *= corr0;
+        o[i][3] *= corr1;
+      }
+      // ---- P = 2^(t - M), O^T += V^T P ---------------------------------------
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const float p0 = exp2f(sc[mt][0] - Mn0), p1 = exp2f(sc[mt][1] - Mn1);
+        const float p2 = exp2f(sc[mt][2] - Mn0), p3 = exp2f(sc[mt][3] - Mn1);
+        l0 += p0 + p2;
+        l1 += p1 + p3;
+        const uint32_t hi01 = pack_bf16(p0, p1), hi23 = pack_bf16(p2, p3);
+        const uint32_t lo01 = pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01));
+        const uint32_t lo23 = pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23));
+        const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
+        const uint32_t bl0 = movmatrix_trans(lo01), bl1 = movmatrix_trans(lo23);
+        const int row = mt * 16 + v_row;
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+          uint32_t af[4];
+          const int chunk = 2 * (dt & 3) + v_chk;
+          ldmatrix_x4_trans(af,
+                            st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
+          mma_bf16(o[dt], af, bh0, bh1);
+          mma_bf16(o[dt], af, bl0, bl1);
+        }
+      }
     }
+    // Slots that were issued for this item past its last tile are empty groups:
+    // step over them.  The slots after those are the next item's first tiles,
+    // already in flight.
+    consumed += skip_after;
+
+    // ---- merge the four warps: (w0 + w2) + (w1 + w3), fixed order ---------------
 #pragma unroll
     for (int off = 4; off < 32; off <<= 1) {
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
     }
-    const float Mn0 = fmaxf(M0, mx0), Mn1 = fmaxf(M1, mx1);
-    const float corr0 = exp2f(M0 - Mn0), corr1 = exp2f(M1 - Mn1);
-    M0 = Mn0;
-    M1 = Mn1;
-    l0 *= corr0;
-    l1 *= corr1;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      o[i][0] *= corr0;
-      o[i][1] *= corr1;
-      o[i][2] *= corr0;
-      o[i][3] *= corr1;
+    if (gp == 0) {
+      sm_m[warp * 8 + 2 * c] = M0;
+      sm_m[warp * 8 + 2 * c + 1] = M1;
+      sm_l[warp * 8 + 2 * c] = l0;
+      sm_l[warp * 8 + 2 * c + 1] = l1;
     }
-    // ---- P = 2^(t - M), O^T += V^T P ---------------------------------------
+    if (threadIdx.x == 0) s_next = fetched_next;
+    __syncthreads();  // (max, sum) of every warp and the next item index are visible
+    const int after_next = s_next;
+    float Mx0 = -INFINITY, Mx1 = -INFINITY;
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      const float p0 = exp2f(sc[mt][0] - Mn0), p1 = exp2f(sc[mt][1] - Mn1);
-      const float p2 = exp2f(sc[mt][2] - Mn0), p3 = exp2f(sc[mt][3] - Mn1);
-      l0 += p0 + p2;
-      l1 += p1 + p3;
-      const uint32_t hi01 = pack_bf16(p0, p1), hi23 = pack_bf16(p2, p3);
-      const uint32_t lo01 = pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01));
-      const uint32_t lo23 = pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23));
-      const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
-      const uint32_t bl0 = movmatrix_trans(lo01), bl1 = movmatrix_trans(lo23);
-      const int row = mt * 16 + v_row;
+    for (int ww = 0; ww < WARPS; ++ww) {
+      Mx0 = fmaxf(Mx0, sm_m[ww * 8 + 2 * c]);
+      Mx1 = fmaxf(Mx1, sm_m[ww * 8 + 2 * c + 1]);
+    }
+    float ls0 = 0.f, ls1 = 0.f;
+    if (Mx0 > -INFINITY)
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
-        uint32_t af[4];
-        const int chunk = 2 * (dt & 3) + v_chk;
-        ldmatrix_x4_trans(af, st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-        mma_bf16(o[dt], af, bh0, bh1);
-        mma_bf16(o[dt], af, bl0, bl1);
+      for (int ww = 0; ww < WARPS; ++ww) ls0 += exp2f(sm_m[ww * 8 + 2 * c] - Mx0) * sm_l[ww * 8 + 2 * c];
+    if (Mx1 > -INFINITY)
+#pragma unroll
+      for (int ww = 0; ww < WARPS; ++ww) ls1 += exp2f(sm_m[ww * 8 + 2 * c + 1] - Mx1) * sm_l[ww * 8 + 2 * c + 1];
+    {
+      const float f0 = Mx0 > -INFINITY ? exp2f(M0 - Mx0) : 0.f;
+      const float f1 = Mx1 > -INFINITY ? exp2f(M1 - Mx1) : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        o[i][0] *= f0;
+        o[i][1] *= f1;
+        o[i][2] *= f0;
+        o[i][3] *= f1;
       }
     }
+    // element (head 2c + e, d = dt*16 + gp + 8*half) of a warp's O at buffer offset below
+    auto buf_at = [&](int which, int dt) { return sm_buf + which * (8 * kD) + (2 * c) * kD + dt * 16 + gp; };
+    if (warp >= 2) {
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        float* p = buf_at(warp - 2, dt);
+        p[0] = o[dt][0];
+        p[kD] = o[dt][1];
+        p[8] = o[dt][2];
+        p[kD + 8] = o[dt][3];
+      }
+    }
+    __syncthreads();
+    if (warp < 2) {
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        const float* p = buf_at(warp, dt);
+        o[dt][0] += p[0];
+        o[dt][1] += p[kD];
+        o[dt][2] += p[8];
+        o[dt][3] += p[kD + 8];
+      }
+    }
+    __syncthreads();  // buffer 0 has been read by warp 0 before warp 1 overwrites it
+    if (warp == 1) {
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        float* p = buf_at(0, dt);
+        p[0] = o[dt][0];
+        p[kD] = o[dt][1];
+        p[8] = o[dt][2];
+        p[kD + 8] = o[dt][3];
+      }
+    }
+    __syncthreads();
+    const bool single = w.nc <= 1;  // the whole (layer, b, kv head) is this one chunk
+    if (warp == 0) {
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        const float* p = buf_at(0, dt);
+        o[dt][0] += p[0];
+        o[dt][1] += p[kD];
+        o[dt][2] += p[8];
+        o[dt][3] += p[kD + 8];
+      }
+      if (single) {
+        // no partials: normalise and write the output of heads 2c, 2c + 1 directly
+        const long long ob = (((long long)l * s.batch + b) * s.n_q_heads + h * G) * kD;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int g = 2 * c + e;
+          if (g < G) {
+            const float den = e ? ls1 : ls0;
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                const float num = o[dt][e + 2 * half];
+                const float r = den > 0.f ? num / den : 0.f;
+                const long long oi = ob + (long long)g * kD + dt * 16 + gp + 8 * half;
+                if (a.out_dtype == LT_F32) ((float*)a.out)[oi] = r;
+                else ((__nv_bfloat16*)a.out)[oi] = __float2bfloat16_rn(r);
+              }
+            }
+          }
+        }
+      } else {
+        const long long unit = partial_unit(a, w);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int g = 2 * c + e;
+          if (g < G) {
+            float* po = a.part_o + (unit * G + g) * kD + gp;
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+              po[dt * 16] = o[dt][e];
+              po[dt * 16 + 8] = o[dt][e + 2];
+            }
+            if (gp == 0) {
+              a.part_ml[(unit * G + g) * 2] = e ? Mx1 : Mx0;
+              a.part_ml[(unit * G + g) * 2 + 1] = e ? ls1 : ls0;
+            }
+          }
+        }
+      }
+    }
+    if (!single) {
+      if (count_item_in(a, w, &s_flag)) combine_unit(a, w, reinterpret_cast<float2*>(sm_buf));
+    }
+    __syncthreads();  // merge buffers and flags are free for the next item
+
+    // ---- move on: the next item becomes current ----------------------------------
+    cur = nxt;
+    nxt = after_next;
+    const int pre = la_in_next ? la_idx : 0;  // slots already issued on behalf of the new current item
+    src_cur = src_nxt;
+    la_in_next = 0;
+    la_idx = pre;
+    skip_after = max(0, pre - src_cur.my_tiles);
+    if (cur < n_items) w = wl.item(a, cur);
+    src_nxt.my_tiles = 0;
+    if (nxt < n_items) src_nxt = make_src(wl.item(a, nxt));
   }
   cp_async_wait<0>();
-
-  // ---- warp totals, then merge the warps of the CTA through shared memory ----
-#pragma unroll
-  for (int off = 4; off < 32; off <<= 1) {
-    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-  }
-  __syncthreads();  // every warp has drained its ring: the memory can be reused
-  float* sm_m = reinterpret_cast<float*>(smem);  // [WARPS][8]
-  float* sm_l = sm_m + WARPS * 8;                // [WARPS][8]
-  float* sm_o = sm_l + WARPS * 8;                // [WARPS][8][128]
-  if (gp == 0) {
-    sm_m[warp * 8 + 2 * c] = M0;
-    sm_m[warp * 8 + 2 * c + 1] = M1;
-    sm_l[warp * 8 + 2 * c] = l0;
-    sm_l[warp * 8 + 2 * c + 1] = l1;
-  }
-#pragma unroll
-  for (int dt = 0; dt < 8; ++dt) {
-    float* base = sm_o + (warp * 8 + 2 * c) * kD + dt * 16 + gp;
-    base[0] = o[dt][0];
-    base[kD] = o[dt][1];
-    base[8] = o[dt][2];
-    base[kD + 8] = o[dt][3];
-  }
-  __syncthreads();
-  const long long unit = (((long long)l * s.batch + b) * s.n_kv_heads + h) * a.n_chunks_max + blockIdx.x;
-  for (int idx = threadIdx.x; idx < G * kD; idx += WARPS * 32) {
-    const int g = idx / kD, d = idx - g * kD;
-    float Mx = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < WARPS; ++w) Mx = fmaxf(Mx, sm_m[w * 8 + g]);
-    float acc = 0.f, lsum = 0.f;
-#pragma unroll
-    for (int w = 0; w < WARPS; ++w) {
-      const float wgt = exp2f(sm_m[w * 8 + g] - Mx);
-      acc += wgt * sm_o[(w * 8 + g) * kD + d];
-      lsum += wgt * sm_l[w * 8 + g];
-    }
-    a.part_o[(unit * G + g) * kD + d] = acc;
-    if (d == 0) {
-      a.part_ml[(unit * G + g) * 2] = Mx;
-      a.part_ml[(unit * G + g) * 2 + 1] = lsum;
-    }
-  }
+  finish_launch(a);
 }
-
 bool decode_mma_supported(const lt_shape& s) {
   return s.dtype == LT_BF16 && s.head_dim == 128 && (s.n_q_heads / s.n_kv_heads) <= 8;
 }
@@ -297,12 +468,18 @@ bool decode_mma_supported(const lt_shape& s) {
 template <int TILE, int NSTAGE, int WARPS, int MINB>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int smem = WARPS * NSTAGE * TILE * 512;
-  static_assert(smem >= WARPS * (16 + 8 * 128) * 4, "merge buffer must fit in the pipeline memory");
+  constexpr int ring = WARPS * NSTAGE * TILE * 512;
+  constexpr int merge = 2 * 8 * 128 * 4 + 2 * WARPS * 8 * 4;
+  static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
+  const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
   auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(a.n_chunks_launch, a.s.batch * a.s.n_kv_heads, a.layer_count);
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, WARPS * 32, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  const int grid = persistent_grid(a, per_sm);
   kern<<<grid, WARPS * 32, smem, st>>>(a, kf, vf, ks, vs);
   return cudaGetLastError();
 }

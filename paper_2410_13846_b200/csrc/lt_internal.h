@@ -15,9 +15,13 @@ struct LayerTable {
   const void* p[LT_MAX_LAYERS];
 };
 
-// Workspace layout: [header 256 B][region used by the running call].
+// Workspace layout: [header 256 B: error word][counters of the decode step]
+// [region used by the running call: split-KV partials or scoring statistics].
 constexpr size_t kWsHeaderBytes = 256;
 constexpr size_t kWsAlign = 256;
+// Bytes of header + counters ([L][B][Hkv] unit counters, then the two launch
+// counters); everything here must be zero between calls (lt_workspace_init).
+size_t ws_prefix_bytes(const lt_shape& s);
 
 // Split-KV plan of the decode step; a function of the shape alone so that the
 // workspace query and every later call agree.
@@ -54,27 +58,42 @@ cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const Lay
                                const LayerTable& vf, const int32_t* seq_lens, const LayerTable& ks,
                                const LayerTable& vs, uint32_t* dev_err, cudaStream_t st);
 
+// One decode step (or the attention half of it).  `fused` = the step appends
+// k_new / v_new itself: the visible length is seq_lens[b] + 1 and the item that
+// owns the new token's row stores it into the cache.
 struct DecodeArgs {
   lt_shape s;
   const void* q;
+  const void* k_new;  // fused only
+  const void* v_new;  // fused only
   const uint8_t* mask;
   const int32_t* seq_lens;
+  int32_t* seq_lens_rw;  // fused + advance: incremented by the last CTA of the launch
   void* out;
   int out_dtype;
   int layer_begin, layer_count;
-  int chunk_keys, n_chunks_max, n_chunks_launch;
+  int chunk_keys, n_chunks_max;
+  int fused, advance;
   float cs;  // softmax scale * log2(e)
   float* part_ml;
   float* part_o;
+  int* unit_counters;  // [L][B][Hkv], zero between launches
+  int* done_counter;   // zero between launches
+  int* work_counter;   // zero between launches: dynamic item hand-out
   uint32_t* dev_err;
 };
+// Most (layer, batch row) pairs one launch can take (its work list lives in
+// shared memory); larger stacks are split by layers on the host.
+constexpr int kMaxWorkEntries = 2048;
+// CTAs of a persistent decode launch: per_sm * SM count, but no more than the
+// most items the launch can have.
+int persistent_grid(const DecodeArgs& a, int ctas_per_sm);
 cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 // bf16, head_dim 128, group size <= 8: tensor-core path.
 bool decode_mma_supported(const lt_shape& s);
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                               const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
-cudaError_t launch_decode_combine(const DecodeArgs& a, cudaStream_t st);
 
 struct ScoreArgs {
   lt_shape s;

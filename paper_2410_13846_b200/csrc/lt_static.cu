@@ -74,8 +74,8 @@ extern "C" lt_status lt_hybrid_decode_attn_static(const lt_shape* shape, const v
   void* scratch = nullptr;
   if (scratch_for_current_device(&scratch) != cudaSuccess) return LT_ERR_CUDA;
   cudaStream_t cs = (cudaStream_t)stream;
-  // The header holds the error word; start every call from zero.
-  if (cudaMemsetAsync(scratch, 0, kWsHeaderBytes, cs) != cudaSuccess) return LT_ERR_CUDA;
+  // The header holds the error word and the merge counters; start every call from zero.
+  if (cudaMemsetAsync(scratch, 0, ws_prefix_bytes(*shape), cs) != cudaSuccess) return LT_ERR_CUDA;
   st = lt_hybrid_decode_attn(shape, q, k_full, v_full, k_stream, v_stream, layer_mask, seq_lens, out, out_dtype,
                              max_seq_len_hint, layer_begin, layer_count, scratch, (size_t)LT_STATIC_SCRATCH_BYTES,
                              stream);
