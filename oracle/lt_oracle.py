@@ -14,7 +14,10 @@ the paper one step at a time, with no blocking, fusion or reordering:
   O2  streaming_attention   the same with the sink+recent mask M_lazy
                             (Appendix E, masked MHA; Section 5.1, retained KV)
   O3  lazy_scores           the lazy ratio of Eq. 1, per query head; a second
-                            route through the log-sum-exp identity of Table 1
+                            route through the log-sum-exp identity of Table 1;
+                            causal_lse / lazy_scores_from_lse: the form Section
+                            5.1 actually deploys - the prefill's log-sum-exp is
+                            given, only the window block is recomputed
   O4  select_lazy           keep the P lowest ratios full (Section 5.1, the
                             priority queue; Figure 3)
   O5  ring_slot / ring_owner / stream_cache_after / HybridReplay
@@ -47,6 +50,8 @@ __all__ = [
     "kept_positions",
     "lazy_scores",
     "lazy_scores_lse_route",
+    "causal_lse",
+    "lazy_scores_from_lse",
     "layer_ratios",
     "select_lazy",
     "select_lazy_priority_queue",
@@ -205,6 +210,51 @@ def lazy_scores_lse_route(Q_tail, K, n_sink: int, n_recent: int, scale=None):
             lse_all = _logsumexp(s)
             lse_win = _logsumexp(s[keep[: i + 1]])
             acc += math.exp(lse_win - lse_all) if np.isfinite(lse_win) else 0.0
+        score[hq] = acc / T
+    return score
+
+
+def causal_lse(Q_tail, K, scale=None):
+    """What the prefill's attention hands over for the tail rows (Table 1, the
+    `lse` returned next to `attn_out`): lse[hq, t] = log sum_{j <= i} exp(scale *
+    q_t . k_j), natural logarithm, i = n - T + t.  returns [Hq, T].
+    """
+    Q_tail, K = _f64(Q_tail), _f64(K)
+    Hq, T, D = Q_tail.shape
+    Hkv, n, _ = K.shape
+    G = Hq // Hkv
+    sc = _default_scale(D, scale)
+    out = np.zeros((Hq, T), dtype=np.float64)
+    for hq in range(Hq):
+        for t in range(T):
+            i = n - T + t
+            out[hq, t] = _logsumexp(sc * (K[hq // G, : i + 1] @ Q_tail[hq, t]))
+    return out
+
+
+def lazy_scores_from_lse(Q_tail, K, lse, n_sink: int, n_recent: int, scale=None):
+    """O3 as deployed (Section 5.1, "only need to recompute the streaming
+    attention score"; Table 1): the denominator of every tail row comes in as
+    its log-sum-exp, and only the logits of the kept keys {j < n_sink} U
+    {j >= n - n_recent} (causally visible ones) are computed:
+        mass_t = sum_{j kept, j <= i} exp(scale * q_t . k_j - lse[hq, t]),
+    averaged over the T tail rows.  K is the whole prompt [Hkv, n, D] only so
+    that positions can be indexed; rows outside the kept set are not touched.
+    """
+    Q_tail, K, lse = _f64(Q_tail), _f64(K), _f64(lse)
+    Hq, T, D = Q_tail.shape
+    Hkv, n, _ = K.shape
+    G = Hq // Hkv
+    sc = _default_scale(D, scale)
+    kept = np.nonzero(kept_positions(n, n_sink, n_recent))[0]
+    score = np.zeros(Hq, dtype=np.float64)
+    for hq in range(Hq):
+        acc = 0.0
+        for t in range(T):
+            i = n - T + t
+            js = kept[kept <= i]
+            logits = sc * (K[hq // G, js] @ Q_tail[hq, t])
+            acc += float(np.sum(np.exp(logits - lse[hq, t])))
         score[hq] = acc / T
     return score
 

@@ -37,6 +37,61 @@ def test_two_routes_agree(seed):
         assert np.all(a >= 0) and np.all(a <= 1 + 1e-15)
 
 
+def test_causal_lse_matches_library_logsumexp_and_closed_forms():
+    """The denominator handed over by the prefill: scipy's logsumexp as the
+    library special case; q = 0 gives log(i + 1); logits that are logarithms of
+    integers give the logarithm of their sum (tests/golden/log_integer_logits.txt)."""
+    from scipy.special import logsumexp
+    g = _rng(31)
+    n, T, D = 90, 7, 12
+    Q = 1.7 * g.standard_normal((4, T, D))
+    K = g.standard_normal((2, n, D))
+    lse = O.causal_lse(Q, K, 0.3)
+    for hq in range(4):
+        for t in range(T):
+            i = n - T + t
+            ref = logsumexp(0.3 * np.einsum("jd,d->j", K[hq // 2, : i + 1], Q[hq, t]))
+            assert abs(lse[hq, t] - ref) < 1e-12
+    z = O.causal_lse(np.zeros((2, T, D)), K)
+    assert np.max(np.abs(z - np.log(np.arange(n - T + 1, n + 1))[None, :])) < 1e-13
+    for n_ in (4, 6, 8):
+        k = np.log(np.arange(1, n_ + 1, dtype=np.float64)).reshape(1, n_, 1)
+        assert abs(O.causal_lse(np.ones((1, 1, 1)), k, 1.0)[0, 0] - math.log(n_ * (n_ + 1) / 2)) < 1e-13
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_scores_from_lse_equal_eq1_and_the_hand_worked_rationals(seed):
+    """Recomputing only the window block against the given log-sum-exp is Eq. 1
+    itself (Table 1's identity), including overlap of sink and window, no sink,
+    and a tail longer than the window."""
+    g = _rng(40 + seed)
+    n, T, D = 130, 11, 20
+    Q = 2.0 * g.standard_normal((6, T, D))
+    K = g.standard_normal((3, n, D))
+    for S, R, sc in [(4, 20, None), (0, 5, 0.2), (3, 200, None), (4, 4, None), (2, 7, 0.05)]:
+        lse = O.causal_lse(Q, K, sc)
+        a = O.lazy_scores(Q, K, S, R, sc)
+        b = O.lazy_scores_from_lse(Q, K, lse, S, R, sc)
+        assert np.max(np.abs(a - b)) < 1e-12
+    # a wrong denominator shows: doubling exp(lse) halves every mass
+    lse = O.causal_lse(Q, K)
+    a = O.lazy_scores_from_lse(Q, K, lse, 4, 20)
+    assert np.max(np.abs(O.lazy_scores_from_lse(Q, K, lse + math.log(2.0), 4, 20) - a / 2)) < 1e-13
+    # hand-worked fixture: logits ln 1 .. ln n, lse = ln(n(n+1)/2), mass of the last query as a fraction
+    import os
+    from fractions import Fraction
+    path = os.path.join(os.path.dirname(__file__), "golden", "log_integer_logits.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        n_, S, R, _, _, mass = line.split()
+        n_, S, R = int(n_), int(S), int(R)
+        k = np.log(np.arange(1, n_ + 1, dtype=np.float64)).reshape(1, n_, 1)
+        lse1 = np.array([[math.log(n_ * (n_ + 1) / 2)]])
+        got = O.lazy_scores_from_lse(np.ones((1, 1, 1)), k, lse1, S, R, 1.0)[0]
+        assert abs(got - float(Fraction(mass))) < 1e-14
+
+
 def _uniform_mass(n, S, R, T):
     """Closed form for q = 0 (uniform attention): the tail query at position i
     sees i+1 keys of which |{j<=i: j<S or j>=n-R}| are kept."""
