@@ -130,6 +130,25 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
                          float* scores /* dev */, void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
+ * Lazy ratio with the denominator given (Section 5.1: FlashAttention's prefill
+ * already produced the log-sum-exp of every attention row, so "we only need to
+ * recompute the streaming attention score", a constant-size product; Table 1).
+ * Same result as lt_lazy_scores, but only the kept keys are read:
+ *   lse     dev float [L][B][Hq][w_last]: natural logarithm of
+ *           sum_{j <= i} exp(scale * q_i . k_j) for the tail rows
+ *           i = n_ctx - w_last .. n_ctx - 1 (what the prefill attention returns)
+ *   k_full  rows j < n_sink and j >= n_ctx - n_recent of every (b, kv head) are
+ *           read; the rest of the prompt keys is not touched.
+ *   scores[l][b][hq] = mean over the tail rows of
+ *           sum_{j kept, j <= i} exp(scale * q_i . k_j - lse_i).
+ * Cost is independent of n_ctx.  Same workspace as lt_lazy_scores.
+ */
+lt_status lt_lazy_scores_lse(const lt_shape* shape, const void* q_tail /* dev */,
+                             const void* const* k_full /* host table */, const float* lse /* dev */,
+                             int32_t n_ctx, int32_t w_last, float* scores /* dev */, void* ws /* dev */,
+                             size_t ws_bytes, void* stream);
+
+/*
  * Selection (Section 5.1, the max-priority queue of size P = L - n_lazy; Fig. 3):
  * r_l = mean over [B][Hq] of scores[l] (accumulated in double, fixed order);
  * layer_mask[l] = 1 for the n_lazy layers with the largest r_l, ties to the

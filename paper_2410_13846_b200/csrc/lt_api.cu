@@ -38,14 +38,27 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   return p;
 }
 
-ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last) {
+ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only) {
   ScorePlan p;
   const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
-  int64_t want = (148 * 4 + units - 1) / units;
-  int64_t most = (n_ctx + 1023) / 1024;
+  int64_t want = (148 * 4 + units - 1) / units;  // a few CTAs per SM even for small stacks
+  int span = n_ctx;                              // keys that are divided among the splits
+  if (window_only) {
+    const int S = s.n_sink < n_ctx ? s.n_sink : n_ctx;
+    int w0 = n_ctx - s.n_recent;
+    if (w0 < S) w0 = S;
+    span = n_ctx - w0;
+  }
+  int64_t most = (span + 1023) / 1024;
   if (want > most) want = most;
   if (want < 1) want = 1;
-  p.n_splits = (int)want;
+  int len = (int)((span + want - 1) / want);
+  len = (len + 63) / 64 * 64;
+  if (len < 64) len = 64;
+  p.split_len = len;
+  p.n_splits = (int)((span + len - 1) / len);
+  if (p.n_splits < 1) p.n_splits = 1;
+  if (window_only && s.n_sink > 0) p.n_splits += 1;
   p.stat_floats = (size_t)s.n_layers * s.batch * s.n_q_heads * w_last * p.n_splits * 3;
   return p;
 }
@@ -123,8 +136,9 @@ lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w
   size_t decode_bytes = round_up(dp.ml_floats * 4, kWsAlign) + round_up(dp.o_floats * 4, kWsAlign);
   size_t score_bytes = 0;
   if (n_ctx_max > 0 && w_last_max > 0) {
-    ScorePlan sp = make_score_plan(*shape, n_ctx_max, w_last_max);
-    score_bytes = round_up(sp.stat_floats * 4, kWsAlign);
+    const ScorePlan sp = make_score_plan(*shape, n_ctx_max, w_last_max, false);
+    const ScorePlan sw = make_score_plan(*shape, n_ctx_max, w_last_max, true);
+    score_bytes = round_up((sp.stat_floats > sw.stat_floats ? sp.stat_floats : sw.stat_floats) * 4, kWsAlign);
   }
   *bytes_out = ws_prefix_bytes(*shape) + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
   return LT_OK;
@@ -148,41 +162,51 @@ lt_status lt_check(void* ws, uint32_t* flags_out, void* stream) {
   return flags ? LT_ERR_DEVICE_RANGE : LT_OK;
 }
 
-lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* const* k_full, int32_t n_ctx,
-                         int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
+// Shared body of lt_lazy_scores (lse == NULL) and lt_lazy_scores_lse.
+static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,
+                             int window_only, int32_t n_ctx, int32_t w_last, float* scores, void* ws, size_t ws_bytes,
+                             void* stream) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
+  if (window_only && !lse) return LT_ERR_INVALID_ARG;
   if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
-  if (((uintptr_t)q_tail & 15u) != 0) return LT_ERR_INVALID_ARG;
+  if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0) return LT_ERR_INVALID_ARG;
   LayerTable kf;
   if ((st = fill_table(&kf, k_full, shape->n_layers, true)) != LT_OK) return st;
-  ScorePlan sp = make_score_plan(*shape, n_ctx, w_last);
+  const ScorePlan sp = make_score_plan(*shape, n_ctx, w_last, window_only != 0);
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   const size_t prefix = ws_prefix_bytes(*shape);
   if (ws_bytes < prefix + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
   ScoreArgs a;
   a.s = *shape;
   a.q_tail = q_tail;
+  a.lse = lse;
   a.n_ctx = n_ctx;
   a.w_last = w_last;
+  a.window_only = window_only;
   a.n_splits = sp.n_splits;
+  a.split_len = sp.split_len;
   a.stats = reinterpret_cast<float*>((char*)ws + prefix);
   a.scores = scores;
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
   a.dev_err = err_word(ws);
   cudaStream_t cs = (cudaStream_t)stream;
-  // LT_SCORES_IMPL = umma | mma | generic picks a path explicitly (for A/B measurements).
-  const char* impl = getenv("LT_SCORES_IMPL");
-  cudaError_t e;
-  if (impl && !strcmp(impl, "generic")) e = launch_scores_generic(a, kf, cs);
-  else if (impl && !strcmp(impl, "mma") && scores_mma_supported(*shape, w_last)) e = launch_scores_mma(a, kf, cs);
-  else if (scores_umma_supported(*shape, w_last)) e = launch_scores_umma(a, kf, cs);
-  else if (scores_mma_supported(*shape, w_last)) e = launch_scores_mma(a, kf, cs);
-  else e = launch_scores_generic(a, kf, cs);
+  cudaError_t e = scores_umma_supported(*shape, w_last) ? launch_scores_umma(a, kf, cs)
+                                                        : launch_scores_generic(a, kf, cs);
   if (e != cudaSuccess) return LT_ERR_CUDA;
   e = launch_scores_finish(a, cs);
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* const* k_full, int32_t n_ctx,
+                         int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  return scores_impl(shape, q_tail, k_full, nullptr, 0, n_ctx, w_last, scores, ws, ws_bytes, stream);
+}
+
+lt_status lt_lazy_scores_lse(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,
+                             int32_t n_ctx, int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  return scores_impl(shape, q_tail, k_full, lse, 1, n_ctx, w_last, scores, ws, ws_bytes, stream);
 }
 
 lt_status lt_select_lazy(const float* scores, int32_t n_layers, int32_t batch, int32_t n_q_heads, int32_t n_lazy,

@@ -33,12 +33,15 @@ struct DecodePlan {
 };
 DecodePlan make_decode_plan(const lt_shape& s);
 
-// Split plan of the scoring pass.
+// Split plan of the scoring pass.  With the denominator given (window_only)
+// only the kept keys are visited: split 0 is the sink range when n_sink > 0,
+// the other splits are equal parts of the recent range.
 struct ScorePlan {
   int n_splits;        // key-range splits per (layer, batch row, kv head)
+  int split_len;       // keys per split (of the whole prompt, or of the recent range)
   size_t stat_floats;  // [L][B][Hq][T][n_splits][3] partial (max, sum_all, sum_window)
 };
-ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last);
+ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only);
 
 inline float resolved_scale(const lt_shape& s) {
   return s.softmax_scale > 0.f ? s.softmax_scale : 1.0f / sqrtf((float)s.head_dim);
@@ -98,16 +101,39 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const L
 struct ScoreArgs {
   lt_shape s;
   const void* q_tail;
+  const float* lse;  // window_only: natural-log denominators [L][B][Hq][T]
   int n_ctx, w_last;
-  int n_splits;
+  int window_only;
+  int n_splits, split_len;
   float cs;      // softmax scale * log2(e)
   float* stats;  // workspace
   float* scores;
   uint32_t* dev_err;
 };
+// Key range [*k0, *k1) of split sp (see ScorePlan).
+__host__ __device__ inline void score_split_range(const ScoreArgs& a, int sp, int* k0, int* k1) {
+  if (!a.window_only) {
+    *k0 = sp * a.split_len;
+    *k1 = (*k0 + a.split_len < a.n_ctx) ? *k0 + a.split_len : a.n_ctx;
+    if (*k0 > a.n_ctx) *k0 = a.n_ctx;
+    return;
+  }
+  const int S = a.s.n_sink < a.n_ctx ? a.s.n_sink : a.n_ctx;
+  if (a.s.n_sink > 0) {
+    if (sp == 0) {
+      *k0 = 0;
+      *k1 = S;
+      return;
+    }
+    sp -= 1;
+  }
+  int w0 = a.n_ctx - a.s.n_recent;
+  if (w0 < S) w0 = S;
+  *k0 = w0 + sp * a.split_len;
+  if (*k0 > a.n_ctx) *k0 = a.n_ctx;
+  *k1 = (*k0 + a.split_len < a.n_ctx) ? *k0 + a.split_len : a.n_ctx;
+}
 cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
-bool scores_mma_supported(const lt_shape& s, int w_last);
-cudaError_t launch_scores_mma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
 // bf16, head_dim 128: tcgen05 / TMEM path.
 bool scores_umma_supported(const lt_shape& s, int w_last);
 cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);

@@ -23,11 +23,6 @@ __device__ __forceinline__ float ld_f32<__nv_bfloat16>(const __nv_bfloat16* p) {
   return __bfloat162float(*p);
 }
 
-__host__ __device__ inline int score_split_len(int n_ctx, int n_splits) {
-  int len = (n_ctx + n_splits - 1) / n_splits;
-  return (len + 63) / 64 * 64;
-}
-
 // grid (w_last * n_splits, B * Hq, L); block 128.
 template <typename T, int D>
 __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
@@ -43,9 +38,9 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
   for (int d = threadIdx.x; d < D; d += blockDim.x) qs[d] = ld_f32<T>(qp + d);
   __syncthreads();
   const int i = a.n_ctx - a.w_last + t;  // position of this query; sees keys 0..i
-  const int len = score_split_len(a.n_ctx, a.n_splits);
-  const int j0 = sp * len;
-  const int j1 = min(i + 1, j0 + len);
+  int j0, j1;
+  score_split_range(a, sp, &j0, &j1);
+  j1 = min(i + 1, j1);
   const T* Kb = (const T*)kf.p[l] + ((long long)(b * s.n_kv_heads + h) * s.full_capacity) * D;
   float M = -INFINITY, A = 0.f, W = 0.f;
   for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
@@ -108,13 +103,21 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
     const float* st = a.stats + ((idx * a.w_last + t) * a.n_splits) * 3;
     float Mx = -INFINITY;
     for (int sp = 0; sp < a.n_splits; ++sp) Mx = fmaxf(Mx, st[sp * 3]);
-    float A = 0.f, W = 0.f;
-    for (int sp = 0; sp < a.n_splits; ++sp) {
-      const float w = exp2f(st[sp * 3] - Mx);
-      A += w * st[sp * 3 + 1];
-      W += w * st[sp * 3 + 2];
+    if (a.window_only) {
+      // denominator given: mass = sum over splits of W * 2^(M - lse * log2(e))
+      const float lse2 = a.lse[idx * a.w_last + t] * 1.4426950408889634f;
+      float W = 0.f;
+      for (int sp = 0; sp < a.n_splits; ++sp) W += st[sp * 3 + 2] * exp2f(st[sp * 3] - lse2);
+      sum += W;
+    } else {
+      float A = 0.f, W = 0.f;
+      for (int sp = 0; sp < a.n_splits; ++sp) {
+        const float w = exp2f(st[sp * 3] - Mx);
+        A += w * st[sp * 3 + 1];
+        W += w * st[sp * 3 + 2];
+      }
+      sum += W / A;
     }
-    sum += W / A;
   }
   a.scores[idx] = sum / (float)a.w_last;
 }
@@ -152,7 +155,5 @@ cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy,
   select_kernel<<<1, LT_MAX_LAYERS, 0, st>>>(scores, L, B * Hq, n_lazy, mask, ratio);
   return cudaGetLastError();
 }
-
-// Tensor-core scoring path: provided by lt_scores_mma.cu.
 
 }  // namespace lt

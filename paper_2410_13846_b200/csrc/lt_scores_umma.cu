@@ -188,11 +188,6 @@ __device__ __forceinline__ float sum_ex2_64(const uint32_t (&v)[64], float cs, f
   return (s0 + s1) + (s2 + s3);
 }
 
-__host__ __device__ inline int split_len_umma(int n_ctx, int n_splits) {
-  int len = (n_ctx + n_splits - 1) / n_splits;
-  return (len + 63) / 64 * 64;
-}
-
 }  // namespace
 
 // grid (n_splits * row_blocks, B * Hkv, L); block 384.
@@ -225,9 +220,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int l = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_ctx = a.n_ctx;
-  const int len = split_len_umma(n_ctx, a.n_splits);
-  const int k0 = sp * len;
-  const int k1 = min(n_ctx, k0 + len);
+  int k0, k1;
+  score_split_range(a, sp, &k0, &k1);
   const int n_tiles = k1 > k0 ? (k1 - k0 + kBlockN - 1) / kBlockN : 0;
   const int rows_here = min(kBlockM, M - rb * kBlockM);  // valid query rows of this CTA
   const int n_mb = (rows_here + 127) / 128;              // UMMA row blocks in use

@@ -81,3 +81,60 @@ def test_select_ties_go_to_lower_index():
         mask = torch.zeros(6, dtype=torch.uint8, device="cuda")
         lt.select_lazy(d, 6, 1, 3, n_lazy, mask)
         assert np.array_equal(mask.cpu().numpy(), O.select_lazy(sc, n_lazy)[0])
+
+
+# ---- the deployed form: denominator given, only the kept keys are read ---------------
+def _oracle_lse(st, q_tail, n_ctx):
+    s = st.shape
+    scale = s.softmax_scale if s.softmax_scale > 0 else None
+    return np.array([[O.causal_lse(f64(q_tail[l, b]), f64(st.k_full[l][b, :, :n_ctx]), scale)
+                      for b in range(s.batch)] for l in range(s.n_layers)])          # [L, B, Hq, T]
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv,S,R,n_ctx,T,scale", CASES)
+def test_scores_from_lse_match_eq1(dtype, D, Hq, Hkv, S, R, n_ctx, T, scale):
+    """lt_lazy_scores_lse against the DEFINITION (O3, Eq. 1 over all keys), with the
+    log-sum-exp an fp64 prefill would hand over rounded to fp32.  Keys outside the
+    kept set hold NaN: the call must not read them."""
+    torch.manual_seed(7)
+    L, B = 2, 2
+    cap = n_ctx + 3
+    st = Stack(L, B, Hq, Hkv, D, S, R, cap, dtype, scale, n_ctx_max=n_ctx, w_last_max=T)
+    for l in range(L):
+        st.k_full[l][:, :, :n_ctx] = torch.randn(B, Hkv, n_ctx, D).to(dtype).cuda()
+        st.k_full[l][:, :, n_ctx:] = float("nan")
+    q_tail = (1.3 * torch.randn(L, B, Hq, T, D)).to(dtype).cuda()
+    ref = _oracle_scores(st, q_tail, n_ctx)
+    lse = torch.from_numpy(_oracle_lse(st, q_tail, n_ctx)).float().cuda().contiguous()
+    for l in range(L):                                   # poison everything a lazy layer would discard
+        lo, hi = min(S, n_ctx), max(S, n_ctx - R)
+        st.k_full[l][:, :, lo:hi] = float("nan")
+    s = st.shape
+    got = torch.full((L, B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+    lt.lazy_scores_lse(s, q_tail, st.tables, lse, n_ctx, T, got, st.ws)
+    assert lt.check(st.ws) == 0
+    g = f64(got)
+    assert np.isfinite(g).all()
+    assert np.max(np.abs(g - ref)) <= SCORE_ABS, np.max(np.abs(g - ref))
+    ref2 = np.array([[O.lazy_scores_from_lse(f64(q_tail[l, b]), np.nan_to_num(f64(st.k_full[l][b, :, :n_ctx])),
+                                             f64(lse[l, b]), S, R, s.softmax_scale if s.softmax_scale > 0 else None)
+                      for b in range(B)] for l in range(L)])
+    assert np.max(np.abs(g - ref2)) <= SCORE_ABS
+
+
+def test_both_scoring_routes_give_the_same_mask_on_a_planted_stack():
+    from synth import CONFIGS
+    from tests.gpu_util import build_stack
+    cfg = CONFIGS["llama3_8b_32k"].scaled(name="mini", n_layers=6, batch=2, n_ctx=3000, n_recent=252, n_lazy=3, steps=1)
+    st, q_tail, planted = build_stack(cfg)
+    s = st.shape
+    L, B, Hq = cfg.n_layers, cfg.batch, cfg.n_q_heads
+    a = torch.zeros((L, B, Hq), dtype=torch.float32, device="cuda")
+    b = torch.zeros_like(a)
+    lt.lazy_scores(s, q_tail, st.tables, cfg.n_ctx, cfg.w_last, a, st.ws)
+    lse = torch.from_numpy(_oracle_lse(st, q_tail, cfg.n_ctx)).float().cuda().contiguous()
+    lt.lazy_scores_lse(s, q_tail, st.tables, lse, cfg.n_ctx, cfg.w_last, b, st.ws)
+    assert float((a - b).abs().max()) <= 2e-4
+    ma = torch.zeros(L, dtype=torch.uint8, device="cuda"); mb = torch.zeros_like(ma)
+    lt.select_lazy(a, L, B, Hq, cfg.n_lazy, ma); lt.select_lazy(b, L, B, Hq, cfg.n_lazy, mb)
+    assert torch.equal(ma, mb) and sorted(torch.nonzero(ma).flatten().tolist()) == planted
