@@ -55,6 +55,9 @@ __all__ = [
     "layer_ratios",
     "select_lazy",
     "select_lazy_priority_queue",
+    "select_lazy_priority_queue_trace",
+    "select_lazy_per_sequence",
+    "lazy_scores_per_row_window",
     "ring_slot",
     "ring_valid_slots",
     "ring_owner",
@@ -259,6 +262,31 @@ def lazy_scores_from_lse(Q_tail, K, lse, n_sink: int, n_recent: int, scale=None)
     return score
 
 
+def lazy_scores_per_row_window(Q_tail, K, n_sink: int, n_recent: int, scale=None):
+    """O3 under the other reading of X_recent (Appendix E: the mask M_lazy keeps,
+    for row i, "the first 4 and the last 1020 tokens" of [i]): the recent set of
+    the tail query at position i is {i - n_recent + 1 .. i} instead of the fixed
+    block {n - n_recent .. n - 1}.  Both readings agree for the last query.
+    """
+    Q_tail, K = _f64(Q_tail), _f64(K)
+    Hq, T, D = Q_tail.shape
+    Hkv, n, _ = K.shape
+    assert Hq % Hkv == 0 and 1 <= T <= n
+    G = Hq // Hkv
+    sc = _default_scale(D, scale)
+    score = np.zeros(Hq, dtype=np.float64)
+    for hq in range(Hq):
+        acc = 0.0
+        for t in range(T):
+            i = n - T + t
+            s = sc * (K[hq // G, : i + 1] @ Q_tail[hq, t])
+            p = softmax(s)
+            j = np.arange(i + 1)
+            acc += float(np.sum(p[(j < n_sink) | (j > i - n_recent)]))
+        score[hq] = acc / T
+    return score
+
+
 # --------------------------------------------------------------------------
 # O4: selection
 # --------------------------------------------------------------------------
@@ -302,6 +330,40 @@ def select_lazy_priority_queue(ratios, n_full: int):
             _, popped = heapq.heappop(heap)
             mask[popped] = 1
     return mask
+
+
+def select_lazy_priority_queue_trace(ratios, n_full: int):
+    """The same queue, one layer at a time (Figure 3): popped[l] is the layer
+    that leaves the queue - and becomes lazy, its KV reduced at once - when
+    layer l arrives, or -1 while the queue still has room.  returns (mask, popped).
+    """
+    ratios = _f64(ratios)
+    L = ratios.shape[0]
+    mask = np.zeros(L, dtype=np.uint8)
+    popped = np.full(L, -1, dtype=np.int64)
+    queue = []  # layers currently held, kept as a plain list: the definition, not a heap
+    for l in range(L):
+        queue.append(l)
+        if len(queue) > n_full:
+            top = max(queue, key=lambda m: (ratios[m], -m))  # highest ratio, lower index on ties
+            queue.remove(top)
+            mask[top] = 1
+            popped[l] = top
+    return mask, popped
+
+
+def select_lazy_per_sequence(scores, n_lazy: int):
+    """O4 per prompt (Section 4: the lazy layers "vary according to different
+    prompts"): row b of the result is select_lazy on that batch row's scores
+    alone.  scores [L, B, Hq] -> mask uint8 [B, L], r float64 [B, L].
+    """
+    scores = _f64(scores)
+    L, B, _ = scores.shape
+    mask = np.zeros((B, L), dtype=np.uint8)
+    r = np.zeros((B, L), dtype=np.float64)
+    for b in range(B):
+        mask[b], r[b] = select_lazy(scores[:, b : b + 1, :], n_lazy)
+    return mask, r
 
 
 # --------------------------------------------------------------------------

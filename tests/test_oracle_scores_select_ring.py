@@ -214,6 +214,86 @@ def test_priority_queue_follows_figure_3_trace():
     assert mask.tolist() == [0, 1, 1, 1, 0]
 
 
+def test_priority_queue_trace_pops_on_arrival_and_ends_at_the_sorted_selection():
+    """Figure 3 again, step by step: with P = 2 on .3 .8 .5 .9 .1 nothing leaves
+    while layers 0, 1 arrive, layer 1 leaves when layer 2 arrives, layer 3 leaves
+    on its own arrival, layer 2 leaves when layer 4 arrives."""
+    mask, popped = O.select_lazy_priority_queue_trace([0.3, 0.8, 0.5, 0.9, 0.1], 2)
+    assert popped.tolist() == [-1, -1, 1, 3, 2] and mask.tolist() == [0, 1, 1, 1, 0]
+    g = _rng(77)
+    for _ in range(20):
+        L = int(g.integers(1, 12))
+        r = np.round(g.random(L), 1)                     # coarse values: ties happen
+        for P in range(L + 1):
+            mask, popped = O.select_lazy_priority_queue_trace(r, P)
+            assert np.array_equal(mask, O.select_lazy_priority_queue(r, P))
+            assert np.array_equal(mask, O.select_lazy(r.reshape(L, 1, 1), L - P)[0])
+            out = [x for x in popped.tolist() if x >= 0]
+            assert len(out) == len(set(out)) == L - P == int(mask.sum())
+            assert all(x <= l for l, x in enumerate(popped.tolist()))    # only layers that have arrived can leave
+            # while at most P layers have arrived nothing leaves
+            assert all(x == -1 for x in popped.tolist()[:P])
+
+
+def test_per_sequence_selection_is_the_single_prompt_selection_row_by_row():
+    g = _rng(78)
+    L, B, Hq = 7, 4, 3
+    scores = g.random((L, B, Hq))
+    for n_lazy in range(L + 1):
+        mask, r = O.select_lazy_per_sequence(scores, n_lazy)
+        assert mask.shape == (B, L) and np.all(mask.sum(axis=1) == n_lazy)
+        for b in range(B):
+            rb = scores[:, b, :].mean(axis=1)
+            assert np.allclose(r[b], rb, atol=1e-15)
+            best = max(sum(rb[list(c)]) for c in itertools.combinations(range(L), n_lazy))
+            assert abs(rb[mask[b] == 1].sum() - best) < 1e-12
+    # one prompt: identical to the batch selection
+    one = g.random((L, 1, Hq))
+    assert np.array_equal(O.select_lazy_per_sequence(one, 3)[0][0], O.select_lazy(one, 3)[0])
+    # prompts that disagree get different masks
+    two = np.zeros((2, 2, 1)); two[0, 0] = 0.9; two[1, 0] = 0.1; two[0, 1] = 0.2; two[1, 1] = 0.7
+    assert O.select_lazy_per_sequence(two, 1)[0].tolist() == [[1, 0], [0, 1]]
+
+
+def _brute_lazy_per_row(Q, K, G, S, R, scale):
+    res = []
+    for hq in range(len(Q)):
+        T, n = len(Q[hq]), len(K[0])
+        acc = 0.0
+        for t in range(T):
+            i = n - T + t
+            lg = [scale * math.fsum(a * b for a, b in zip(Q[hq][t], K[hq // G][j])) for j in range(i + 1)]
+            mx = max(lg)
+            w = [math.exp(x - mx) for x in lg]
+            acc += math.fsum(w[j] for j in range(i + 1) if (j < S or j > i - R)) / math.fsum(w)
+        res.append(acc / T)
+    return res
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_per_row_window_reading(seed):
+    """Brute force; agreement with the fixed-block reading for the last query
+    (T = 1); closed form for uniform attention; 1 when every row's window covers
+    its keys; never below the fixed-block ratio minus the keys the block adds."""
+    g = _rng(90 + seed)
+    Hkv, G = int(g.integers(1, 3)), int(g.integers(1, 4))
+    n = int(g.integers(2, 12))
+    T = int(g.integers(1, n + 1))
+    D = int(g.integers(1, 5))
+    S, R = int(g.integers(0, 4)), int(g.integers(1, 6))
+    Q = g.standard_normal((Hkv * G, T, D))
+    K = g.standard_normal((Hkv, n, D))
+    got = O.lazy_scores_per_row_window(Q, K, S, R)
+    bf = np.array(_brute_lazy_per_row(Q.tolist(), K.tolist(), G, S, R, 1 / math.sqrt(D)))
+    assert np.max(np.abs(got - bf)) < 1e-13
+    last = O.lazy_scores_per_row_window(Q[:, -1:], K, S, R)
+    assert np.max(np.abs(last - O.lazy_scores(Q[:, -1:], K, S, R))) < 1e-13
+    z = O.lazy_scores_per_row_window(np.zeros((1, T, D)), K[:1], S, R)[0]
+    exp = sum(len({j for j in range(i + 1) if j < S or j > i - R}) / (i + 1) for i in range(n - T, n)) / T
+    assert abs(z - exp) < 1e-13
+    assert np.max(np.abs(O.lazy_scores_per_row_window(Q, K, S, n) - 1.0)) < 1e-12
+
+
 # ---------------------------------------------------------------- O5 --------
 @pytest.mark.parametrize("S,R", [(0, 1), (0, 5), (4, 1), (4, 6), (3, 8), (2, 2)])
 def test_ring_exhaustive(S, R):
