@@ -27,7 +27,8 @@
  *       full cache of one layer    [batch][n_kv_heads][full_capacity][head_dim]
  *       stream cache of one layer  [batch][n_kv_heads][n_sink+n_recent][head_dim]
  *     Every cache pointer must be 16-byte aligned.
- *   - layer_mask is uint8[n_layers] on the device, 1 = lazy (streaming).
+ *   - layer_mask is uint8[n_layers] on the device, 1 = lazy (streaming); with
+ *     shape.per_sequence_mask it is uint8[batch][n_layers], one row per prompt.
  *   - seq_lens is int32[batch] on the device: tokens already in the cache of
  *     that batch row = position of the next token.
  *   - A decode step is "append, then attend": the new token attends to itself
@@ -76,6 +77,12 @@ typedef struct lt_shape {
   int32_t full_capacity; /* rows per (batch, kv head) of a full cache */
   int32_t dtype;         /* LT_F32 or LT_BF16: q, k, v and both caches */
   float softmax_scale;   /* <= 0 means 1/sqrt(head_dim) */
+  int32_t per_sequence_mask; /* 0: layer_mask is uint8[n_layers], one hybrid for the batch;
+                                1: uint8[batch][n_layers], every prompt has its own lazy layers
+                                   (Section 4: the lazy layers vary with the prompt) */
+  int32_t recent_per_row;    /* scoring only.  0: X_recent is the fixed block of the last n_recent prompt
+                                positions (Table 1, the set a lazy layer retains); 1: the recent set of the
+                                tail query at position i is i - n_recent + 1 .. i (Appendix E, M_lazy row by row) */
 } lt_shape;
 
 /* Text for a status code (static storage, never NULL). */
@@ -161,6 +168,37 @@ lt_status lt_select_lazy(const float* scores /* dev [L][B][Hq] */, int32_t n_lay
                          float* layer_ratio /* dev [L] or NULL */, void* stream);
 
 /*
+ * Per-prompt selection (Section 4: the layers that are lazy "vary according to
+ * different prompts"): for every batch row b, r = mean over [Hq] of
+ * scores[l][b] and the n_lazy layers with the largest r become lazy for that
+ * prompt.  layer_mask dev uint8 [B][L], layer_ratio dev float [B][L] or NULL.
+ * Use the result with shape.per_sequence_mask = 1.
+ */
+lt_status lt_select_lazy_per_seq(const float* scores /* dev [L][B][Hq] */, int32_t n_layers, int32_t batch,
+                                 int32_t n_q_heads, int32_t n_lazy, uint8_t* layer_mask /* dev [B][L] */,
+                                 float* layer_ratio /* dev [B][L] or NULL */, void* stream);
+
+/*
+ * Streaming selection, one layer at a time (Section 5.1 and Figure 3: the
+ * ratios enter a priority queue of capacity P = n_full during prefilling; when
+ * the queue overflows, the layer with the highest ratio is popped, labelled
+ * lazy and its KV reduced at once, so at most P full caches ever exist).
+ * Call in layer order, right after layer `layer`'s scores are known:
+ *   layer_scores  dev float [B][Hq]: this layer's slice of the lt_lazy_scores output
+ *   queue_state   dev, 8 * n_layers bytes, 8-byte aligned, owned by the caller;
+ *                 layer 0 starts a new prompt (state and mask are reset)
+ *   layer_mask    dev uint8 [L]: updated in place (the popped layer becomes 1)
+ *   popped_layer  dev int32 or NULL: the layer that left the queue, or -1
+ * After the last layer the mask equals lt_select_lazy(n_lazy = L - n_full) on
+ * the same scores.  lt_stream_init_layer compacts the popped layer without a
+ * host round trip.
+ */
+lt_status lt_select_lazy_push(const float* layer_scores /* dev */, int32_t layer, int32_t n_layers, int32_t batch,
+                              int32_t n_q_heads, int32_t n_full, void* queue_state /* dev */,
+                              uint8_t* layer_mask /* dev [L] */, int32_t* popped_layer /* dev or NULL */,
+                              void* stream);
+
+/*
  * Prefill -> decode compaction of the lazy layers (Section 5.1: "retain only
  * the KV caches corresponding to {X_initial, X_recent} and discard others";
  * Fig. 3).  For every layer with mask 1 and every (b, kv head), prompt rows
@@ -174,6 +212,17 @@ lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask /* dev
                          const int32_t* seq_lens /* dev [B] */, void* const* k_stream,
                          void* const* v_stream /* host tables */, void* ws /* dev, for the error word; may be NULL */,
                          void* stream);
+
+/*
+ * lt_stream_init for the one layer whose index is stored at *layer on the
+ * device (nothing happens when it is -1 or the mask of that layer is 0): the
+ * compaction step of the streaming selection above.
+ */
+lt_status lt_stream_init_layer(const lt_shape* shape, const uint8_t* layer_mask /* dev */,
+                               const int32_t* layer /* dev */, const void* const* k_full,
+                               const void* const* v_full /* host tables */, const int32_t* seq_lens /* dev [B] */,
+                               void* const* k_stream, void* const* v_stream /* host tables */,
+                               void* ws /* dev, for the error word; may be NULL */, void* stream);
 
 /*
  * Per-step KV append (Section 3: decoding "saves their KV cache"; Section 5.1

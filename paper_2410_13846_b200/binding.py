@@ -25,7 +25,8 @@ class LtError(RuntimeError):
 class _CShape(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_sink", "n_recent",
-                 "full_capacity", "dtype")] + [("softmax_scale", C.c_float)]
+                 "full_capacity", "dtype")] + [("softmax_scale", C.c_float), ("per_sequence_mask", C.c_int32),
+                                                ("recent_per_row", C.c_int32)]
 
 
 @dataclass
@@ -40,10 +41,13 @@ class Shape:
     full_capacity: int
     dtype: int = LT_BF16
     softmax_scale: float = 0.0
+    per_sequence_mask: int = 0
+    recent_per_row: int = 0
 
     def c(self) -> _CShape:
         return _CShape(self.n_layers, self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_sink,
-                       self.n_recent, self.full_capacity, self.dtype, self.softmax_scale)
+                       self.n_recent, self.full_capacity, self.dtype, self.softmax_scale, self.per_sequence_mask,
+                       self.recent_per_row)
 
     @property
     def stream_capacity(self) -> int:
@@ -85,6 +89,12 @@ def lib() -> C.CDLL:
     L.lt_lazy_scores_lse.argtypes = [shp, vp, tab, vp, i32, i32, vp, vp, sz, vp]
     L.lt_select_lazy.restype = i32
     L.lt_select_lazy.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    L.lt_select_lazy_per_seq.restype = i32
+    L.lt_select_lazy_per_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    L.lt_select_lazy_push.restype = i32
+    L.lt_select_lazy_push.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    L.lt_stream_init_layer.restype = i32
+    L.lt_stream_init_layer.argtypes = [shp, vp, vp, tab, tab, vp, tab, tab, vp, vp]
     L.lt_stream_init.restype = i32
     L.lt_stream_init.argtypes = [shp, vp, tab, tab, vp, tab, tab, vp, vp]
     L.lt_kv_append.restype = i32
@@ -194,6 +204,24 @@ def select_lazy(scores, n_layers: int, batch: int, n_q_heads: int, n_lazy: int, 
                 stream=None):
     _ok(lib().lt_select_lazy(_ptr(scores), n_layers, batch, n_q_heads, n_lazy, _ptr(layer_mask),
                              _ptr(layer_ratio), _stream(stream)), "lt_select_lazy")
+
+
+def select_lazy_per_seq(scores, n_layers: int, batch: int, n_q_heads: int, n_lazy: int, layer_mask, layer_ratio=None,
+                        stream=None):
+    _ok(lib().lt_select_lazy_per_seq(_ptr(scores), n_layers, batch, n_q_heads, n_lazy, _ptr(layer_mask),
+                                     _ptr(layer_ratio), _stream(stream)), "lt_select_lazy_per_seq")
+
+
+def select_lazy_push(layer_scores, layer: int, n_layers: int, batch: int, n_q_heads: int, n_full: int, queue_state,
+                     layer_mask, popped_layer=None, stream=None):
+    _ok(lib().lt_select_lazy_push(_ptr(layer_scores), layer, n_layers, batch, n_q_heads, n_full, _ptr(queue_state),
+                                  _ptr(layer_mask), _ptr(popped_layer), _stream(stream)), "lt_select_lazy_push")
+
+
+def stream_init_layer(shape: Shape, layer_mask, layer, tables: LayerTables, seq_lens, ws=None, stream=None):
+    _ok(lib().lt_stream_init_layer(C.byref(shape.c()), _ptr(layer_mask), _ptr(layer), tables.k_full, tables.v_full,
+                                   _ptr(seq_lens), tables.k_stream, tables.v_stream, _ptr(ws), _stream(stream)),
+        "lt_stream_init_layer")
 
 
 def stream_init(shape: Shape, layer_mask, tables: LayerTables, seq_lens, ws=None, stream=None):

@@ -19,6 +19,7 @@ lt_status validate_shape(const lt_shape* s) {
   if (s->head_dim != 64 && s->head_dim != 128) return LT_ERR_UNSUPPORTED;
   if (s->dtype != LT_F32 && s->dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
   if (!(s->softmax_scale == s->softmax_scale)) return LT_ERR_INVALID_ARG;  // NaN
+  if ((s->per_sequence_mask | s->recent_per_row) & ~1) return LT_ERR_INVALID_ARG;
   return LT_OK;
 }
 
@@ -45,7 +46,7 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
   int span = n_ctx;                              // keys that are divided among the splits
   if (window_only) {
     const int S = s.n_sink < n_ctx ? s.n_sink : n_ctx;
-    int w0 = n_ctx - s.n_recent;
+    int w0 = n_ctx - s.n_recent - (s.recent_per_row ? w_last - 1 : 0);
     if (w0 < S) w0 = S;
     span = n_ctx - w0;
   }
@@ -220,9 +221,34 @@ lt_status lt_select_lazy(const float* scores, int32_t n_layers, int32_t batch, i
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 
-lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask, const void* const* k_full,
-                         const void* const* v_full, const int32_t* seq_lens, void* const* k_stream,
-                         void* const* v_stream, void* ws, void* stream) {
+lt_status lt_select_lazy_per_seq(const float* scores, int32_t n_layers, int32_t batch, int32_t n_q_heads,
+                                 int32_t n_lazy, uint8_t* layer_mask, float* layer_ratio, void* stream) {
+  if (!scores || !layer_mask) return LT_ERR_INVALID_ARG;
+  if (n_layers < 1 || batch < 1 || n_q_heads < 1) return LT_ERR_INVALID_ARG;
+  if (n_layers > LT_MAX_LAYERS) return LT_ERR_UNSUPPORTED;
+  if (n_lazy < 0 || n_lazy > n_layers) return LT_ERR_INVALID_ARG;
+  cudaError_t e = launch_select_per_seq(scores, n_layers, batch, n_q_heads, n_lazy, layer_mask, layer_ratio,
+                                        (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_select_lazy_push(const float* layer_scores, int32_t layer, int32_t n_layers, int32_t batch,
+                              int32_t n_q_heads, int32_t n_full, void* queue_state, uint8_t* layer_mask,
+                              int32_t* popped_layer, void* stream) {
+  if (!layer_scores || !queue_state || !layer_mask) return LT_ERR_INVALID_ARG;
+  if (n_layers < 1 || batch < 1 || n_q_heads < 1) return LT_ERR_INVALID_ARG;
+  if (n_layers > LT_MAX_LAYERS) return LT_ERR_UNSUPPORTED;
+  if (layer < 0 || layer >= n_layers || n_full < 0 || n_full > n_layers) return LT_ERR_INVALID_ARG;
+  if (((uintptr_t)queue_state & 7u) != 0) return LT_ERR_INVALID_ARG;
+  cudaError_t e = launch_select_push(layer_scores, layer, n_layers, batch * n_q_heads, n_full,
+                                     reinterpret_cast<double*>(queue_state), layer_mask, popped_layer,
+                                     (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+static lt_status stream_init_impl(const lt_shape* shape, const uint8_t* layer_mask, const void* const* k_full,
+                                  const void* const* v_full, const int32_t* seq_lens, void* const* k_stream,
+                                  void* const* v_stream, const int32_t* only_layer, void* ws, void* stream) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!layer_mask || !k_full || !v_full || !seq_lens || !k_stream || !v_stream) return LT_ERR_INVALID_ARG;
@@ -233,9 +259,22 @@ lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask, const
   if ((st = fill_table(&vf, v_full, L, false)) != LT_OK) return st;
   if ((st = fill_table(&ks, (const void* const*)k_stream, L, false)) != LT_OK) return st;
   if ((st = fill_table(&vs, (const void* const*)v_stream, L, false)) != LT_OK) return st;
-  cudaError_t e = launch_stream_init(*shape, layer_mask, kf, vf, seq_lens, ks, vs, ws ? err_word(ws) : nullptr,
-                                     (cudaStream_t)stream);
+  cudaError_t e = launch_stream_init(*shape, layer_mask, kf, vf, seq_lens, ks, vs, only_layer,
+                                     ws ? err_word(ws) : nullptr, (cudaStream_t)stream);
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+lt_status lt_stream_init(const lt_shape* shape, const uint8_t* layer_mask, const void* const* k_full,
+                         const void* const* v_full, const int32_t* seq_lens, void* const* k_stream,
+                         void* const* v_stream, void* ws, void* stream) {
+  return stream_init_impl(shape, layer_mask, k_full, v_full, seq_lens, k_stream, v_stream, nullptr, ws, stream);
+}
+
+lt_status lt_stream_init_layer(const lt_shape* shape, const uint8_t* layer_mask, const int32_t* layer,
+                               const void* const* k_full, const void* const* v_full, const int32_t* seq_lens,
+                               void* const* k_stream, void* const* v_stream, void* ws, void* stream) {
+  if (!layer) return LT_ERR_INVALID_ARG;
+  return stream_init_impl(shape, layer_mask, k_full, v_full, seq_lens, k_stream, v_stream, layer, ws, stream);
 }
 
 lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask, const void* k_new, const void* v_new,

@@ -12,6 +12,7 @@ __global__ void append_kernel(const uint8_t* __restrict__ mask, const uint4* __r
                               const uint4* __restrict__ v_new, const int32_t* __restrict__ seq_lens,
                               LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs, int layer_begin,
                               int layer_count, int B, int Hkv, int vec_per_row, int S, int R, int cap,
+                              int mask_row /* layers per mask row, 0 = one mask for the batch */,
                               uint32_t* dev_err) {
   const long long total = (long long)layer_count * B * Hkv * vec_per_row;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -22,7 +23,7 @@ __global__ void append_kernel(const uint8_t* __restrict__ mask, const uint4* __r
   const int b = (int)((row / Hkv) % B);
   const int l = layer_begin + (int)(row / ((long long)Hkv * B));
   const int pos = seq_lens[b];
-  const bool lazy = mask[l] != 0;
+  const bool lazy = mask[b * mask_row + l] != 0;
   uint4* kdst = (uint4*)(lazy ? ks.p[l] : kf.p[l]);
   uint4* vdst = (uint4*)(lazy ? vs.p[l] : vf.p[l]);
   if (!kdst || !vdst) {
@@ -62,7 +63,8 @@ cudaError_t launch_append(const lt_shape& s, const uint8_t* mask, const void* k_
   // k_new / v_new are indexed by absolute layer: shift the base so that layer_begin lands at its row
   append_kernel<<<(unsigned)blocks, threads, 0, st>>>(mask, (const uint4*)k_new, (const uint4*)v_new, seq_lens, kf, vf,
                                                       ks, vs, layer_begin, layer_count, s.batch, s.n_kv_heads,
-                                                      vec_per_row, s.n_sink, s.n_recent, s.full_capacity, dev_err);
+                                                      vec_per_row, s.n_sink, s.n_recent, s.full_capacity,
+                                                      s.per_sequence_mask ? s.n_layers : 0, dev_err);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (advance) {
@@ -76,11 +78,13 @@ cudaError_t launch_append(const lt_shape& s, const uint8_t* mask, const void* k_
 // row of the last position that maps to it, so no two threads write one row.
 __global__ void stream_init_kernel(const uint8_t* __restrict__ mask, LayerTable kf, LayerTable vf,
                                    const int32_t* __restrict__ seq_lens, LayerTable ks, LayerTable vs, int B,
-                                   int Hkv, int vec_per_row, int S, int R, int cap, uint32_t* dev_err) {
+                                   int Hkv, int vec_per_row, int S, int R, int cap, int mask_row,
+                                   const int32_t* __restrict__ only_layer, uint32_t* dev_err) {
   const int l = blockIdx.z;
-  if (mask[l] == 0) return;
   const int bh = blockIdx.y;
   const int b = bh / Hkv;
+  if (only_layer && *only_layer != l) return;  // compaction of the one layer named on the device
+  if (mask[b * mask_row + l] == 0) return;
   const int C = S + R;
   const uint4* ksrc = (const uint4*)kf.p[l];
   const uint4* vsrc = (const uint4*)vf.p[l];
@@ -118,7 +122,7 @@ __global__ void stream_init_kernel(const uint8_t* __restrict__ mask, LayerTable 
 
 cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const LayerTable& kf, const LayerTable& vf,
                                const int32_t* seq_lens, const LayerTable& ks, const LayerTable& vs,
-                               uint32_t* dev_err, cudaStream_t st) {
+                               const int32_t* only_layer, uint32_t* dev_err, cudaStream_t st) {
   const int vec_per_row = (int)(s.head_dim * elem_bytes(s.dtype) / 16);
   const int C = s.n_sink + s.n_recent;
   const long long total = (long long)C * vec_per_row;
@@ -127,7 +131,8 @@ cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const Lay
   if (bx > 64) bx = 64;
   dim3 grid(bx, s.batch * s.n_kv_heads, s.n_layers);
   stream_init_kernel<<<grid, threads, 0, st>>>(mask, kf, vf, seq_lens, ks, vs, s.batch, s.n_kv_heads, vec_per_row,
-                                               s.n_sink, s.n_recent, s.full_capacity, dev_err);
+                                               s.n_sink, s.n_recent, s.full_capacity,
+                                               s.per_sequence_mask ? s.n_layers : 0, only_layer, dev_err);
   return cudaGetLastError();
 }
 

@@ -34,13 +34,13 @@ __device__ __forceinline__ int ring_slot_of(int p, int S, int R) { return p < S 
 
 // Shared-memory footprint of the work list (bytes) for `entries` (layer, b) pairs.
 __host__ __device__ inline int worklist_smem_bytes(int entries, int batch) {
-  return ((entries + 1 + batch) * 4 + 128 + 15) / 16 * 16;
+  return ((entries + 1 + batch) * 4 + entries + 15) / 16 * 16;
 }
 
 struct WorkList {
   int* prefix;    // [entries + 1]
   int* seq;       // [batch]   seq_lens as read at kernel start
-  uint8_t* kind;  // [layer_count]  bit 0 lazy, bit 1 table entry missing
+  uint8_t* kind;  // [entries]  bit 0 lazy, bit 1 table entry missing
   int entries;
 
   __device__ __forceinline__ void carve(uint8_t* mem, int layer_count, int batch) {
@@ -51,9 +51,9 @@ struct WorkList {
   }
 
   // visible keys of (layer kind, batch row) after clamping; raises the error bits
-  __device__ __forceinline__ int visible(const DecodeArgs& a, int lr, int b, bool report) const {
+  __device__ __forceinline__ int visible(const DecodeArgs& a, int e, int b, bool report) const {
     const lt_shape& s = a.s;
-    const bool lazy = kind[lr] & 1;
+    const bool lazy = kind[e] & 1;
     const int rows = lazy ? s.n_sink + s.n_recent : s.full_capacity;
     int n = seq[b] + (a.fused ? 1 : 0);
     if (n < 0) n = 0;
@@ -70,11 +70,12 @@ struct WorkList {
     const lt_shape& s = a.s;
     const int B = s.batch;
     for (int b = threadIdx.x; b < B; b += blockDim.x) seq[b] = a.seq_lens[b];
-    for (int lr = threadIdx.x; lr < a.layer_count; lr += blockDim.x) {
+    for (int e = threadIdx.x; e < entries; e += blockDim.x) {
+      const int lr = e / B, b = e - lr * B;
       const int l = a.layer_begin + lr;
-      const bool lazy = a.mask[l] != 0;
+      const bool lazy = a.mask[mask_index(s, l, b)] != 0;
       const bool missing = lazy ? (!ks.p[l] || !vs.p[l]) : (!kf.p[l] || !vf.p[l]);
-      kind[lr] = (lazy ? 1 : 0) | (missing ? 2 : 0);
+      kind[e] = (lazy ? 1 : 0) | (missing ? 2 : 0);
       if (missing && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_NULL_LAYER);
     }
     __syncthreads();
@@ -85,8 +86,8 @@ struct WorkList {
     for (int e = e0; e < e1; ++e) {
       const int lr = e / B, b = e - lr * B;
       int items = 0;
-      if (!(kind[lr] & 2)) {
-        const int n = visible(a, lr, b, blockIdx.x == 0);
+      if (!(kind[e] & 2)) {
+        const int n = visible(a, e, b, blockIdx.x == 0);
         const int nc = max(1, (n + a.chunk_keys - 1) / a.chunk_keys);
         items = s.n_kv_heads * nc;
       }
@@ -128,9 +129,9 @@ struct WorkList {
     const int lr = lo / s.batch;
     w.b = lo - lr * s.batch;
     w.l = a.layer_begin + lr;
-    w.lazy = kind[lr] & 1;
+    w.lazy = kind[lo] & 1;
     w.rows = w.lazy ? s.n_sink + s.n_recent : s.full_capacity;
-    w.n = visible(a, lr, w.b, false);
+    w.n = visible(a, lo, w.b, false);
     w.nc = max(1, (w.n + a.chunk_keys - 1) / a.chunk_keys);
     const int rem = idx - prefix[lo];
     w.h = rem / w.nc;

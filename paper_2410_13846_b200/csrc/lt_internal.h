@@ -43,6 +43,10 @@ struct ScorePlan {
 };
 ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only);
 
+// Index of (layer l, batch row b) in layer_mask.
+__host__ __device__ inline int mask_index(const lt_shape& s, int l, int b) {
+  return s.per_sequence_mask ? b * s.n_layers + l : l;
+}
 inline float resolved_scale(const lt_shape& s) {
   return s.softmax_scale > 0.f ? s.softmax_scale : 1.0f / sqrtf((float)s.head_dim);
 }
@@ -59,7 +63,7 @@ cudaError_t launch_append(const lt_shape& s, const uint8_t* mask, const void* k_
 
 cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const LayerTable& kf,
                                const LayerTable& vf, const int32_t* seq_lens, const LayerTable& ks,
-                               const LayerTable& vs, uint32_t* dev_err, cudaStream_t st);
+                               const LayerTable& vs, const int32_t* only_layer, uint32_t* dev_err, cudaStream_t st);
 
 // One decode step (or the attention half of it).  `fused` = the step appends
 // k_new / v_new itself: the visible length is seq_lens[b] + 1 and the item that
@@ -127,7 +131,7 @@ __host__ __device__ inline void score_split_range(const ScoreArgs& a, int sp, in
     }
     sp -= 1;
   }
-  int w0 = a.n_ctx - a.s.n_recent;
+  int w0 = a.n_ctx - a.s.n_recent - (a.s.recent_per_row ? a.w_last - 1 : 0);  // first key any tail row keeps
   if (w0 < S) w0 = S;
   *k0 = w0 + sp * a.split_len;
   if (*k0 > a.n_ctx) *k0 = a.n_ctx;
@@ -141,5 +145,10 @@ cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st);
 
 cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask,
                           float* ratio, cudaStream_t st);
+
+cudaError_t launch_select_per_seq(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,
+                                  cudaStream_t st);
+cudaError_t launch_select_push(const float* scores_l, int layer, int L, int per_layer, int n_full, double* state,
+                               uint8_t* mask, int32_t* popped, cudaStream_t st);
 
 }  // namespace lt

@@ -42,6 +42,7 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
   score_split_range(a, sp, &j0, &j1);
   j1 = min(i + 1, j1);
   const T* Kb = (const T*)kf.p[l] + ((long long)(b * s.n_kv_heads + h) * s.full_capacity) * D;
+  const int win_lo = s.recent_per_row ? i - s.n_recent + 1 : a.n_ctx - s.n_recent;  // first recent key of this row
   float M = -INFINITY, A = 0.f, W = 0.f;
   for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
     const T* kr = Kb + (long long)j * D;
@@ -52,7 +53,7 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
     const float Mn = fmaxf(M, tj);
     const float corr = exp2f(M - Mn), p = exp2f(tj - Mn);
     A = A * corr + p;
-    W = W * corr + ((j < s.n_sink || j >= a.n_ctx - s.n_recent) ? p : 0.f);
+    W = W * corr + ((j < s.n_sink || j >= win_lo) ? p : 0.f);
     M = Mn;
   }
   red[0][threadIdx.x] = M;
@@ -148,6 +149,75 @@ __global__ void select_kernel(const float* __restrict__ scores, int L, int per_l
     mask[l] = rank < n_lazy ? 1 : 0;
     if (ratio) ratio[l] = (float)r[l];
   }
+}
+
+// Per-prompt selection: block b ranks the layers by the mean over the query
+// heads of scores[l][b][:] (same total order as select_kernel).
+__global__ void select_per_seq_kernel(const float* __restrict__ scores, int L, int B, int Hq, int n_lazy,
+                                      uint8_t* __restrict__ mask, float* __restrict__ ratio) {
+  __shared__ double r[LT_MAX_LAYERS];
+  const int l = threadIdx.x, b = blockIdx.x;
+  if (l < L) {
+    double acc = 0.0;
+    const float* p = scores + ((long long)l * B + b) * Hq;
+    for (int k = 0; k < Hq; ++k) acc += (double)p[k];
+    r[l] = acc / (double)Hq;
+  }
+  __syncthreads();
+  if (l < L) {
+    int rank = 0;
+    for (int m = 0; m < L; ++m) rank += (r[m] > r[l]) || (r[m] == r[l] && m < l);
+    mask[(long long)b * L + l] = rank < n_lazy ? 1 : 0;
+    if (ratio) ratio[(long long)b * L + l] = (float)r[l];
+  }
+}
+
+cudaError_t launch_select_per_seq(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,
+                                  cudaStream_t st) {
+  select_per_seq_kernel<<<B, LT_MAX_LAYERS, 0, st>>>(scores, L, B, Hq, n_lazy, mask, ratio);
+  return cudaGetLastError();
+}
+
+// One arrival at the priority queue of Figure 3.  The queue is "the layers
+// 0..layer whose mask is still 0"; state[l] holds their ratios (double).  When
+// more than n_full layers are queued, the one with the highest ratio (lower
+// index on ties) leaves: mask = 1, *popped = its index.
+__global__ void select_push_kernel(const float* __restrict__ scores_l, int layer, int L, int per_layer, int n_full,
+                                   double* __restrict__ state, uint8_t* __restrict__ mask,
+                                   int32_t* __restrict__ popped) {
+  __shared__ double r[LT_MAX_LAYERS];
+  __shared__ uint8_t queued[LT_MAX_LAYERS];
+  const int t = threadIdx.x;
+  if (layer == 0 && t < L) mask[t] = 0;  // a new prompt: empty queue, nothing lazy yet
+  if (t == 0) {
+    double acc = 0.0;
+    for (int k = 0; k < per_layer; ++k) acc += (double)scores_l[k];
+    state[layer] = acc / (double)per_layer;
+  }
+  __syncthreads();
+  const bool in_queue = t <= layer && mask[t] == 0;
+  queued[t] = in_queue ? 1 : 0;
+  r[t] = (t <= layer) ? state[t] : 0.0;
+  const int count = __syncthreads_count(in_queue);
+  if (count <= n_full) {
+    if (t == 0 && popped) *popped = -1;
+    return;
+  }
+  if (in_queue) {
+    int beaten_by = 0;
+    for (int m = 0; m <= layer; ++m)
+      if (queued[m]) beaten_by += (r[m] > r[t]) || (r[m] == r[t] && m < t);
+    if (beaten_by == 0) {
+      mask[t] = 1;
+      if (popped) *popped = t;
+    }
+  }
+}
+
+cudaError_t launch_select_push(const float* scores_l, int layer, int L, int per_layer, int n_full, double* state,
+                               uint8_t* mask, int32_t* popped, cudaStream_t st) {
+  select_push_kernel<<<1, LT_MAX_LAYERS, 0, st>>>(scores_l, layer, L, per_layer, n_full, state, mask, popped);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,

@@ -335,7 +335,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     const bool row_valid = r_local < rows_here;
     const int vis = n_ctx - T + (r % T);  // last visible key of this row
     const float cs = a.cs;
-    const int S = s.n_sink, win_lo = n_ctx - s.n_recent;
+    const int S = s.n_sink;
+    const int win_lo = s.recent_per_row ? vis - s.n_recent + 1 : n_ctx - s.n_recent;  // first recent key of this row
     const int lim = min(vis, k1 - 1);     // last key of this split that the row may see
     float m = -INFINITY, sA = 0.f, sWn = 0.f;
     const bool active = mb < n_mb;
