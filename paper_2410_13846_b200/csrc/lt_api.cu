@@ -28,14 +28,19 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   const int64_t n_max = (int64_t)((s.full_capacity > s.n_sink + s.n_recent) ? s.full_capacity
                                                                             : s.n_sink + s.n_recent);
   const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
-  const int64_t target = 148 * 4;  // a few CTAs per SM even for small stacks
-  int ck = 2048;
-  while (ck > 256 && units * ((n_max + ck - 1) / ck) < target) ck /= 2;
-  p.chunk_keys = ck;
-  p.n_chunks_max = (int)((n_max + ck - 1) / ck);
+  // Measured on B200 (32K context, whole stack and one layer per call): long chunks win, per-item
+  // hand-off costs more than an uneven last round; shorter chunks only pay when a launch has very few keys.
+  p.min_chunk = 512;
+  p.max_chunk = 2048;
+  p.target_items = 592;
+  // chunk = clamp(ceil(keys / target), min, max) gives at most target + units items
+  // when it is not clamped at max, and units * ceil(n_max / max) when it is
+  int64_t cap = units * ((n_max + p.max_chunk - 1) / p.max_chunk) + p.target_items + units;
+  if (cap > (int64_t)0x7fffffff) cap = 0x7fffffff;
+  p.items_cap = (int)cap;
   const int G = s.n_q_heads / s.n_kv_heads;
-  p.ml_floats = (size_t)units * p.n_chunks_max * G * 2;
-  p.o_floats = (size_t)units * p.n_chunks_max * G * s.head_dim;
+  p.ml_floats = (size_t)cap * G * 2;
+  p.o_floats = (size_t)cap * G * s.head_dim;
   return p;
 }
 
@@ -78,7 +83,7 @@ int persistent_grid(const DecodeArgs& a, int ctas_per_sm) {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
     sm_count[dev] = n;
   }
-  const long long most = (long long)a.layer_count * a.s.batch * a.s.n_kv_heads * a.n_chunks_max;
+  const long long most = a.items_cap;
   long long grid = (long long)sm_count[dev] * ctas_per_sm;
   if (grid > most) grid = most;
   return (int)(grid < 1 ? 1 : grid);
@@ -342,8 +347,10 @@ static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k
   a.seq_lens_rw = seq_lens;
   a.out = out;
   a.out_dtype = out_dtype;
-  a.chunk_keys = dp.chunk_keys;
-  a.n_chunks_max = dp.n_chunks_max;
+  a.min_chunk = dp.min_chunk;
+  a.max_chunk = dp.max_chunk;
+  a.target_items = dp.target_items;
+  a.items_cap = dp.items_cap;
   a.fused = fused;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
   a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;

@@ -11,7 +11,10 @@
 //   entry e = (layer, batch row)      n_e = visible keys, nc_e = chunks
 //   items of e = n_kv_heads * nc_e    item -> (kv head, chunk)
 // The prefix sum over entries lives in shared memory; an item index is turned
-// into (entry, kv head, chunk) by binary search.
+// into (entry, kv head, chunk) by binary search.  The chunk length is chosen on
+// the device from the total number of keys of the launch, so that a whole stack
+// (2048-key chunks) and a single layer (shorter chunks) both give every CTA
+// several items; the partials of item i live in slot i of the workspace.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -27,6 +30,7 @@ struct WorkItem {
   int j0, j1;      // key rows [j0, j1) of this chunk
   int rows;        // rows per (b, kv head) of the cache that is read
   int new_row;     // fused append: row taken from k_new / v_new (and stored) by this item, else -1
+  int slot0;       // partial slot of chunk 0 of this (layer, b, kv head); chunk c uses slot0 + c
   bool lazy;
 };
 
@@ -42,6 +46,7 @@ struct WorkList {
   int* seq;       // [batch]   seq_lens as read at kernel start
   uint8_t* kind;  // [entries]  bit 0 lazy, bit 1 table entry missing
   int entries;
+  int chunk;      // keys per chunk of this launch (before balancing)
 
   __device__ __forceinline__ void carve(uint8_t* mem, int layer_count, int batch) {
     entries = layer_count * batch;
@@ -79,16 +84,34 @@ struct WorkList {
       if (missing && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_NULL_LAYER);
     }
     __syncthreads();
-    // items per entry, then an exclusive scan: thread t owns a contiguous run of entries
+    // thread t owns a contiguous run of entries
     const int per = (entries + blockDim.x - 1) / blockDim.x;
     const int e0 = min(entries, (int)threadIdx.x * per), e1 = min(entries, e0 + per);
+    // chunk length: total keys of the launch spread over a few items per CTA
+    __shared__ unsigned long long total_keys;
+    if (threadIdx.x == 0) total_keys = 0ull;
+    __syncthreads();
+    {
+      unsigned long long mine = 0ull;
+      for (int e = e0; e < e1; ++e)
+        if (!(kind[e] & 2)) mine += (unsigned long long)visible(a, e, e % B, blockIdx.x == 0) * s.n_kv_heads;
+      if (mine) atomicAdd(&total_keys, mine);
+    }
+    __syncthreads();
+    {
+      const long long target = min((long long)gridDim.x * 8, (long long)a.target_items);
+      long long c = (long long)((total_keys + target - 1) / target);
+      c = (c + 63) / 64 * 64;
+      chunk = (int)max((long long)a.min_chunk, min((long long)a.max_chunk, c));
+    }
+    // items per entry, then an exclusive scan
     int run = 0;
     for (int e = e0; e < e1; ++e) {
-      const int lr = e / B, b = e - lr * B;
+      const int b = e % B;
       int items = 0;
       if (!(kind[e] & 2)) {
-        const int n = visible(a, e, b, blockIdx.x == 0);
-        const int nc = max(1, (n + a.chunk_keys - 1) / a.chunk_keys);
+        const int n = visible(a, e, b, false);
+        const int nc = max(1, (n + chunk - 1) / chunk);
         items = s.n_kv_heads * nc;
       }
       prefix[e + 1] = items;  // turned into the prefix below
@@ -115,7 +138,16 @@ struct WorkList {
     __syncthreads();
   }
 
-  __device__ __forceinline__ int total() const { return prefix[entries]; }
+  // Items of the launch; never more than the partial slots the workspace holds
+  // (the plan's bound covers every chunk length this build can choose).
+  __device__ __forceinline__ int total(const DecodeArgs& a) const {
+    const int t = prefix[entries];
+    if (t > a.items_cap) {
+      if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(a.dev_err, LT_DEVERR_LEN_CLAMPED);
+      return a.items_cap;
+    }
+    return t;
+  }
 
   __device__ __forceinline__ WorkItem item(const DecodeArgs& a, int idx) const {
     const lt_shape& s = a.s;
@@ -132,10 +164,11 @@ struct WorkList {
     w.lazy = kind[lo] & 1;
     w.rows = w.lazy ? s.n_sink + s.n_recent : s.full_capacity;
     w.n = visible(a, lo, w.b, false);
-    w.nc = max(1, (w.n + a.chunk_keys - 1) / a.chunk_keys);
+    w.nc = max(1, (w.n + chunk - 1) / chunk);
     const int rem = idx - prefix[lo];
     w.h = rem / w.nc;
     w.c = rem - w.h * w.nc;
+    w.slot0 = idx - w.c;
     const int len = (w.n + w.nc - 1) / w.nc;  // balanced chunks: no tiny last chunk
     w.j0 = min(w.n, w.c * len);
     w.j1 = min(w.n, w.j0 + len);
@@ -149,10 +182,8 @@ struct WorkList {
   }
 };
 
-// Index of the partials of (layer, b, kv head, chunk).
-__device__ __forceinline__ long long partial_unit(const DecodeArgs& a, const WorkItem& w) {
-  return ((((long long)w.l * a.s.batch + w.b) * a.s.n_kv_heads + w.h) * a.n_chunks_max) + w.c;
-}
+// Slot of the partials of (layer, b, kv head, chunk): the item's own index.
+__device__ __forceinline__ long long partial_unit(const DecodeArgs&, const WorkItem& w) { return w.slot0 + w.c; }
 
 // Staging buffer (shared memory) for the (max, sum) pairs of a unit's chunks
 // while they are merged; units with more pairs read them from global memory.
@@ -190,8 +221,7 @@ __device__ __forceinline__ bool count_item_in(const DecodeArgs& a, const WorkIte
 __device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem& w, float2* s_ml) {
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads, D = s.head_dim;
-  const long long unit = ((long long)w.l * s.batch + w.b) * s.n_kv_heads + w.h;
-  const long long unit0 = unit * a.n_chunks_max;
+  const long long unit0 = w.slot0;
   const int pairs = w.nc * G;
   const bool staged = pairs <= kCombineStagePairs;
   const float2* ml_g = reinterpret_cast<const float2*>(a.part_ml) + unit0 * G;  // [c][g]

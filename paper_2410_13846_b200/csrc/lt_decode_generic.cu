@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a, Layer
   WorkList wl;
   wl.carve(smem, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
-  const int n_items = wl.total();
+  const int n_items = wl.total(a);
   const float cs = a.cs;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 

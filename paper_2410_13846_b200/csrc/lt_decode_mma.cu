@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   WorkList wl;
   wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
-  const int n_items = wl.total();
+  const int n_items = wl.total(a);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
@@ -473,12 +473,22 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
   static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
   auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, WARPS * 32, smem);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  // attribute and occupancy are looked up once per shared-memory size (host time matters for per-layer callers)
+  static int cached_smem_of[64], cached_per_sm_of[64];  // per device; zero = not looked up yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  int& cached_smem = cached_smem_of[dev];
+  int& cached_per_sm = cached_per_sm_of[dev];
+  int per_sm = cached_per_sm;
+  if (smem != cached_smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, WARPS * 32, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    cached_smem = smem;
+    cached_per_sm = per_sm;
+  }
   const int grid = persistent_grid(a, per_sm);
   kern<<<grid, WARPS * 32, smem, st>>>(a, kf, vf, ks, vs);
   return cudaGetLastError();

@@ -26,10 +26,11 @@ size_t ws_prefix_bytes(const lt_shape& s);
 // Split-KV plan of the decode step; a function of the shape alone so that the
 // workspace query and every later call agree.
 struct DecodePlan {
-  int chunk_keys;    // keys per KV chunk (multiple of 64)
-  int n_chunks_max;  // chunks that cover max(full_capacity, n_sink + n_recent)
-  size_t ml_floats;  // [L][B][Hkv][n_chunks_max][G][2]
-  size_t o_floats;   // [L][B][Hkv][n_chunks_max][G][D]
+  int min_chunk, max_chunk;  // the kernels pick the chunk length of a launch in this range (multiples of 64)
+  int target_items;          // items a launch aims for when its keys allow (a few per CTA)
+  int items_cap;             // most items (= partial slots) any launch over this shape can have
+  size_t ml_floats;          // [items_cap][G][2]
+  size_t o_floats;           // [items_cap][G][D]
 };
 DecodePlan make_decode_plan(const lt_shape& s);
 
@@ -79,7 +80,7 @@ struct DecodeArgs {
   void* out;
   int out_dtype;
   int layer_begin, layer_count;
-  int chunk_keys, n_chunks_max;
+  int min_chunk, max_chunk, target_items, items_cap;
   int fused, advance;
   float cs;  // softmax scale * log2(e)
   float* part_ml;
