@@ -64,6 +64,8 @@ CONFIGS = {
     "qwq32b_longgen": Config("qwq32b_longgen", 64, 40, 8, 128, 4, 1024, 4, 4092, 64, 32, "bf16", 16384),
     # 5: Llama-3.1-8B-shaped, 128K context
     "llama31_8b_128k": Config("llama31_8b_128k", 32, 32, 8, 128, 2, 131072, 4, 4092, 64, 16, "bf16", 128),
+    # 6: Llama-3-70B-shaped (80 layers, GQA group 8), 16K context
+    "llama3_70b_16k": Config("llama3_70b_16k", 80, 64, 8, 128, 2, 16384, 4, 2044, 64, 40, "bf16", 128),
 }
 
 

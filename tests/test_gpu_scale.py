@@ -1,7 +1,9 @@
 """GPU parity at the full sizes of the other workloads, on sampled units:
 the Llama-2-7B-shaped MHA stack (G = 1), the QwQ-32B-shaped long generation
 (G = 5, 16384 appended tokens, rings wrap four times) and the Llama-3.1-8B-shaped
-128K stack with the lazy fraction swept over 0 / 25 / 50 / 75 %."""
+128K stack with the lazy fraction swept over 0 / 25 / 50 / 75 %, and the
+Llama-3-70B-shaped stack (80 layers, G = 8) with batch rows of different lengths
+through the fused decode step."""
 import numpy as np
 import pytest
 import torch
@@ -163,3 +165,49 @@ def test_llama31_8b_128k_lazy_fraction_sweep():
             units.append((int(np.nonzero(mask)[0][0]), 1, 7))
         units.append((int(np.nonzero(mask == 0)[0][-1]), 0, 2))
         _check_units(st, cfg, mask, q, out, [k], [v], units)
+
+
+def test_llama3_70b_gqa8_ragged_rows_fused_steps():
+    """80 layers, 64 query / 8 kv heads: 512 query rows per scoring unit (two row
+    blocks), group of 8 in the decode kernel; after identification the two batch
+    rows continue from different lengths."""
+    _need_gb(30)
+    cfg = CONFIGS["llama3_70b_16k"]
+    L, B, Hkv, G, n0 = cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.group, cfg.n_ctx
+    steps = 3
+    st, q_tail, planted = build_stack(cfg, steps)
+    g = np.random.default_rng(61)
+    sc = f64(_score_select(st, q_tail, cfg, cfg.n_lazy))
+    _check_scores(st, q_tail, cfg, sc, g, 4)
+    mask = st.mask.cpu().numpy()
+    assert sorted(np.nonzero(mask)[0].tolist()) == planted
+    assert np.array_equal(mask, O.select_lazy(sc, cfg.n_lazy)[0])
+    lens = [n0, 9001]                                            # row 1 is a shorter prompt
+    st.set_seq_lens(lens)
+    lt.stream_init(st.shape, st.mask, st.tables, st.seq_lens, ws=st.ws)
+    out = torch.zeros((L, B, cfg.n_q_heads, 128), dtype=torch.float32, device="cuda")
+    new_k, new_v = [], []
+    for step in range(steps):
+        q, k, v = decode_inputs(cfg, step, "cuda")
+        new_k.append(k); new_v.append(v)
+        lt.decode_step(st.shape, q, k, v, st.tables, st.mask, st.seq_lens, out, st.ws)
+    assert lt.check(st.ws) == 0 and st.seq_lens.cpu().tolist() == [x + steps for x in lens]
+    lazy, full = np.nonzero(mask)[0], np.nonzero(mask == 0)[0]
+    units = [(int(full[0]), 0, 0), (int(full[-1]), 1, 7), (int(lazy[0]), 1, 1), (int(lazy[-1]), 0, 6)]
+    units += [(int(g.integers(L)), int(g.integers(B)), int(g.integers(Hkv))) for _ in range(4)]
+    for l, b, h in units:
+        nb = lens[b]
+        kb = torch.stack([x[l, b, h] for x in new_k]); vb = torch.stack([x[l, b, h] for x in new_v])
+        # row 1's appended tokens overwrote prompt rows nb.. of a full layer's cache; a lazy layer's full cache still holds the prompt
+        K = np.concatenate([f64(st.k_full[l][b, h, :nb]), f64(kb)])[None]
+        V = np.concatenate([f64(st.v_full[l][b, h, :nb]), f64(vb)])[None]
+        qh = f64(q[l, b, h * G:(h + 1) * G])
+        ref = O.streaming_attention(qh, K, V, cfg.n_sink, cfg.n_recent) if mask[l] else O.full_attention(qh, K, V)
+        mx, rel = attn_errors(f64(out[l, b, h * G:(h + 1) * G]), ref)
+        assert mx <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (l, b, h, mx, rel)
+        hist = np.concatenate([bits(st.k_full[l][b, h, :nb]), bits(kb)])
+        if mask[l]:
+            ek, _ = O.stream_cache_after(hist, cfg.n_sink, cfg.n_recent)
+            assert np.array_equal(bits(st.k_stream[l][b, h]), ek)
+        else:
+            assert np.array_equal(bits(st.k_full[l][b, h, nb:nb + steps]), bits(kb))
