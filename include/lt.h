@@ -25,6 +25,7 @@
  *     mask selects is skipped and reported through the error word.
  *   - Layouts are dense row-major, last index fastest:
  *       full cache of one layer    [batch][n_kv_heads][full_capacity][head_dim]
+ *                                  (or a page pool, see lt_shape.page_size)
  *       stream cache of one layer  [batch][n_kv_heads][n_sink+n_recent][head_dim]
  *     Every cache pointer must be 16-byte aligned.
  *   - layer_mask is uint8[n_layers] on the device, 1 = lazy (streaming); with
@@ -83,6 +84,17 @@ typedef struct lt_shape {
   int32_t recent_per_row;    /* scoring only.  0: X_recent is the fixed block of the last n_recent prompt
                                 positions (Table 1, the set a lazy layer retains); 1: the recent set of the
                                 tail query at position i is i - n_recent + 1 .. i (Appendix E, M_lazy row by row) */
+  /* Paged full caches (block tables, as serving engines keep them).  page_size = 0: contiguous caches as
+     described above.  page_size > 0 (a multiple of 128): the full cache of a layer is a pool
+     [n_pages][n_kv_heads][page_size][head_dim]; token j of batch row b lives in page
+     block_table[b][j / page_size] at row j % page_size, and full_capacity must equal
+     pages_per_seq * page_size.  One table serves every layer (each layer has its own pool of the same
+     geometry).  Stream caches are constant-size and stay contiguous. */
+  int32_t page_size;
+  int32_t pages_per_seq;       /* columns of block_table */
+  int32_t n_pages;             /* pages in every layer's pool */
+  int32_t reserved_;           /* keep the pointer 8-byte aligned; must be 0 */
+  const int32_t* block_table;  /* dev int32 [batch][pages_per_seq], entries in [0, n_pages); read during device work */
 } lt_shape;
 
 /* Text for a status code (static storage, never NULL). */

@@ -26,7 +26,9 @@ class _CShape(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_sink", "n_recent",
                  "full_capacity", "dtype")] + [("softmax_scale", C.c_float), ("per_sequence_mask", C.c_int32),
-                                                ("recent_per_row", C.c_int32)]
+                                                ("recent_per_row", C.c_int32), ("page_size", C.c_int32),
+                                                ("pages_per_seq", C.c_int32), ("n_pages", C.c_int32),
+                                                ("reserved_", C.c_int32), ("block_table", C.c_void_p)]
 
 
 @dataclass
@@ -43,11 +45,21 @@ class Shape:
     softmax_scale: float = 0.0
     per_sequence_mask: int = 0
     recent_per_row: int = 0
+    page_size: int = 0           # > 0: paged full caches (see lt_shape in include/lt.h)
+    pages_per_seq: int = 0
+    n_pages: int = 0
+    block_table: object = None   # int32 CUDA tensor [batch][pages_per_seq]
 
     def c(self) -> _CShape:
+        bt = None
+        if self.block_table is not None:
+            t = self.block_table
+            if not (t.is_cuda and t.is_contiguous() and t.element_size() == 4):
+                raise ValueError("block_table must be a contiguous int32 CUDA tensor")
+            bt = t.data_ptr()
         return _CShape(self.n_layers, self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_sink,
                        self.n_recent, self.full_capacity, self.dtype, self.softmax_scale, self.per_sequence_mask,
-                       self.recent_per_row)
+                       self.recent_per_row, self.page_size, self.pages_per_seq, self.n_pages, 0, bt)
 
     @property
     def stream_capacity(self) -> int:

@@ -20,6 +20,13 @@ lt_status validate_shape(const lt_shape* s) {
   if (s->dtype != LT_F32 && s->dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
   if (!(s->softmax_scale == s->softmax_scale)) return LT_ERR_INVALID_ARG;  // NaN
   if ((s->per_sequence_mask | s->recent_per_row) & ~1) return LT_ERR_INVALID_ARG;
+  if (s->page_size < 0 || s->reserved_ != 0) return LT_ERR_INVALID_ARG;
+  if (s->page_size > 0) {
+    if (s->page_size % 128 != 0) return LT_ERR_UNSUPPORTED;
+    if (s->pages_per_seq < 1 || s->n_pages < 1 || !s->block_table) return LT_ERR_INVALID_ARG;
+    if ((int64_t)s->pages_per_seq * s->page_size != s->full_capacity) return LT_ERR_INVALID_ARG;
+    if ((int64_t)s->n_pages * s->n_kv_heads * s->page_size >= (1ll << 31)) return LT_ERR_UNSUPPORTED;
+  }
   return LT_OK;
 }
 

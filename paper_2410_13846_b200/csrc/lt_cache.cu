@@ -8,12 +8,11 @@ namespace lt {
 __device__ __forceinline__ int ring_slot_dev(int p, int S, int R) { return p < S ? p : S + (p - S) % R; }
 
 // One thread per 16-byte vector of one (layer, b, kv head) row of k_new / v_new.
-__global__ void append_kernel(const uint8_t* __restrict__ mask, const uint4* __restrict__ k_new,
+__global__ void append_kernel(lt_shape s, const uint8_t* __restrict__ mask, const uint4* __restrict__ k_new,
                               const uint4* __restrict__ v_new, const int32_t* __restrict__ seq_lens,
                               LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs, int layer_begin,
-                              int layer_count, int B, int Hkv, int vec_per_row, int S, int R, int cap,
-                              int mask_row /* layers per mask row, 0 = one mask for the batch */,
-                              uint32_t* dev_err) {
+                              int layer_count, int vec_per_row, uint32_t* dev_err) {
+  const int B = s.batch, Hkv = s.n_kv_heads, S = s.n_sink, R = s.n_recent;
   const long long total = (long long)layer_count * B * Hkv * vec_per_row;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
@@ -23,27 +22,22 @@ __global__ void append_kernel(const uint8_t* __restrict__ mask, const uint4* __r
   const int b = (int)((row / Hkv) % B);
   const int l = layer_begin + (int)(row / ((long long)Hkv * B));
   const int pos = seq_lens[b];
-  const bool lazy = mask[b * mask_row + l] != 0;
+  const bool lazy = mask[mask_index(s, l, b)] != 0;
   uint4* kdst = (uint4*)(lazy ? ks.p[l] : kf.p[l]);
   uint4* vdst = (uint4*)(lazy ? vs.p[l] : vf.p[l]);
   if (!kdst || !vdst) {
     if (dev_err && v == 0) atomicOr(dev_err, LT_DEVERR_NULL_LAYER);
     return;
   }
-  int slot, rows;
-  if (lazy) {
-    slot = ring_slot_dev(pos, S, R);
-    rows = S + R;
-  } else {
-    slot = pos;
-    rows = cap;
-  }
+  const int slot = lazy ? ring_slot_dev(pos, S, R) : pos;
+  const int rows = lazy ? S + R : s.full_capacity;
   if (pos < 0 || slot >= rows) {
     if (dev_err && v == 0) atomicOr(dev_err, LT_DEVERR_POS_OUT_OF_RANGE);
     return;
   }
   const long long src = ((long long)(l * B + b) * Hkv + h) * vec_per_row + v;
-  const long long dst = (((long long)b * Hkv + h) * rows + slot) * vec_per_row + v;
+  const long long drow = lazy ? ((long long)b * Hkv + h) * rows + slot : full_cache_row(s, b, h, slot);
+  const long long dst = drow * vec_per_row + v;
   kdst[dst] = k_new[src];
   vdst[dst] = v_new[src];
 }
@@ -60,11 +54,8 @@ cudaError_t launch_append(const lt_shape& s, const uint8_t* mask, const void* k_
   const long long total = (long long)layer_count * s.batch * s.n_kv_heads * vec_per_row;
   const int threads = 256;
   const long long blocks = (total + threads - 1) / threads;
-  // k_new / v_new are indexed by absolute layer: shift the base so that layer_begin lands at its row
-  append_kernel<<<(unsigned)blocks, threads, 0, st>>>(mask, (const uint4*)k_new, (const uint4*)v_new, seq_lens, kf, vf,
-                                                      ks, vs, layer_begin, layer_count, s.batch, s.n_kv_heads,
-                                                      vec_per_row, s.n_sink, s.n_recent, s.full_capacity,
-                                                      s.per_sequence_mask ? s.n_layers : 0, dev_err);
+  append_kernel<<<(unsigned)blocks, threads, 0, st>>>(s, mask, (const uint4*)k_new, (const uint4*)v_new, seq_lens, kf,
+                                                      vf, ks, vs, layer_begin, layer_count, vec_per_row, dev_err);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (advance) {
@@ -76,15 +67,15 @@ cudaError_t launch_append(const lt_shape& s, const uint8_t* mask, const void* k_
 
 // Gather by destination slot: slot s of the stream cache receives the prompt
 // row of the last position that maps to it, so no two threads write one row.
-__global__ void stream_init_kernel(const uint8_t* __restrict__ mask, LayerTable kf, LayerTable vf,
-                                   const int32_t* __restrict__ seq_lens, LayerTable ks, LayerTable vs, int B,
-                                   int Hkv, int vec_per_row, int S, int R, int cap, int mask_row,
-                                   const int32_t* __restrict__ only_layer, uint32_t* dev_err) {
+__global__ void stream_init_kernel(lt_shape s, const uint8_t* __restrict__ mask, LayerTable kf, LayerTable vf,
+                                   const int32_t* __restrict__ seq_lens, LayerTable ks, LayerTable vs,
+                                   int vec_per_row, const int32_t* __restrict__ only_layer, uint32_t* dev_err) {
+  const int Hkv = s.n_kv_heads, S = s.n_sink, R = s.n_recent, cap = s.full_capacity;
   const int l = blockIdx.z;
   const int bh = blockIdx.y;
-  const int b = bh / Hkv;
+  const int b = bh / Hkv, h = bh - b * Hkv;
   if (only_layer && *only_layer != l) return;  // compaction of the one layer named on the device
-  if (mask[b * mask_row + l] == 0) return;
+  if (mask[mask_index(s, l, b)] == 0) return;
   const int C = S + R;
   const uint4* ksrc = (const uint4*)kf.p[l];
   const uint4* vsrc = (const uint4*)vf.p[l];
@@ -113,7 +104,7 @@ __global__ void stream_init_kernel(const uint8_t* __restrict__ mask, LayerTable 
       if (last >= ri) p = S + last - ((last - ri) % R);
     }
     if (p < 0) continue;
-    const long long src = ((long long)bh * cap + p) * vec_per_row + v;
+    const long long src = full_cache_row(s, b, h, p) * vec_per_row + v;
     const long long dst = ((long long)bh * C + slot) * vec_per_row + v;
     kdst[dst] = ksrc[src];
     vdst[dst] = vsrc[src];
@@ -130,9 +121,7 @@ cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const Lay
   int bx = (int)((total + threads - 1) / threads);
   if (bx > 64) bx = 64;
   dim3 grid(bx, s.batch * s.n_kv_heads, s.n_layers);
-  stream_init_kernel<<<grid, threads, 0, st>>>(mask, kf, vf, seq_lens, ks, vs, s.batch, s.n_kv_heads, vec_per_row,
-                                               s.n_sink, s.n_recent, s.full_capacity,
-                                               s.per_sequence_mask ? s.n_layers : 0, only_layer, dev_err);
+  stream_init_kernel<<<grid, threads, 0, st>>>(s, mask, kf, vf, seq_lens, ks, vs, vec_per_row, only_layer, dev_err);
   return cudaGetLastError();
 }
 

@@ -45,16 +45,18 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a, Layer
     const WorkItem w = wl.item(a, item);
     const int l = w.l, b = w.b, h = w.h;
     const long long bh = (long long)b * s.n_kv_heads + h;
-    const T* Kb = (const T*)(w.lazy ? ks.p[l] : kf.p[l]) + bh * w.rows * D;
-    const T* Vb = (const T*)(w.lazy ? vs.p[l] : vf.p[l]) + bh * w.rows * D;
+    const T* Kl = (const T*)(w.lazy ? ks.p[l] : kf.p[l]);
+    const T* Vl = (const T*)(w.lazy ? vs.p[l] : vf.p[l]);
+    // element offset of cache row j of this (b, kv head): stream caches are contiguous, full caches may be paged
+    auto row_off = [&](int j) { return (w.lazy ? bh * w.rows + j : full_cache_row(s, b, h, j)) * D; };
     const T* k_new_row = nullptr;
     const T* v_new_row = nullptr;
     if (w.new_row >= 0) {
       const long long src = (((long long)l * s.batch + b) * s.n_kv_heads + h) * D;
       k_new_row = (const T*)a.k_new + src;
       v_new_row = (const T*)a.v_new + src;
-      T* kd = const_cast<T*>(Kb) + (long long)w.new_row * D;
-      T* vd = const_cast<T*>(Vb) + (long long)w.new_row * D;
+      T* kd = const_cast<T*>(Kl) + row_off(w.new_row);
+      T* vd = const_cast<T*>(Vl) + row_off(w.new_row);
       for (int d = threadIdx.x; d < D; d += blockDim.x) {
         kd[d] = k_new_row[d];
         vd[d] = v_new_row[d];
@@ -72,8 +74,9 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a, Layer
       }
       float M = -INFINITY, lsum = 0.f;
       for (int j = w.j0; j < w.j1; ++j) {
-        const T* kr = (j == w.new_row) ? k_new_row : Kb + (long long)j * D;
-        const T* vr = (j == w.new_row) ? v_new_row : Vb + (long long)j * D;
+        const long long ro = row_off(j);
+        const T* kr = (j == w.new_row) ? k_new_row : Kl + ro;
+        const T* vr = (j == w.new_row) ? v_new_row : Vl + ro;
         float part = 0.f;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) part += qr[e] * to_f32<T>(kr[lane * EPL + e]);

@@ -89,6 +89,7 @@ struct TileSrc {
   int j0, j1;                // key rows of the chunk
   int new_row;               // -1 when the chunk does not hold the new token
   int my_tiles;              // tiles of this warp (tiles warp, warp + WARPS, ... of the chunk)
+  int tbl_off;               // paged full cache: offset of this batch row's block-table row, else -1
 };
 
 // Shared memory: [rings: WARPS x NSTAGE x stage][merge: two 8 x 128 fp32 buffers,
@@ -128,9 +129,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   auto make_src = [&](const WorkItem& w) {
     TileSrc t;
-    const long long bh = (long long)w.b * s.n_kv_heads + w.h;
-    t.Kb = (const uint8_t*)(w.lazy ? ks.p[w.l] : kf.p[w.l]) + bh * w.rows * kRowBytes;
-    t.Vb = (const uint8_t*)(w.lazy ? vs.p[w.l] : vf.p[w.l]) + bh * w.rows * kRowBytes;
+    // contiguous: base of this (b, kv head); paged: base of kv head h inside page 0 of the layer's pool
+    const bool paged = !w.lazy && s.page_size > 0;
+    const long long base_row = paged ? (long long)w.h * s.page_size
+                                     : ((long long)w.b * s.n_kv_heads + w.h) * w.rows;
+    t.Kb = (const uint8_t*)(w.lazy ? ks.p[w.l] : kf.p[w.l]) + base_row * kRowBytes;
+    t.Vb = (const uint8_t*)(w.lazy ? vs.p[w.l] : vf.p[w.l]) + base_row * kRowBytes;
+    t.tbl_off = paged ? w.b * s.pages_per_seq : -1;
     t.j0 = w.j0;
     t.j1 = w.j1;
     t.new_row = w.new_row;
@@ -146,8 +151,15 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     return t;
   };
   // copy this warp's idx-th tile of `t` into ring stage `stage` (no commit)
+  // row of key `row` relative to t.Kb / t.Vb (a paged chunk starts on a multiple of 16, so a tile has one page)
+  auto cache_row = [&](const TileSrc& t, int row) -> long long {
+    if (t.tbl_off < 0) return row;
+    const int page = s.block_table[t.tbl_off + row / s.page_size];
+    return (long long)page * s.n_kv_heads * s.page_size + row % s.page_size;
+  };
   auto fetch_tile = [&](const TileSrc& t, int idx, int stage) {
     const int key_base = t.j0 + (warp + idx * WARPS) * TILE;
+    const long long tile_row = cache_row(t, key_base);
     const uint32_t st = wsm + stage * STAGE_BYTES;
 #pragma unroll
     for (int i = 0; i < TILE / 2; ++i) {
@@ -155,7 +167,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       const int p = lane & 15;
       const int row = key_base + r;
       const bool valid = row < t.j1;
-      const long long goff = (long long)(valid ? row : (t.j1 - 1)) * kRowBytes + p * 16;
+      const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
       const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
       const bool fresh = row == t.new_row;
       cp_async16(st + soff, fresh ? t.k_new_row + p * 16 : t.Kb + goff, valid ? 16 : 0);
@@ -204,7 +216,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     if (src_cur.new_row >= 0 && warp == 0) {
       const uint8_t* sp = (lane < 16 ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 15) * 16;
       uint8_t* dp = const_cast<uint8_t*>(lane < 16 ? src_cur.Kb : src_cur.Vb) +
-                    (long long)src_cur.new_row * kRowBytes + (lane & 15) * 16;
+                    cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane & 15) * 16;
       *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
     }
 

@@ -48,6 +48,13 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
 __host__ __device__ inline int mask_index(const lt_shape& s, int l, int b) {
   return s.per_sequence_mask ? b * s.n_layers + l : l;
 }
+// Row (in units of head_dim elements) of token j of (batch row b, kv head h) in a layer's full cache.
+// The block table is dereferenced on the device only.
+__device__ __forceinline__ long long full_cache_row(const lt_shape& s, int b, int h, int j) {
+  if (s.page_size <= 0) return ((long long)b * s.n_kv_heads + h) * s.full_capacity + j;
+  const int page = s.block_table[(long long)b * s.pages_per_seq + j / s.page_size];
+  return ((long long)page * s.n_kv_heads + h) * s.page_size + j % s.page_size;
+}
 inline float resolved_scale(const lt_shape& s) {
   return s.softmax_scale > 0.f ? s.softmax_scale : 1.0f / sqrtf((float)s.head_dim);
 }

@@ -41,11 +41,11 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
   int j0, j1;
   score_split_range(a, sp, &j0, &j1);
   j1 = min(i + 1, j1);
-  const T* Kb = (const T*)kf.p[l] + ((long long)(b * s.n_kv_heads + h) * s.full_capacity) * D;
+  const T* Kl = (const T*)kf.p[l];
   const int win_lo = s.recent_per_row ? i - s.n_recent + 1 : a.n_ctx - s.n_recent;  // first recent key of this row
   float M = -INFINITY, A = 0.f, W = 0.f;
   for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
-    const T* kr = Kb + (long long)j * D;
+    const T* kr = Kl + full_cache_row(s, b, h, j) * D;
     float dot = 0.f;
 #pragma unroll 8
     for (int d = 0; d < D; ++d) dot += qs[d] * ld_f32<T>(kr + d);

@@ -222,7 +222,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int n_ctx = a.n_ctx;
   int k0, k1;
   score_split_range(a, sp, &k0, &k1);
-  const int n_tiles = k1 > k0 ? (k1 - k0 + kBlockN - 1) / kBlockN : 0;
+  // Paged caches: tiles start on multiples of 128 keys so that none straddles two pages (the page size
+  // is a multiple of 128); the keys before k0 in the first tile are masked by the statistics warps.
+  const int ts0 = s.page_size > 0 ? (k0 & ~(kBlockN - 1)) : k0;
+  const int n_tiles = k1 > k0 ? (k1 - ts0 + kBlockN - 1) / kBlockN : 0;
   const int rows_here = min(kBlockM, M - rb * kBlockM);  // valid query rows of this CTA
   const int n_mb = (rows_here + 127) / 128;              // UMMA row blocks in use
 
@@ -264,7 +267,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int row0 = (b * s.n_kv_heads + h) * s.full_capacity;  // first cache row of this (b, kv head)
+  // tensor-map row of key j of this (b, kv head); j is a tile start
+  auto map_row = [&](int j) {
+    if (s.page_size <= 0) return (b * s.n_kv_heads + h) * s.full_capacity + j;
+    const int page = s.block_table[(long long)b * s.pages_per_seq + j / s.page_size];
+    return (page * s.n_kv_heads + h) * s.page_size + j % s.page_size;
+  };
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsLight));
@@ -283,8 +291,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         const uint32_t dst = sK + st * kStageBytes;
         const uint32_t bar = bar_full + 8 * st;
         mbar_expect_tx(bar, kStageBytes);
-        tma_load_2d(dst, map, 0, row0 + k0 + it * kBlockN, bar);
-        tma_load_2d(dst + kKHalfBytes, map, 64, row0 + k0 + it * kBlockN, bar);
+        const int y = map_row(ts0 + it * kBlockN);
+        tma_load_2d(dst, map, 0, y, bar);
+        tma_load_2d(dst + kKHalfBytes, map, 64, y, bar);
         issued = it + 1;
       }
       if (!ok) {
@@ -347,19 +356,19 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int jend = jb + 64;
       const bool all_win = (jend <= S) || (jb >= win_lo);
       const bool no_win = (jb >= S) && (jend <= win_lo);
-      if ((jend - 1 <= lim) && (all_win || no_win)) {
+      if ((jb >= k0) && (jend - 1 <= lim) && (all_win || no_win)) {
         const float mn = fmaxf(m, max64(v));
         const float corr = ex2((m - mn) * cs);
         const float ps = sum_ex2_64(v, cs, -mn * cs);
         sA = fmaf(sA, corr, ps);
         sWn = fmaf(sWn, corr, all_win ? ps : 0.f);
         m = mn;
-      } else if (jb <= lim) {
-        // boundary half (causal tail, split end or window edge): mask in place.
-        // 2^(-inf) = 0, and key jb is visible, so the maximum is finite.
+      } else if (max(jb, k0) <= min(jend - 1, lim)) {
+        // boundary half (split start, causal tail, split end or window edge): mask in place.
+        // 2^(-inf) = 0, and at least one key is visible, so the maximum is finite.
 #pragma unroll
         for (int i = 0; i < 64; ++i)
-          if (jb + i > lim) v[i] = 0xff800000u;
+          if (jb + i > lim || jb + i < k0) v[i] = 0xff800000u;
         const float mn = fmaxf(m, max64(v));
         const float corr = ex2((m - mn) * cs);
         const float off = -mn * cs;
@@ -388,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     for (int it = 0; it < n_tiles && ok; ++it) {
       const int t = it & 1;
-      const int kb = k0 + it * kBlockN;
+      const int kb = ts0 + it * kBlockN;
       const uint32_t taddr = lane_base + t * 256;
       // first half is (being) loaded; start the second half, then work on the first
       tmem_ld_wait();
@@ -437,7 +446,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 bool scores_umma_supported(const lt_shape& s, int /*w_last*/) {
   return s.dtype == LT_BF16 && s.head_dim == 128 &&
-         (long long)s.batch * s.n_kv_heads * s.full_capacity < (1ll << 31);
+         (long long)s.batch * s.n_kv_heads * s.full_capacity < (1ll << 31);  // tensor-map rows fit an int32 coordinate
 }
 
 namespace {
@@ -465,7 +474,9 @@ cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStr
   const int row_blocks = (M + kBlockM - 1) / kBlockM;
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return cudaErrorNotSupported;
-  const cuuint64_t gdim[2] = {(cuuint64_t)kD, (cuuint64_t)a.s.batch * a.s.n_kv_heads * a.s.full_capacity};
+  const cuuint64_t rows_total = a.s.page_size > 0 ? (cuuint64_t)a.s.n_pages * a.s.n_kv_heads * a.s.page_size
+                                                  : (cuuint64_t)a.s.batch * a.s.n_kv_heads * a.s.full_capacity;
+  const cuuint64_t gdim[2] = {(cuuint64_t)kD, rows_total};
   const cuuint64_t gstride[1] = {(cuuint64_t)kRowBytes};
   const cuuint32_t box[2] = {64u, (cuuint32_t)kBlockN};
   const cuuint32_t estride[2] = {1u, 1u};
