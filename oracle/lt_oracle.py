@@ -57,6 +57,7 @@ __all__ = [
     "select_lazy_priority_queue",
     "select_lazy_priority_queue_trace",
     "select_lazy_per_sequence",
+    "select_lazy_by_frequency",
     "lazy_scores_per_row_window",
     "ring_slot",
     "ring_valid_slots",
@@ -364,6 +365,26 @@ def select_lazy_per_sequence(scores, n_lazy: int):
     for b in range(B):
         mask[b], r[b] = select_lazy(scores[:, b : b + 1, :], n_lazy)
     return mask, r
+
+
+def select_lazy_by_frequency(masks, n_lazy: int):
+    """Layer choice of LightTransfer-Train (Section 5.2): every training sample
+    labels its own lazy layers; count, per layer, how many samples labelled it
+    lazy and keep the n_lazy layers with the highest counts (lower index on
+    ties).  masks [N, L] of 0/1 -> (mask uint8 [L], counts int64 [L]).
+    """
+    masks = np.asarray(masks)
+    N, L = masks.shape
+    assert 0 <= n_lazy <= L
+    counts = np.zeros(L, dtype=np.int64)
+    for i in range(N):
+        for l in range(L):
+            counts[l] += 1 if masks[i, l] else 0
+    order = sorted(range(L), key=lambda l: (-counts[l], l))
+    out = np.zeros(L, dtype=np.uint8)
+    for l in order[:n_lazy]:
+        out[l] = 1
+    return out, counts
 
 
 # --------------------------------------------------------------------------

@@ -255,6 +255,31 @@ def test_per_sequence_selection_is_the_single_prompt_selection_row_by_row():
     assert O.select_lazy_per_sequence(two, 1)[0].tolist() == [[1, 0], [0, 1]]
 
 
+def test_frequency_selection_hand_example_and_brute_force():
+    """Section 5.2: four samples over five layers; layer 3 is lazy in all four,
+    layers 0 and 4 in two each, layer 1 in one, layer 2 never."""
+    masks = np.array([[1, 0, 0, 1, 0],
+                      [0, 1, 0, 1, 1],
+                      [1, 0, 0, 1, 0],
+                      [0, 0, 0, 1, 1]])
+    m, c = O.select_lazy_by_frequency(masks, 2)
+    assert c.tolist() == [2, 1, 0, 4, 2] and m.tolist() == [1, 0, 0, 1, 0]        # tie 0 vs 4 -> lower index
+    assert O.select_lazy_by_frequency(masks, 3)[0].tolist() == [1, 0, 0, 1, 1]
+    assert O.select_lazy_by_frequency(masks, 0)[0].sum() == 0 and O.select_lazy_by_frequency(masks, 5)[0].sum() == 5
+    g = _rng(79)
+    for _ in range(10):
+        N, L = int(g.integers(1, 9)), int(g.integers(1, 8))
+        mk = (g.random((N, L)) < 0.4).astype(np.uint8)
+        for n_lazy in range(L + 1):
+            m, c = O.select_lazy_by_frequency(mk, n_lazy)
+            assert np.array_equal(c, mk.sum(axis=0)) and m.sum() == n_lazy
+            best = max(sum(c[list(s_)]) for s_ in itertools.combinations(range(L), n_lazy))
+            assert c[m == 1].sum() == best
+    # one sample: its own mask comes back when n_lazy matches
+    one = np.array([[0, 1, 1, 0]])
+    assert O.select_lazy_by_frequency(one, 2)[0].tolist() == [0, 1, 1, 0]
+
+
 def _brute_lazy_per_row(Q, K, G, S, R, scale):
     res = []
     for hq in range(len(Q)):
