@@ -191,6 +191,21 @@ lt_status lt_select_lazy_per_seq(const float* scores /* dev [L][B][Hq] */, int32
                                  float* layer_ratio /* dev [B][L] or NULL */, void* stream);
 
 /*
+ * Frequency-count choice of the lazy layers over many samples (Section 5.2,
+ * LightTransfer-Train: every training sample reveals its own lazy layers, "we
+ * then compute the frequency for each layer and select those with the highest
+ * lazy layer counts").
+ *   sample_masks  dev uint8 [n_samples][L]: per-sample masks, e.g. the rows that
+ *                 lt_select_lazy_per_seq wrote for successive batches
+ *   layer_mask    dev uint8 [L]: 1 for the n_lazy layers with the highest counts,
+ *                 ties to the lower layer index
+ *   layer_counts  dev int32 [L] or NULL
+ */
+lt_status lt_select_lazy_frequency(const uint8_t* sample_masks /* dev */, int32_t n_samples, int32_t n_layers,
+                                   int32_t n_lazy, uint8_t* layer_mask /* dev [L] */,
+                                   int32_t* layer_counts /* dev [L] or NULL */, void* stream);
+
+/*
  * Streaming selection, one layer at a time (Section 5.1 and Figure 3: the
  * ratios enter a priority queue of capacity P = n_full during prefilling; when
  * the queue overflows, the layer with the highest ratio is popped, labelled

@@ -103,6 +103,8 @@ def lib() -> C.CDLL:
     L.lt_select_lazy.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
     L.lt_select_lazy_per_seq.restype = i32
     L.lt_select_lazy_per_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    L.lt_select_lazy_frequency.restype = i32
+    L.lt_select_lazy_frequency.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     L.lt_select_lazy_push.restype = i32
     L.lt_select_lazy_push.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     L.lt_stream_init_layer.restype = i32
@@ -222,6 +224,12 @@ def select_lazy_per_seq(scores, n_layers: int, batch: int, n_q_heads: int, n_laz
                         stream=None):
     _ok(lib().lt_select_lazy_per_seq(_ptr(scores), n_layers, batch, n_q_heads, n_lazy, _ptr(layer_mask),
                                      _ptr(layer_ratio), _stream(stream)), "lt_select_lazy_per_seq")
+
+
+def select_lazy_frequency(sample_masks, n_samples: int, n_layers: int, n_lazy: int, layer_mask, layer_counts=None,
+                          stream=None):
+    _ok(lib().lt_select_lazy_frequency(_ptr(sample_masks), n_samples, n_layers, n_lazy, _ptr(layer_mask),
+                                       _ptr(layer_counts), _stream(stream)), "lt_select_lazy_frequency")
 
 
 def select_lazy_push(layer_scores, layer: int, n_layers: int, batch: int, n_q_heads: int, n_full: int, queue_state,

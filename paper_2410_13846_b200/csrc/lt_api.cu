@@ -244,6 +244,17 @@ lt_status lt_select_lazy_per_seq(const float* scores, int32_t n_layers, int32_t 
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 
+lt_status lt_select_lazy_frequency(const uint8_t* sample_masks, int32_t n_samples, int32_t n_layers, int32_t n_lazy,
+                                   uint8_t* layer_mask, int32_t* layer_counts, void* stream) {
+  if (!sample_masks || !layer_mask) return LT_ERR_INVALID_ARG;
+  if (n_samples < 1 || n_layers < 1) return LT_ERR_INVALID_ARG;
+  if (n_layers > LT_MAX_LAYERS) return LT_ERR_UNSUPPORTED;
+  if (n_lazy < 0 || n_lazy > n_layers) return LT_ERR_INVALID_ARG;
+  cudaError_t e = launch_select_frequency(sample_masks, n_samples, n_layers, n_lazy, layer_mask, layer_counts,
+                                          (cudaStream_t)stream);
+  return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
 lt_status lt_select_lazy_push(const float* layer_scores, int32_t layer, int32_t n_layers, int32_t batch,
                               int32_t n_q_heads, int32_t n_full, void* queue_state, uint8_t* layer_mask,
                               int32_t* popped_layer, void* stream) {

@@ -156,6 +156,8 @@ cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy,
 
 cudaError_t launch_select_per_seq(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,
                                   cudaStream_t st);
+cudaError_t launch_select_frequency(const uint8_t* masks, int N, int L, int n_lazy, uint8_t* mask, int32_t* counts,
+                                    cudaStream_t st);
 cudaError_t launch_select_push(const float* scores_l, int layer, int L, int per_layer, int n_full, double* state,
                                uint8_t* mask, int32_t* popped, cudaStream_t st);
 

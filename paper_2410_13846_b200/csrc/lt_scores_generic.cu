@@ -220,6 +220,32 @@ cudaError_t launch_select_push(const float* scores_l, int layer, int L, int per_
   return cudaGetLastError();
 }
 
+// Frequency-count choice: thread l counts the samples that labelled layer l lazy
+// (integer, exact), then ranks itself (count descending, index ascending).
+__global__ void select_frequency_kernel(const uint8_t* __restrict__ masks, int N, int L, int n_lazy,
+                                        uint8_t* __restrict__ mask, int32_t* __restrict__ counts) {
+  __shared__ int c[LT_MAX_LAYERS];
+  const int l = threadIdx.x;
+  if (l < L) {
+    int acc = 0;
+    for (int i = 0; i < N; ++i) acc += masks[(long long)i * L + l] != 0;
+    c[l] = acc;
+  }
+  __syncthreads();
+  if (l < L) {
+    int rank = 0;
+    for (int m = 0; m < L; ++m) rank += (c[m] > c[l]) || (c[m] == c[l] && m < l);
+    mask[l] = rank < n_lazy ? 1 : 0;
+    if (counts) counts[l] = c[l];
+  }
+}
+
+cudaError_t launch_select_frequency(const uint8_t* masks, int N, int L, int n_lazy, uint8_t* mask, int32_t* counts,
+                                    cudaStream_t st) {
+  select_frequency_kernel<<<1, LT_MAX_LAYERS, 0, st>>>(masks, N, L, n_lazy, mask, counts);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_select(const float* scores, int L, int B, int Hq, int n_lazy, uint8_t* mask, float* ratio,
                           cudaStream_t st) {
   select_kernel<<<1, LT_MAX_LAYERS, 0, st>>>(scores, L, B * Hq, n_lazy, mask, ratio);

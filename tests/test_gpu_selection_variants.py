@@ -26,6 +26,29 @@ def test_per_sequence_selection_fed_oracle_scores_is_bit_exact():
             assert np.allclose(ratio.cpu().numpy(), er, rtol=0, atol=1e-7)
 
 
+def test_frequency_choice_over_per_sample_masks_is_bit_exact():
+    """Section 5.2: per-sample masks (here from lt_select_lazy_per_seq over several
+    batches of samples) are counted per layer and the most frequent layers chosen."""
+    g = np.random.default_rng(26)
+    L, B, Hq, n_lazy = 12, 5, 4, 5
+    rows = []
+    for _ in range(3):                                            # three batches of five samples
+        sc = g.random((L, B, Hq)).astype(np.float32)
+        sc[[2, 7, 9]] += 0.5                                      # layers that most samples find lazy
+        m = torch.zeros((B, L), dtype=torch.uint8, device="cuda")
+        lt.select_lazy_per_seq(torch.from_numpy(sc).cuda(), L, B, Hq, n_lazy, m)
+        assert np.array_equal(m.cpu().numpy(), O.select_lazy_per_sequence(sc, n_lazy)[0])
+        rows.append(m)
+    masks = torch.cat(rows).contiguous()                          # [15][L]
+    for k in (0, 3, 5, L):
+        out = torch.full((L,), 9, dtype=torch.uint8, device="cuda")
+        cnt = torch.zeros(L, dtype=torch.int32, device="cuda")
+        lt.select_lazy_frequency(masks, masks.shape[0], L, k, out, cnt)
+        em, ec = O.select_lazy_by_frequency(masks.cpu().numpy(), k)
+        assert np.array_equal(out.cpu().numpy(), em) and np.array_equal(cnt.cpu().numpy(), ec)
+    assert {2, 7, 9} <= set(np.nonzero(O.select_lazy_by_frequency(masks.cpu().numpy(), 5)[0])[0].tolist())
+
+
 def test_per_sequence_masks_through_compaction_and_decode():
     """Every prompt of the batch has its own lazy layers: compaction, fused decode
     steps (ring wraps) and the separate append/attend calls follow the [B][L] mask."""
