@@ -23,6 +23,10 @@ the paper one step at a time, with no blocking, fusion or reordering:
   O5  ring_slot / ring_owner / stream_cache_after / HybridReplay
                             integer model of the constant-size cache of a lazy
                             layer (Section 5.1, retained {X_initial, X_recent})
+  O6  quantize_e4m3         8-bit storage of cached keys / values (not in the
+                            paper, which keeps BF16 everywhere, Appendix A; an
+                            adjacent deployment option): the OCP FP8 E4M3
+                            format written out from its definition
 
 Readings taken where the paper is silent or inconsistent (scale 1/sqrt(D) in
 numerator and denominator, causal mask inside the tail block, X_recent as the
@@ -64,6 +68,8 @@ __all__ = [
     "ring_owner",
     "stream_cache_after",
     "HybridReplay",
+    "e4m3_values",
+    "quantize_e4m3",
 ]
 
 
@@ -449,3 +455,65 @@ class HybridReplay:
         if self.mask[l]:
             return streaming_attention(q, self.K[l], self.V[l], self.S, self.R, self.scale)
         return full_attention(q, self.K[l], self.V[l], self.scale)
+
+
+# --------------------------------------------------------------------------
+# O6: FP8 E4M3 storage (OCP 8-bit floating point specification, E4M3 variant)
+# --------------------------------------------------------------------------
+def e4m3_values():
+    """Value of every E4M3 code 0..255 as float64 (NaN for the two NaN codes).
+    Layout s.eeee.mmm, exponent bias 7; e = 0 is subnormal (m/8 * 2^-6); there
+    are no infinities, and s.1111.111 is NaN, so the largest finite value is
+    1.75 * 2^8 = 448."""
+    out = np.zeros(256, dtype=np.float64)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e = (code >> 3) & 0xF
+        m = code & 0x7
+        if e == 0xF and m == 0x7:
+            out[code] = np.nan
+        elif e == 0:
+            out[code] = sign * (m / 8.0) * 2.0 ** -6
+        else:
+            out[code] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return out
+
+
+def quantize_e4m3(x, scale):
+    """Codes and dequantised values of x stored as E4M3 with one scale:
+        y = float32(x) / float32(scale)          (one IEEE float32 division)
+        code = nearest E4M3 value to y, ties to the even code, saturating at +-448
+        value = E4M3(code) * float32(scale)      (exact in float64)
+    NaN maps to the NaN code.  returns (codes uint8, values float64), shaped like x.
+    """
+    table = e4m3_values()
+    xs = np.asarray(x, dtype=np.float32)
+    y = (xs / np.float32(scale)).astype(np.float32).astype(np.float64)
+    flat = y.reshape(-1)
+    codes = np.zeros(flat.shape, dtype=np.uint8)
+    pos_codes = np.arange(0, 0x7F)               # 0 .. 126: non-negative finite values, increasing
+    pos_vals = table[pos_codes]
+    for i, v in enumerate(flat):
+        if np.isnan(v):
+            codes[i] = 0x7F
+            continue
+        a = min(abs(v), 448.0)
+        hi = int(np.searchsorted(pos_vals, a, side="left"))      # first value >= a
+        if hi == 0:
+            c = 0
+        else:
+            lo = hi - 1
+            if hi >= len(pos_vals):
+                c = lo
+            else:
+                dlo, dhi = a - pos_vals[lo], pos_vals[hi] - a
+                if dlo < dhi:
+                    c = lo
+                elif dhi < dlo:
+                    c = hi
+                else:
+                    c = lo if (lo & 1) == 0 else hi              # tie: even mantissa
+        codes[i] = c | (0x80 if np.signbit(v) else 0)
+    codes = codes.reshape(y.shape)
+    values = table[codes] * float(np.float32(scale))
+    return codes, values
