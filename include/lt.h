@@ -95,6 +95,16 @@ typedef struct lt_shape {
   int32_t n_pages;             /* pages in every layer's pool */
   int32_t reserved_;           /* keep the pointer 8-byte aligned; must be 0 */
   const int32_t* block_table;  /* dev int32 [batch][pages_per_seq], entries in [0, n_pages); read during device work */
+  /* 8-bit caches (not in the paper, which keeps BF16 everywhere, Appendix A; a deployment option).
+     kv_fp8 = 1: full and stream caches hold FP8 E4M3 bytes (rows of head_dim bytes) while q, k_new,
+     v_new and out stay in `dtype`.  A stored byte c of layer l means E4M3(c) * kv_scales[l][0] for K and
+     * kv_scales[l][1] for V; lt_kv_append / lt_decode_step store code(x) = E4M3 nearest to
+     float32(x) / scale (float32 division, round to nearest even, saturating at +-448).  Needs
+     dtype = LT_BF16, head_dim = 128 and a query group of at most 8.  lt_lazy_scores and lt_lazy_scores_lse
+     do not read 8-bit keys: score from the prefill's 16-bit keys with a shape whose kv_fp8 is 0. */
+  int32_t kv_fp8;
+  int32_t reserved2_;      /* must be 0 */
+  const float* kv_scales;  /* dev float [n_layers][2] (K scale, V scale), positive; read during device work */
 } lt_shape;
 
 /* Text for a status code (static storage, never NULL). */

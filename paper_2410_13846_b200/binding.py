@@ -28,7 +28,9 @@ class _CShape(C.Structure):
                  "full_capacity", "dtype")] + [("softmax_scale", C.c_float), ("per_sequence_mask", C.c_int32),
                                                 ("recent_per_row", C.c_int32), ("page_size", C.c_int32),
                                                 ("pages_per_seq", C.c_int32), ("n_pages", C.c_int32),
-                                                ("reserved_", C.c_int32), ("block_table", C.c_void_p)]
+                                                ("reserved_", C.c_int32), ("block_table", C.c_void_p),
+                                                ("kv_fp8", C.c_int32), ("reserved2_", C.c_int32),
+                                                ("kv_scales", C.c_void_p)]
 
 
 @dataclass
@@ -49,6 +51,8 @@ class Shape:
     pages_per_seq: int = 0
     n_pages: int = 0
     block_table: object = None   # int32 CUDA tensor [batch][pages_per_seq]
+    kv_fp8: int = 0              # 1: caches hold FP8 E4M3 bytes with per-layer scales
+    kv_scales: object = None     # float32 CUDA tensor [n_layers][2]
 
     def c(self) -> _CShape:
         bt = None
@@ -59,7 +63,17 @@ class Shape:
             bt = t.data_ptr()
         return _CShape(self.n_layers, self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_sink,
                        self.n_recent, self.full_capacity, self.dtype, self.softmax_scale, self.per_sequence_mask,
-                       self.recent_per_row, self.page_size, self.pages_per_seq, self.n_pages, 0, bt)
+                       self.recent_per_row, self.page_size, self.pages_per_seq, self.n_pages, 0, bt, self.kv_fp8, 0,
+                       self._scales_ptr())
+
+    def _scales_ptr(self):
+        t = self.kv_scales
+        if t is None:
+            return None
+        import torch
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32):
+            raise ValueError("kv_scales must be a contiguous float32 CUDA tensor")
+        return t.data_ptr()
 
     @property
     def stream_capacity(self) -> int:

@@ -20,7 +20,12 @@ lt_status validate_shape(const lt_shape* s) {
   if (s->dtype != LT_F32 && s->dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
   if (!(s->softmax_scale == s->softmax_scale)) return LT_ERR_INVALID_ARG;  // NaN
   if ((s->per_sequence_mask | s->recent_per_row) & ~1) return LT_ERR_INVALID_ARG;
-  if (s->page_size < 0 || s->reserved_ != 0) return LT_ERR_INVALID_ARG;
+  if (s->page_size < 0 || s->reserved_ != 0 || s->reserved2_ != 0) return LT_ERR_INVALID_ARG;
+  if (s->kv_fp8 & ~1) return LT_ERR_INVALID_ARG;
+  if (s->kv_fp8) {
+    if (!s->kv_scales) return LT_ERR_INVALID_ARG;
+    if (s->dtype != LT_BF16 || s->head_dim != 128 || s->n_q_heads / s->n_kv_heads > 8) return LT_ERR_UNSUPPORTED;
+  }
   if (s->page_size > 0) {
     if (s->page_size % 128 != 0) return LT_ERR_UNSUPPORTED;
     if (s->pages_per_seq < 1 || s->n_pages < 1 || !s->block_table) return LT_ERR_INVALID_ARG;
@@ -183,6 +188,7 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   if (st != LT_OK) return st;
   if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
   if (window_only && !lse) return LT_ERR_INVALID_ARG;
+  if (shape->kv_fp8) return LT_ERR_UNSUPPORTED;  // scoring reads 16- or 32-bit keys only
   if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
   if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0) return LT_ERR_INVALID_ARG;
   LayerTable kf;

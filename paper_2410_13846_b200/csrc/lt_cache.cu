@@ -1,6 +1,9 @@
 // KV-cache movement: per-step append (full layers and lazy layers) and the
 // prefill -> decode compaction of the lazy layers.  Pure data movement with
 // integer addressing; every row is copied bit for bit in 16-byte vectors.
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+
 #include "lt_internal.h"
 
 namespace lt {
@@ -37,6 +40,26 @@ __global__ void append_kernel(lt_shape s, const uint8_t* __restrict__ mask, cons
   }
   const long long src = ((long long)(l * B + b) * Hkv + h) * vec_per_row + v;
   const long long drow = lazy ? ((long long)b * Hkv + h) * rows + slot : full_cache_row(s, b, h, slot);
+  if (s.kv_fp8) {
+    // 8 bf16 values -> 8 E4M3 bytes: float32 division by the layer's scale, round to nearest even, saturate
+    auto quantize8 = [](uint4 x, float scale) {
+      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+      uint2 out = make_uint2(0u, 0u);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t pair = w[e >> 1];
+        const float f = __uint_as_float((e & 1) ? (pair & 0xffff0000u) : (pair << 16));
+        const uint32_t code = (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(f, scale), __NV_SATFINITE, __NV_E4M3);
+        if (e < 4) out.x |= code << (8 * e);
+        else out.y |= code << (8 * (e - 4));
+      }
+      return out;
+    };
+    const long long dst8 = drow * vec_per_row + v;  // 8-byte units: a cached row has vec_per_row of them
+    reinterpret_cast<uint2*>(kdst)[dst8] = quantize8(k_new[src], s.kv_scales[2 * l]);
+    reinterpret_cast<uint2*>(vdst)[dst8] = quantize8(v_new[src], s.kv_scales[2 * l + 1]);
+    return;
+  }
   const long long dst = drow * vec_per_row + v;
   kdst[dst] = k_new[src];
   vdst[dst] = v_new[src];
@@ -114,7 +137,7 @@ __global__ void stream_init_kernel(lt_shape s, const uint8_t* __restrict__ mask,
 cudaError_t launch_stream_init(const lt_shape& s, const uint8_t* mask, const LayerTable& kf, const LayerTable& vf,
                                const int32_t* seq_lens, const LayerTable& ks, const LayerTable& vs,
                                const int32_t* only_layer, uint32_t* dev_err, cudaStream_t st) {
-  const int vec_per_row = (int)(s.head_dim * elem_bytes(s.dtype) / 16);
+  const int vec_per_row = (int)(cache_row_bytes(s) / 16);
   const int C = s.n_sink + s.n_recent;
   const long long total = (long long)C * vec_per_row;
   const int threads = 256;

@@ -28,6 +28,9 @@
 // bf16 residual (two MMAs) so that the probabilities keep ~16 bits.
 #include <cuda_bf16.h>
 
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+
 #include "lt_decode_common.cuh"
 #include "lt_internal.h"
 
@@ -62,6 +65,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
@@ -75,8 +84,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float f16_lo(uint32_t x) { return __low2float(*reinterpret_cast<__half2*>(&x)); }
+__device__ __forceinline__ float f16_hi(uint32_t x) { return __high2float(*reinterpret_cast<__half2*>(&x)); }
+// Four E4M3 bytes -> four f16 whose value is the E4M3 value / 256, by moving bits only: an E4M3 byte
+// s.eeee.mmm placed at bits 15..8 and shifted so that eeee.mmm lands in f16's exponent / mantissa
+// field reads as 2^(e-15) (1 + m/8) instead of 2^(e-7) (1 + m/8), subnormals included (m/8 * 2^-14
+// instead of m/8 * 2^-6).  The factor 256 is folded into the per-layer scales.
+__device__ __forceinline__ void e4m3x4_to_f16x4_div256(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t t0 = __byte_perm(w, 0u, 0x1404);  // byte 0 -> bits 15..8, byte 1 -> bits 31..24
+  const uint32_t t1 = __byte_perm(w, 0u, 0x3424);  // bytes 2, 3
+  lo = (t0 & 0x80008000u) | ((t0 >> 1) & 0x3f803f80u);
+  hi = (t1 & 0x80008000u) | ((t1 >> 1) & 0x3f803f80u);
+}
+__device__ __forceinline__ uint32_t ld_shared_u32x4(uint32_t addr, uint32_t& y, uint32_t& z, uint32_t& w) {
+  uint32_t x;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(addr));
+  return x;
+}
+__device__ __forceinline__ void st_shared_u32x4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
 constexpr int kD = 128;
-constexpr int kRowBytes = kD * 2;  // one K or V row
+constexpr int kSrcRowBytes = kD * 2;  // one row of q, k_new, v_new (bf16)
 
 }  // namespace
 
@@ -90,20 +124,32 @@ struct TileSrc {
   int new_row;               // -1 when the chunk does not hold the new token
   int my_tiles;              // tiles of this warp (tiles warp, warp + WARPS, ... of the chunk)
   int tbl_off;               // paged full cache: offset of this batch row's block-table row, else -1
+  int layer;                 // for the per-layer scales of 8-bit caches
 };
 
 // Shared memory: [rings: WARPS x NSTAGE x stage][merge: two 8 x 128 fp32 buffers,
 // (max, sum) of every warp][work list].  A stage holds K half-tiles
 // [2][TILE][128 B] then V half-tiles [2][TILE][128 B]; inside a half-tile the
 // 16-byte column c of row r sits at column c ^ (r & 7).
-template <int TILE, int NSTAGE, int WARPS, int MINB>
+//
+// FP8 = true: the caches hold E4M3 bytes (rows of 128 B) with one scale per layer
+// for K and one for V.  A ring stage then holds the raw bytes of a tile (K rows,
+// then V rows); before the MMAs the warp expands the tile into a private 16-bit
+// buffer in the layout above (f16, by bit moves, as value / 256), Q and P are f16
+// as well, the K scale (x 256) is folded into the softmax scale and the V scale
+// (x 256) into the final normalisation.
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
   constexpr int MT = TILE / 16;                // 16-key MMA tiles per pipeline tile
   constexpr int HALF_BYTES = TILE * 128;       // one half-tile
-  constexpr int STAGE_BYTES = 4 * HALF_BYTES;  // K halves + V halves
-  constexpr int RING_BYTES = WARPS * NSTAGE * STAGE_BYTES;
+  constexpr int STAGE_BYTES = 4 * HALF_BYTES;  // K halves + V halves (16-bit layout)
+  constexpr int kRowBytes = FP8 ? kD : 2 * kD;             // one cached K or V row
+  constexpr int RAW_BYTES = 2 * TILE * kD;                 // FP8: K rows + V rows of a tile as stored
+  constexpr int RING_STAGE = FP8 ? RAW_BYTES : STAGE_BYTES;  // what one ring stage holds
+  constexpr int WARP_BYTES = NSTAGE * RING_STAGE + (FP8 ? STAGE_BYTES : 0);
+  constexpr int RING_BYTES = WARPS * WARP_BYTES;
   constexpr int MERGE_BYTES = 2 * 8 * kD * 4 + 2 * WARPS * 8 * 4;
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ int s_flag, s_next;
@@ -120,7 +166,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
-  const uint32_t wsm = smem_u32(smem) + warp * (NSTAGE * STAGE_BYTES);
+  const uint32_t wsm = smem_u32(smem) + warp * WARP_BYTES;
+  const uint32_t wconv = wsm + NSTAGE * RING_STAGE;  // FP8: the warp's expanded tile
   // lane-constant parts of the ldmatrix addresses
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8;  // K (A operand, not transposed)
   const int k_chk = lane >> 4;
@@ -136,13 +183,14 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     t.Kb = (const uint8_t*)(w.lazy ? ks.p[w.l] : kf.p[w.l]) + base_row * kRowBytes;
     t.Vb = (const uint8_t*)(w.lazy ? vs.p[w.l] : vf.p[w.l]) + base_row * kRowBytes;
     t.tbl_off = paged ? w.b * s.pages_per_seq : -1;
+    t.layer = w.l;
     t.j0 = w.j0;
     t.j1 = w.j1;
     t.new_row = w.new_row;
     t.k_new_row = nullptr;
     t.v_new_row = nullptr;
     if (w.new_row >= 0) {
-      const long long src = (((long long)w.l * s.batch + w.b) * s.n_kv_heads + w.h) * kRowBytes;
+      const long long src = (((long long)w.l * s.batch + w.b) * s.n_kv_heads + w.h) * kSrcRowBytes;
       t.k_new_row = (const uint8_t*)a.k_new + src;
       t.v_new_row = (const uint8_t*)a.v_new + src;
     }
@@ -157,21 +205,83 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     const int page = s.block_table[t.tbl_off + row / s.page_size];
     return (long long)page * s.n_kv_heads * s.page_size + row % s.page_size;
   };
+  // 16 bf16 values of a new row -> 16 E4M3 bytes with the layer's scale (same rounding as lt_kv_append)
+  auto quantize16 = [&](const uint8_t* src32, float scale, uint32_t (&out)[4]) {
+    const uint4 lo = *reinterpret_cast<const uint4*>(src32), hi = *reinterpret_cast<const uint4*>(src32 + 16);
+    const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t packed = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t pair = w[2 * i + (e >> 1)];
+        const float x = (e & 1) ? bf16_hi(pair) : bf16_lo(pair);
+        packed |= (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(x, scale), __NV_SATFINITE, __NV_E4M3) << (8 * e);
+      }
+      out[i] = packed;
+    }
+  };
   auto fetch_tile = [&](const TileSrc& t, int idx, int stage) {
     const int key_base = t.j0 + (warp + idx * WARPS) * TILE;
     const long long tile_row = cache_row(t, key_base);
-    const uint32_t st = wsm + stage * STAGE_BYTES;
+    const uint32_t st = wsm + stage * RING_STAGE;
+    if constexpr (FP8) {
+      // raw rows: 8 chunks of 16 bytes per row, K rows then V rows
 #pragma unroll
-    for (int i = 0; i < TILE / 2; ++i) {
-      const int r = 2 * i + (lane >> 4);
-      const int p = lane & 15;
-      const int row = key_base + r;
-      const bool valid = row < t.j1;
-      const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
-      const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
-      const bool fresh = row == t.new_row;
-      cp_async16(st + soff, fresh ? t.k_new_row + p * 16 : t.Kb + goff, valid ? 16 : 0);
-      cp_async16(st + 2 * HALF_BYTES + soff, fresh ? t.v_new_row + p * 16 : t.Vb + goff, valid ? 16 : 0);
+      for (int i = 0; i < TILE / 4; ++i) {
+        const int ci = i * 32 + lane;
+        const int r = ci >> 3, p = ci & 7;
+        const int row = key_base + r;
+        const bool valid = row < t.j1;
+        const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
+        const uint32_t soff = r * kD + p * 16;
+        if (row == t.new_row) {
+          // the new token's row is quantised on the fly from k_new / v_new
+          uint32_t q4[4];
+          quantize16(t.k_new_row + p * 32, a.s.kv_scales[2 * t.layer], q4);
+          st_shared_u32x4(st + soff, q4[0], q4[1], q4[2], q4[3]);
+          quantize16(t.v_new_row + p * 32, a.s.kv_scales[2 * t.layer + 1], q4);
+          st_shared_u32x4(st + TILE * kD + soff, q4[0], q4[1], q4[2], q4[3]);
+        } else {
+          cp_async16(st + soff, t.Kb + goff, valid ? 16 : 0);
+          cp_async16(st + TILE * kD + soff, t.Vb + goff, valid ? 16 : 0);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < TILE / 2; ++i) {
+        const int r = 2 * i + (lane >> 4);
+        const int p = lane & 15;
+        const int row = key_base + r;
+        const bool valid = row < t.j1;
+        const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
+        const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
+        const bool fresh = row == t.new_row;
+        cp_async16(st + soff, fresh ? t.k_new_row + p * 16 : t.Kb + goff, valid ? 16 : 0);
+        cp_async16(st + 2 * HALF_BYTES + soff, fresh ? t.v_new_row + p * 16 : t.Vb + goff, valid ? 16 : 0);
+      }
+    }
+  };
+  // FP8: expand the raw tile in ring stage `stage` into the warp's 16-bit buffer
+  auto expand_tile = [&](int stage) {
+    const uint32_t raw = wsm + stage * RING_STAGE;
+#pragma unroll
+    for (int kv = 0; kv < 2; ++kv) {
+#pragma unroll
+      for (int i = 0; i < TILE / 4; ++i) {
+        const int ci = i * 32 + lane;
+        const int r = ci >> 3, p = ci & 7;  // row, 16-byte chunk = 16 values d = 16p .. 16p + 15
+        uint32_t w1, w2, w3;
+        const uint32_t w0 = ld_shared_u32x4(raw + kv * TILE * kD + r * kD + p * 16, w1, w2, w3);
+        const uint32_t dst = wconv + kv * 2 * HALF_BYTES + (p >> 2) * HALF_BYTES + r * 128;
+        uint32_t h0, h1, h2, h3, h4, h5, h6, h7;
+        e4m3x4_to_f16x4_div256(w0, h0, h1);
+        e4m3x4_to_f16x4_div256(w1, h2, h3);
+        e4m3x4_to_f16x4_div256(w2, h4, h5);
+        e4m3x4_to_f16x4_div256(w3, h6, h7);
+        st_shared_u32x4(dst + ((((2 * p) & 7) ^ (r & 7)) << 4), h0, h1, h2, h3);
+        st_shared_u32x4(dst + ((((2 * p + 1) & 7) ^ (r & 7)) << 4), h4, h5, h6, h7);
+      }
     }
   };
 
@@ -212,12 +322,31 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     int fetched_next = 0;
     if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
 
+    // per-layer scales of 8-bit caches: K's goes into the softmax scale, V's into the normalisation
+    float cs_l = a.cs, v_scale = 1.f;
+    if constexpr (FP8) {
+      cs_l = a.cs * a.s.kv_scales[2 * l] * 256.f;  // 256: the expanded tile holds value / 256
+      v_scale = a.s.kv_scales[2 * l + 1] * 256.f;
+    }
+
     // fused append: store the new token's row into the cache
     if (src_cur.new_row >= 0 && warp == 0) {
-      const uint8_t* sp = (lane < 16 ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 15) * 16;
-      uint8_t* dp = const_cast<uint8_t*>(lane < 16 ? src_cur.Kb : src_cur.Vb) +
-                    cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane & 15) * 16;
-      *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
+      if constexpr (FP8) {
+        if (lane < 16) {
+          const bool is_k = lane < 8;
+          uint32_t q4[4];
+          quantize16((is_k ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 7) * 32,
+                     a.s.kv_scales[2 * l + (is_k ? 0 : 1)], q4);
+          uint8_t* dp = const_cast<uint8_t*>(is_k ? src_cur.Kb : src_cur.Vb) +
+                        cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane & 7) * 16;
+          *reinterpret_cast<uint4*>(dp) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
+        }
+      } else {
+        const uint8_t* sp = (lane < 16 ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 15) * 16;
+        uint8_t* dp = const_cast<uint8_t*>(lane < 16 ? src_cur.Kb : src_cur.Vb) +
+                      cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane & 15) * 16;
+        *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
+      }
     }
 
     // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
@@ -230,6 +359,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         if (gp < G) {
           qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
           qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
+          if constexpr (FP8) {  // f16 operands: bf16 -> f16 is exact inside f16's range
+            qf[ks8][0] = pack_f16(bf16_lo(qf[ks8][0]), bf16_hi(qf[ks8][0]));
+            qf[ks8][1] = pack_f16(bf16_lo(qf[ks8][1]), bf16_hi(qf[ks8][1]));
+          }
         } else {
           qf[ks8][0] = 0u;
           qf[ks8][1] = 0u;
@@ -250,7 +383,12 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       issue_slot();
       cp_async_wait<NSTAGE - 1>();
       __syncwarp();              // all lanes' copies of this tile have landed
-      const uint32_t st = wsm + (consumed % NSTAGE) * STAGE_BYTES;
+      uint32_t st = wsm + (consumed % NSTAGE) * RING_STAGE;
+      if constexpr (FP8) {
+        expand_tile(consumed % NSTAGE);
+        __syncwarp();  // the expanded tile is complete before any lane's ldmatrix
+        st = wconv;
+      }
       ++consumed;
       const int key_base = src_cur.j0 + (warp + it * WARPS) * TILE;
 
@@ -265,7 +403,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           uint32_t af[4];
           const int chunk = 2 * (ks8 & 3) + k_chk;
           ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-          mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+          if constexpr (FP8) mma_f16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+          else mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
         }
       }
       // ---- scale, mask the ragged tail, tile max per head ---------------------
@@ -274,10 +413,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       for (int mt = 0; mt < MT; ++mt) {
         const int key_lo = key_base + mt * 16 + gp;
         const bool v_lo = key_lo < j1, v_hi = key_lo + 8 < j1;
-        sc[mt][0] = v_lo ? sc[mt][0] * a.cs : -INFINITY;
-        sc[mt][1] = v_lo ? sc[mt][1] * a.cs : -INFINITY;
-        sc[mt][2] = v_hi ? sc[mt][2] * a.cs : -INFINITY;
-        sc[mt][3] = v_hi ? sc[mt][3] * a.cs : -INFINITY;
+        sc[mt][0] = v_lo ? sc[mt][0] * cs_l : -INFINITY;
+        sc[mt][1] = v_lo ? sc[mt][1] * cs_l : -INFINITY;
+        sc[mt][2] = v_hi ? sc[mt][2] * cs_l : -INFINITY;
+        sc[mt][3] = v_hi ? sc[mt][3] * cs_l : -INFINITY;
         mx0 = fmaxf(mx0, fmaxf(sc[mt][0], sc[mt][2]));
         mx1 = fmaxf(mx1, fmaxf(sc[mt][1], sc[mt][3]));
       }
@@ -306,9 +445,18 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         const float p2 = exp2f(sc[mt][2] - Mn0), p3 = exp2f(sc[mt][3] - Mn1);
         l0 += p0 + p2;
         l1 += p1 + p3;
-        const uint32_t hi01 = pack_bf16(p0, p1), hi23 = pack_bf16(p2, p3);
-        const uint32_t lo01 = pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01));
-        const uint32_t lo23 = pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23));
+        uint32_t hi01, hi23, lo01, lo23;  // P as a 16-bit head and a 16-bit residual
+        if constexpr (FP8) {
+          hi01 = pack_f16(p0, p1);
+          hi23 = pack_f16(p2, p3);
+          lo01 = pack_f16(p0 - f16_lo(hi01), p1 - f16_hi(hi01));
+          lo23 = pack_f16(p2 - f16_lo(hi23), p3 - f16_hi(hi23));
+        } else {
+          hi01 = pack_bf16(p0, p1);
+          hi23 = pack_bf16(p2, p3);
+          lo01 = pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01));
+          lo23 = pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23));
+        }
         const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
         const uint32_t bl0 = movmatrix_trans(lo01), bl1 = movmatrix_trans(lo23);
         const int row = mt * 16 + v_row;
@@ -318,8 +466,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           const int chunk = 2 * (dt & 3) + v_chk;
           ldmatrix_x4_trans(af,
                             st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-          mma_bf16(o[dt], af, bh0, bh1);
-          mma_bf16(o[dt], af, bl0, bl1);
+          if constexpr (FP8) {
+            mma_f16(o[dt], af, bh0, bh1);
+            mma_f16(o[dt], af, bl0, bl1);
+          } else {
+            mma_bf16(o[dt], af, bh0, bh1);
+            mma_bf16(o[dt], af, bl0, bl1);
+          }
         }
       }
     }
@@ -425,7 +578,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
               for (int half = 0; half < 2; ++half) {
                 const float num = o[dt][e + 2 * half];
-                const float r = den > 0.f ? num / den : 0.f;
+                const float r = den > 0.f ? (num / den) * v_scale : 0.f;
                 const long long oi = ob + (long long)g * kD + dt * 16 + gp + 8 * half;
                 if (a.out_dtype == LT_F32) ((float*)a.out)[oi] = r;
                 else ((__nv_bfloat16*)a.out)[oi] = __float2bfloat16_rn(r);
@@ -477,14 +630,14 @@ bool decode_mma_supported(const lt_shape& s) {
   return s.dtype == LT_BF16 && s.head_dim == 128 && (s.n_q_heads / s.n_kv_heads) <= 8;
 }
 
-template <int TILE, int NSTAGE, int WARPS, int MINB>
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int ring = WARPS * NSTAGE * TILE * 512;
+  constexpr int ring = FP8 ? WARPS * (NSTAGE * TILE * 256 + TILE * 512) : WARPS * NSTAGE * TILE * 512;
   constexpr int merge = 2 * 8 * 128 * 4 + 2 * WARPS * 8 * 4;
   static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
-  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB>;
+  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8>;
   // attribute and occupancy are looked up once per shared-memory size (host time matters for per-layer callers)
   static int cached_smem_of[64], cached_per_sm_of[64];  // per device; zero = not looked up yet
   int dev = 0;
@@ -508,7 +661,9 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
-  return launch_variant<16, 3, 4, 2>(a, kf, vf, ks, vs, st);
+  // 8-bit caches: four raw stages (4 KB each) + the expanded tile = the 24 KB per warp of the 16-bit ring
+  if (a.s.kv_fp8) return launch_variant<16, 4, 4, 2, true>(a, kf, vf, ks, vs, st);
+  return launch_variant<16, 3, 4, 2, false>(a, kf, vf, ks, vs, st);
 }
 
 }  // namespace lt

@@ -59,6 +59,8 @@ inline float resolved_scale(const lt_shape& s) {
   return s.softmax_scale > 0.f ? s.softmax_scale : 1.0f / sqrtf((float)s.head_dim);
 }
 inline size_t elem_bytes(int dtype) { return dtype == LT_BF16 ? 2 : 4; }
+// Bytes of one cached K or V row.
+inline size_t cache_row_bytes(const lt_shape& s) { return s.kv_fp8 ? (size_t)s.head_dim : s.head_dim * elem_bytes(s.dtype); }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 lt_status validate_shape(const lt_shape* s);

@@ -1,0 +1,107 @@
+"""GPU parity with 8-bit (FP8 E4M3) caches: the append stores exactly the codes
+of the oracle's quantiser (O6), the decode step attends over the dequantised
+values like O1 / O2 on the logical history."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2410_13846_b200 as lt
+from oracle import lt_oracle as O
+from tests.gpu_util import ATTN_MAX_ABS, ATTN_REL_L2, attn_errors, f64
+
+pytestmark = pytest.mark.gpu
+
+
+class Fp8Stack:
+    def __init__(self, L, B, Hq, Hkv, S, R, cap, scales, **kw):
+        D = 128
+        self.scales = torch.tensor(scales, dtype=torch.float32).cuda().contiguous()          # [L][2]
+        self.shape = lt.Shape(L, B, Hq, Hkv, D, S, R, cap, lt.LT_BF16, 0.0, kv_fp8=1, kv_scales=self.scales, **kw)
+        mk = lambda n: [torch.zeros((B, Hkv, n, D), dtype=torch.uint8, device="cuda") for _ in range(L)]
+        self.k_full, self.v_full, self.k_stream, self.v_stream = mk(cap), mk(cap), mk(S + R), mk(S + R)
+        self.tables = lt.LayerTables(self.shape, self.k_full, self.v_full, self.k_stream, self.v_stream)
+        self.ws = torch.empty(lt.workspace_bytes(self.shape), dtype=torch.uint8, device="cuda")
+        lt.workspace_init(self.ws)
+        self.seq_lens = torch.zeros(B, dtype=torch.int32, device="cuda")
+        self.mask = torch.zeros(L, dtype=torch.uint8, device="cuda")
+
+
+@pytest.mark.parametrize("Hq,Hkv,S,R,lens,steps", [
+    (8, 2, 4, 28, [300, 1, 31, 2047], 36),         # G = 4; the ring wraps; a chunk boundary is crossed
+    (5, 1, 0, 16, [70, 15], 20),                   # G = 5, no sink
+    (16, 2, 3, 9, [5, 0], 14),                     # G = 8, starts (almost) empty
+])
+def test_fp8_caches_append_codes_and_attention(Hq, Hkv, S, R, lens, steps):
+    torch.manual_seed(33)
+    g = np.random.default_rng(33)
+    L, B, D = 3, len(lens), 128
+    mask = np.array([0, 1, 0], dtype=np.uint8)
+    cap = max(lens) + steps + 1
+    scales = g.uniform(0.015, 0.04, size=(L, 2)).astype(np.float32)
+    fus = Fp8Stack(L, B, Hq, Hkv, S, R, cap, scales)
+    sep = Fp8Stack(L, B, Hq, Hkv, S, R, cap, scales)
+    replays = [O.HybridReplay(mask, S, R) for _ in range(B)]
+    codes_hist = [[None] * B for _ in range(L)]                                  # K codes of the logical history
+    for l in range(L):
+        hk = torch.randn(B, Hkv, max(lens), D).bfloat16()
+        hv = torch.randn(B, Hkv, max(lens), D).bfloat16()
+        kc, kval = O.quantize_e4m3(f64(hk), scales[l, 0])
+        vc, vval = O.quantize_e4m3(f64(hv), scales[l, 1])
+        for st in (fus, sep):
+            st.k_full[l][:, :, :max(lens)] = torch.from_numpy(kc).cuda()
+            st.v_full[l][:, :, :max(lens)] = torch.from_numpy(vc).cuda()
+        for b, n in enumerate(lens):
+            replays[b].load_prompt(l, kval[b, :, :n], vval[b, :, :n])
+            codes_hist[l][b] = kc[b, :, :n]
+    for st in (fus, sep):
+        st.mask.copy_(torch.from_numpy(mask)); st.seq_lens.copy_(torch.tensor(lens, dtype=torch.int32))
+        lt.stream_init(st.shape, st.mask, st.tables, st.seq_lens, ws=st.ws)
+    out = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+    out2 = torch.zeros_like(out)
+    for step in range(steps):
+        q = torch.randn(L, B, Hq, D).bfloat16().cuda()
+        k = (1.5 * torch.randn(L, B, Hkv, D)).bfloat16().cuda()
+        v = (1.5 * torch.randn(L, B, Hkv, D)).bfloat16().cuda()
+        if step == 3:
+            k[0, 0, 0, :4] = torch.tensor([1e4, -1e4, 0.0, 3e-4]).bfloat16()      # saturation and underflow on the device
+        lt.decode_step(fus.shape, q, k, v, fus.tables, fus.mask, fus.seq_lens, out, fus.ws)
+        lt.kv_append(sep.shape, sep.mask, k, v, sep.seq_lens, sep.tables, ws=sep.ws)
+        lt.hybrid_decode_attn(sep.shape, q, sep.tables, sep.mask, sep.seq_lens, out2, sep.ws)
+        assert torch.equal(out, out2), step                                    # fused == append + attend, bit for bit
+        for l in range(L):
+            kc, kval = O.quantize_e4m3(f64(k[l]), scales[l, 0])
+            vc, vval = O.quantize_e4m3(f64(v[l]), scales[l, 1])
+            for b in range(B):
+                replays[b].append(l, kval[b], vval[b])
+                codes_hist[l][b] = np.concatenate([codes_hist[l][b], kc[b][:, None]], axis=1)
+                mx, rel = attn_errors(f64(out[l, b]), replays[b].attend(l, f64(q[l, b])))
+                assert mx <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (step, l, b, mx, rel)
+    assert lt.check(fus.ws) == 0 and lt.check(sep.ws) == 0
+    assert fus.seq_lens.cpu().tolist() == [n + steps for n in lens]
+    for l in range(L):
+        for st in (fus, sep):
+            for b, n in enumerate(lens):
+                for h in range(Hkv):
+                    hist = codes_hist[l][b][h]                                  # [n + steps, D] codes
+                    if mask[l]:
+                        ek, _ = O.stream_cache_after(hist, S, R)
+                        valid = O.ring_valid_slots(n + steps, S, R)
+                        assert np.array_equal(st.k_stream[l][b, h, :valid].cpu().numpy(), ek[:valid])
+                    else:
+                        assert np.array_equal(st.k_full[l][b, h, :n + steps].cpu().numpy(), hist)
+
+
+def test_fp8_shape_is_validated_and_scoring_refuses_8bit_keys():
+    sc = torch.full((2, 2), 0.02, dtype=torch.float32, device="cuda")
+    ok = lt.Shape(2, 1, 8, 2, 128, 4, 12, 64, lt.LT_BF16, 0.0, kv_fp8=1, kv_scales=sc)
+    assert lt.workspace_bytes(ok) > 0
+    for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=32)):
+        d = dict(ok.__dict__); d.update(kw)
+        with pytest.raises(lt.LtError):
+            lt.workspace_bytes(lt.Shape(**d))
+    k8 = [torch.zeros((1, 2, 64, 128), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    ws = torch.empty(lt.workspace_bytes(ok, 64, 8), dtype=torch.uint8, device="cuda")
+    with pytest.raises(lt.LtError) as e:
+        lt.lazy_scores(ok, torch.zeros((2, 1, 8, 8, 128), dtype=torch.bfloat16, device="cuda"), k8, 64, 8,
+                       torch.zeros((2, 1, 8), device="cuda"), ws)
+    assert e.value.status == 2
