@@ -88,22 +88,20 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float f16_lo(uint32_t x) { return __low2float(*reinterpret_cast<__half2*>(&x)); }
-__device__ __forceinline__ float f16_hi(uint32_t x) { return __high2float(*reinterpret_cast<__half2*>(&x)); }
-// Four E4M3 bytes -> four f16 whose value is the E4M3 value / 256, by moving bits only: an E4M3 byte
-// s.eeee.mmm placed at bits 15..8 and shifted so that eeee.mmm lands in f16's exponent / mantissa
-// field reads as 2^(e-15) (1 + m/8) instead of 2^(e-7) (1 + m/8), subnormals included (m/8 * 2^-14
-// instead of m/8 * 2^-6).  The factor 256 is folded into the per-layer scales.
-__device__ __forceinline__ void e4m3x4_to_f16x4_div256(uint32_t w, uint32_t& lo, uint32_t& hi) {
-  const uint32_t t0 = __byte_perm(w, 0u, 0x1404);  // byte 0 -> bits 15..8, byte 1 -> bits 31..24
-  const uint32_t t1 = __byte_perm(w, 0u, 0x3424);  // bytes 2, 3
-  lo = (t0 & 0x80008000u) | ((t0 >> 1) & 0x3f803f80u);
-  hi = (t1 & 0x80008000u) | ((t1 >> 1) & 0x3f803f80u);
+// Two E4M3 bytes of a 32-bit word -> two f16 whose value is the E4M3 value / 256, by moving bits only:
+// an E4M3 byte s.eeee.mmm placed at bits 15..8 and shifted so that eeee.mmm lands in f16's exponent /
+// mantissa field reads as 2^(e-15) (1 + m/8) instead of 2^(e-7) (1 + m/8), subnormals included
+// (m/8 * 2^-14 instead of m/8 * 2^-6).  The factor 256 is folded into the per-layer scales.
+// SEL picks the two bytes: 0x2404 bytes (0, 2), 0x3414 bytes (1, 3).
+// two E4M3 bytes (low byte first) -> two f16 with the hardware conversion (exact: every E4M3 value is an f16 value)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
+  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two_bytes, __NV_E4M3);
+  return (uint32_t)h.x | ((uint32_t)h.y << 16);
 }
-__device__ __forceinline__ uint32_t ld_shared_u32x4(uint32_t addr, uint32_t& y, uint32_t& z, uint32_t& w) {
-  uint32_t x;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(addr));
-  return x;
+template <uint32_t SEL>
+__device__ __forceinline__ uint32_t e4m3_pair_to_f16x2_div256(uint32_t w) {
+  const uint32_t t = __byte_perm(w, 0u, SEL);  // first byte -> bits 15..8, second byte -> bits 31..24
+  return (t & 0x80008000u) | ((t >> 1) & 0x3f803f80u);
 }
 __device__ __forceinline__ void st_shared_u32x4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
@@ -134,10 +132,18 @@ struct TileSrc {
 //
 // FP8 = true: the caches hold E4M3 bytes (rows of 128 B) with one scale per layer
 // for K and one for V.  A ring stage then holds the raw bytes of a tile (K rows,
-// then V rows); before the MMAs the warp expands the tile into a private 16-bit
-// buffer in the layout above (f16, by bit moves, as value / 256), Q and P are f16
-// as well, the K scale (x 256) is folded into the softmax scale and the V scale
-// (x 256) into the final normalisation.
+// then V rows, the 16-byte column c of row r at column c ^ (r & 7)) and the MMA
+// fragments are made from the bytes in registers, as f16 holding value / 256:
+//   K: ldmatrix on the bytes hands thread (g, c) the four bytes d = 4c .. 4c+3 of
+//      row g - an A fragment for a d order that Q's fragments simply follow;
+//   V: ldmatrix.trans on byte pairs hands it V[2c][2g], V[2c][2g+1], V[2c+1][2g],
+//      V[2c+1][2g+1]: bytes (0, 2) feed an MMA over the even d, bytes (1, 3) one
+//      over the odd d, so an accumulator tile owns d = 32 blk + 16 half + 2 g + parity.
+// K bytes become f16 through the conversion unit, V bytes through integer bit
+// moves that yield value / 256 (two pipes share the work).  Q and P are f16 as
+// well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
+// is folded into the softmax scale and the V scale (x 256) into the final
+// normalisation.  32-key tiles give every warp two independent MMA chains.
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
@@ -148,7 +154,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   constexpr int kRowBytes = FP8 ? kD : 2 * kD;             // one cached K or V row
   constexpr int RAW_BYTES = 2 * TILE * kD;                 // FP8: K rows + V rows of a tile as stored
   constexpr int RING_STAGE = FP8 ? RAW_BYTES : STAGE_BYTES;  // what one ring stage holds
-  constexpr int WARP_BYTES = NSTAGE * RING_STAGE + (FP8 ? STAGE_BYTES : 0);
+  constexpr int WARP_BYTES = NSTAGE * RING_STAGE;
   constexpr int RING_BYTES = WARPS * WARP_BYTES;
   constexpr int MERGE_BYTES = 2 * 8 * kD * 4 + 2 * WARPS * 8 * 4;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -167,13 +173,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
   const uint32_t wsm = smem_u32(smem) + warp * WARP_BYTES;
-  const uint32_t wconv = wsm + NSTAGE * RING_STAGE;  // FP8: the warp's expanded tile
   // lane-constant parts of the ldmatrix addresses
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8;  // K (A operand, not transposed)
   const int k_chk = lane >> 4;
   const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8;  // V (A operand, transposed)
   const int v_chk = (lane >> 3) & 1;
 
+  // d index of accumulator element (tile idx, row half) of this thread
+  auto dmap = [&](int idx, int half) {
+    return FP8 ? 32 * (idx >> 1) + 16 * half + 2 * gp + (idx & 1) : idx * 16 + gp + 8 * half;
+  };
   auto make_src = [&](const WorkItem& w) {
     TileSrc t;
     // contiguous: base of this (b, kv head); paged: base of kv head h inside page 0 of the layer's pool
@@ -234,7 +243,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         const int row = key_base + r;
         const bool valid = row < t.j1;
         const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
-        const uint32_t soff = r * kD + p * 16;
+        const uint32_t soff = r * kD + ((p ^ (r & 7)) << 4);
         if (row == t.new_row) {
           // the new token's row is quantised on the fly from k_new / v_new
           uint32_t q4[4];
@@ -262,29 +271,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       }
     }
   };
-  // FP8: expand the raw tile in ring stage `stage` into the warp's 16-bit buffer
-  auto expand_tile = [&](int stage) {
-    const uint32_t raw = wsm + stage * RING_STAGE;
-#pragma unroll
-    for (int kv = 0; kv < 2; ++kv) {
-#pragma unroll
-      for (int i = 0; i < TILE / 4; ++i) {
-        const int ci = i * 32 + lane;
-        const int r = ci >> 3, p = ci & 7;  // row, 16-byte chunk = 16 values d = 16p .. 16p + 15
-        uint32_t w1, w2, w3;
-        const uint32_t w0 = ld_shared_u32x4(raw + kv * TILE * kD + r * kD + p * 16, w1, w2, w3);
-        const uint32_t dst = wconv + kv * 2 * HALF_BYTES + (p >> 2) * HALF_BYTES + r * 128;
-        uint32_t h0, h1, h2, h3, h4, h5, h6, h7;
-        e4m3x4_to_f16x4_div256(w0, h0, h1);
-        e4m3x4_to_f16x4_div256(w1, h2, h3);
-        e4m3x4_to_f16x4_div256(w2, h4, h5);
-        e4m3x4_to_f16x4_div256(w3, h6, h7);
-        st_shared_u32x4(dst + ((((2 * p) & 7) ^ (r & 7)) << 4), h0, h1, h2, h3);
-        st_shared_u32x4(dst + ((((2 * p + 1) & 7) ^ (r & 7)) << 4), h4, h5, h6, h7);
-      }
-    }
-  };
-
   // The CTA's first two items are fixed; later ones come from the device counter.
   int cur = blockIdx.x, nxt = blockIdx.x + gridDim.x;
   WorkItem w;
@@ -325,7 +311,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     // per-layer scales of 8-bit caches: K's goes into the softmax scale, V's into the normalisation
     float cs_l = a.cs, v_scale = 1.f;
     if constexpr (FP8) {
-      cs_l = a.cs * a.s.kv_scales[2 * l] * 256.f;  // 256: the expanded tile holds value / 256
+      cs_l = a.cs * a.s.kv_scales[2 * l];  // K fragments hold the true values  // 256: the expanded tile holds value / 256
       v_scale = a.s.kv_scales[2 * l + 1] * 256.f;
     }
 
@@ -357,11 +343,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
       for (int ks8 = 0; ks8 < 8; ++ks8) {
         if (gp < G) {
-          qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
-          qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
-          if constexpr (FP8) {  // f16 operands: bf16 -> f16 is exact inside f16's range
-            qf[ks8][0] = pack_f16(bf16_lo(qf[ks8][0]), bf16_hi(qf[ks8][0]));
-            qf[ks8][1] = pack_f16(bf16_lo(qf[ks8][1]), bf16_hi(qf[ks8][1]));
+          if constexpr (FP8) {
+            // k-block ks8 covers d = 16 ks8 .. 16 ks8 + 15 in the order of the byte fragments:
+            // slots (2c, 2c+1) <-> d + 4c, 4c+1 and slots (2c+8, 2c+9) <-> d + 4c+2, 4c+3.
+            // f16 operands: bf16 -> f16 is exact inside f16's range.
+            const uint2 q4 = *reinterpret_cast<const uint2*>(qp + 16 * ks8 + 4 * c);
+            qf[ks8][0] = pack_f16(bf16_lo(q4.x), bf16_hi(q4.x));
+            qf[ks8][1] = pack_f16(bf16_lo(q4.y), bf16_hi(q4.y));
+          } else {
+            qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
+            qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
           }
         } else {
           qf[ks8][0] = 0u;
@@ -383,12 +374,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       issue_slot();
       cp_async_wait<NSTAGE - 1>();
       __syncwarp();              // all lanes' copies of this tile have landed
-      uint32_t st = wsm + (consumed % NSTAGE) * RING_STAGE;
-      if constexpr (FP8) {
-        expand_tile(consumed % NSTAGE);
-        __syncwarp();  // the expanded tile is complete before any lane's ldmatrix
-        st = wconv;
-      }
+      const uint32_t st = wsm + (consumed % NSTAGE) * RING_STAGE;
       ++consumed;
       const int key_base = src_cur.j0 + (warp + it * WARPS) * TILE;
 
@@ -398,13 +384,28 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       for (int mt = 0; mt < MT; ++mt) {
         sc[mt][0] = sc[mt][1] = sc[mt][2] = sc[mt][3] = 0.f;
         const int row = mt * 16 + k_row;
+        if constexpr (FP8) {
 #pragma unroll
-        for (int ks8 = 0; ks8 < 8; ++ks8) {
-          uint32_t af[4];
-          const int chunk = 2 * (ks8 & 3) + k_chk;
-          ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-          if constexpr (FP8) mma_f16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
-          else mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+          for (int blk = 0; blk < 4; ++blk) {  // 32 d per ldmatrix: matrices (rows 0-7 | 8-15) x (chunk 2 blk | 2 blk + 1)
+            uint32_t m[4];
+            const int chunk = 2 * blk + k_chk;
+            ldmatrix_x4(m, st + row * kD + ((chunk ^ (row & 7)) << 4));
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              // K goes through the conversion unit, V (below) through integer bit moves: two pipes share the work
+              const uint32_t af[4] = {e4m3x2_to_f16x2(m[2 * hf] & 0xffffu), e4m3x2_to_f16x2(m[2 * hf + 1] & 0xffffu),
+                                      e4m3x2_to_f16x2(m[2 * hf] >> 16), e4m3x2_to_f16x2(m[2 * hf + 1] >> 16)};
+              mma_f16(sc[mt], af, qf[2 * blk + hf][0], qf[2 * blk + hf][1]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int ks8 = 0; ks8 < 8; ++ks8) {
+            uint32_t af[4];
+            const int chunk = 2 * (ks8 & 3) + k_chk;
+            ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
+            mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+          }
         }
       }
       // ---- scale, mask the ragged tail, tile max per head ---------------------
@@ -445,31 +446,41 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         const float p2 = exp2f(sc[mt][2] - Mn0), p3 = exp2f(sc[mt][3] - Mn1);
         l0 += p0 + p2;
         l1 += p1 + p3;
-        uint32_t hi01, hi23, lo01, lo23;  // P as a 16-bit head and a 16-bit residual
-        if constexpr (FP8) {
-          hi01 = pack_f16(p0, p1);
-          hi23 = pack_f16(p2, p3);
-          lo01 = pack_f16(p0 - f16_lo(hi01), p1 - f16_hi(hi01));
-          lo23 = pack_f16(p2 - f16_lo(hi23), p3 - f16_hi(hi23));
-        } else {
-          hi01 = pack_bf16(p0, p1);
-          hi23 = pack_bf16(p2, p3);
-          lo01 = pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01));
-          lo23 = pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23));
-        }
+        // P for the B operand: one f16 term with 8-bit caches, a bf16 head and a bf16 residual otherwise
+        const uint32_t hi01 = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
+        const uint32_t hi23 = FP8 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
         const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
-        const uint32_t bl0 = movmatrix_trans(lo01), bl1 = movmatrix_trans(lo23);
-        const int row = mt * 16 + v_row;
+        uint32_t bl0 = 0u, bl1 = 0u;
+        if constexpr (!FP8) {
+          bl0 = movmatrix_trans(pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01)));
+          bl1 = movmatrix_trans(pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23)));
+        }
+        if constexpr (FP8) {
+          const int row = mt * 16 + k_row;  // same matrix order as K: (keys 0-7 | 8-15) x (chunk 2 blk | 2 blk + 1)
 #pragma unroll
-        for (int dt = 0; dt < 8; ++dt) {
-          uint32_t af[4];
-          const int chunk = 2 * (dt & 3) + v_chk;
-          ldmatrix_x4_trans(af,
-                            st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-          if constexpr (FP8) {
-            mma_f16(o[dt], af, bh0, bh1);
-            mma_f16(o[dt], af, bl0, bl1);
-          } else {
+          for (int blk = 0; blk < 4; ++blk) {
+            uint32_t m[4];
+            const int chunk = 2 * blk + k_chk;
+            ldmatrix_x4_trans(m, st + TILE * kD + row * kD + ((chunk ^ (row & 7)) << 4));
+            {  // even d: rows g <-> d = 32 blk + 2g (m0, m1), rows g + 8 <-> d = 32 blk + 16 + 2g (m2, m3)
+              const uint32_t af[4] = {e4m3_pair_to_f16x2_div256<0x2404>(m[0]), e4m3_pair_to_f16x2_div256<0x2404>(m[2]),
+                                      e4m3_pair_to_f16x2_div256<0x2404>(m[1]), e4m3_pair_to_f16x2_div256<0x2404>(m[3])};
+              mma_f16(o[2 * blk], af, bh0, bh1);
+            }
+            {  // odd d
+              const uint32_t af[4] = {e4m3_pair_to_f16x2_div256<0x3414>(m[0]), e4m3_pair_to_f16x2_div256<0x3414>(m[2]),
+                                      e4m3_pair_to_f16x2_div256<0x3414>(m[1]), e4m3_pair_to_f16x2_div256<0x3414>(m[3])};
+              mma_f16(o[2 * blk + 1], af, bh0, bh1);
+            }
+          }
+        } else {
+          const int row = mt * 16 + v_row;
+#pragma unroll
+          for (int dt = 0; dt < 8; ++dt) {
+            uint32_t af[4];
+            const int chunk = 2 * (dt & 3) + v_chk;
+            ldmatrix_x4_trans(af,
+                              st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
             mma_bf16(o[dt], af, bh0, bh1);
             mma_bf16(o[dt], af, bl0, bl1);
           }
@@ -520,16 +531,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         o[i][3] *= f1;
       }
     }
-    // element (head 2c + e, d = dt*16 + gp + 8*half) of a warp's O at buffer offset below
-    auto buf_at = [&](int which, int dt) { return sm_buf + which * (8 * kD) + (2 * c) * kD + dt * 16 + gp; };
+    // rows of heads 2c (and 2c + 1 at + kD) of a warp's O in merge buffer `which`
+    auto buf_at = [&](int which, int) { return sm_buf + which * (8 * kD) + (2 * c) * kD; };
     if (warp >= 2) {
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         float* p = buf_at(warp - 2, dt);
-        p[0] = o[dt][0];
-        p[kD] = o[dt][1];
-        p[8] = o[dt][2];
-        p[kD + 8] = o[dt][3];
+        p[dmap(dt, 0)] = o[dt][0];
+        p[kD + dmap(dt, 0)] = o[dt][1];
+        p[dmap(dt, 1)] = o[dt][2];
+        p[kD + dmap(dt, 1)] = o[dt][3];
       }
     }
     __syncthreads();
@@ -537,10 +548,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         const float* p = buf_at(warp, dt);
-        o[dt][0] += p[0];
-        o[dt][1] += p[kD];
-        o[dt][2] += p[8];
-        o[dt][3] += p[kD + 8];
+        o[dt][0] += p[dmap(dt, 0)];
+        o[dt][1] += p[kD + dmap(dt, 0)];
+        o[dt][2] += p[dmap(dt, 1)];
+        o[dt][3] += p[kD + dmap(dt, 1)];
       }
     }
     __syncthreads();  // buffer 0 has been read by warp 0 before warp 1 overwrites it
@@ -548,10 +559,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         float* p = buf_at(0, dt);
-        p[0] = o[dt][0];
-        p[kD] = o[dt][1];
-        p[8] = o[dt][2];
-        p[kD + 8] = o[dt][3];
+        p[dmap(dt, 0)] = o[dt][0];
+        p[kD + dmap(dt, 0)] = o[dt][1];
+        p[dmap(dt, 1)] = o[dt][2];
+        p[kD + dmap(dt, 1)] = o[dt][3];
       }
     }
     __syncthreads();
@@ -560,10 +571,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         const float* p = buf_at(0, dt);
-        o[dt][0] += p[0];
-        o[dt][1] += p[kD];
-        o[dt][2] += p[8];
-        o[dt][3] += p[kD + 8];
+        o[dt][0] += p[dmap(dt, 0)];
+        o[dt][1] += p[kD + dmap(dt, 0)];
+        o[dt][2] += p[dmap(dt, 1)];
+        o[dt][3] += p[kD + dmap(dt, 1)];
       }
       if (single) {
         // no partials: normalise and write the output of heads 2c, 2c + 1 directly
@@ -579,7 +590,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
               for (int half = 0; half < 2; ++half) {
                 const float num = o[dt][e + 2 * half];
                 const float r = den > 0.f ? (num / den) * v_scale : 0.f;
-                const long long oi = ob + (long long)g * kD + dt * 16 + gp + 8 * half;
+                const long long oi = ob + (long long)g * kD + dmap(dt, half);
                 if (a.out_dtype == LT_F32) ((float*)a.out)[oi] = r;
                 else ((__nv_bfloat16*)a.out)[oi] = __float2bfloat16_rn(r);
               }
@@ -592,11 +603,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
           if (g < G) {
-            float* po = a.part_o + (unit * G + g) * kD + gp;
+            float* po = a.part_o + (unit * G + g) * kD;
 #pragma unroll
             for (int dt = 0; dt < 8; ++dt) {
-              po[dt * 16] = o[dt][e];
-              po[dt * 16 + 8] = o[dt][e + 2];
+              po[dmap(dt, 0)] = o[dt][e];
+              po[dmap(dt, 1)] = o[dt][e + 2];
             }
             if (gp == 0) {
               a.part_ml[(unit * G + g) * 2] = e ? Mx1 : Mx0;
@@ -633,7 +644,7 @@ bool decode_mma_supported(const lt_shape& s) {
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int ring = FP8 ? WARPS * (NSTAGE * TILE * 256 + TILE * 512) : WARPS * NSTAGE * TILE * 512;
+  constexpr int ring = FP8 ? WARPS * NSTAGE * TILE * 256 : WARPS * NSTAGE * TILE * 512;
   constexpr int merge = 2 * 8 * 128 * 4 + 2 * WARPS * 8 * 4;
   static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
@@ -661,8 +672,8 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
-  // 8-bit caches: four raw stages (4 KB each) + the expanded tile = the 24 KB per warp of the 16-bit ring
-  if (a.s.kv_fp8) return launch_variant<16, 4, 4, 2, true>(a, kf, vf, ks, vs, st);
+  // 8-bit caches: three raw stages of 32 keys (8 KB) = the 24 KB per warp of the 16-bit ring
+  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true>(a, kf, vf, ks, vs, st);
   return launch_variant<16, 3, 4, 2, false>(a, kf, vf, ks, vs, st);
 }
 
