@@ -345,6 +345,11 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(cfg, wl)
 
+    # ---- the same step with paged and with 8-bit caches (detail only; last, it reuses the caches) ----
+    mask_hybrid = torch.zeros_like(wl.mask)
+    mask_hybrid[torch.as_tensor(wl.planted, device=device)] = 1
+    variants = run_variants(wl, mask_hybrid) if world == 1 else {}
+
     if rank == 0:
         hybrid_step_ms = decode_ms_total / (K * T)
         line = {
@@ -381,6 +386,7 @@ def run_ours(args):
                 "lazy_score_ms": float(ident_ms.mean()),
                 "lazy_score_lse_route_ms": lse_ms,
                 "lazy_score_routes_max_abs_diff": routes_diff,
+                "variants": variants,
                 "paper_context": "paper reports up to 2.17x whole-model throughput vs full attention on A100 "
                                  "(Mistral-7B, 16K, max batch); other hardware, not the target",
             },
@@ -388,6 +394,64 @@ def run_ours(args):
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_variants(wl, mask_hybrid):
+    """The same decode step on the same stack shape with (a) paged full caches
+    (128-token pages behind a shuffled block table) and (b) FP8 E4M3 caches with
+    per-layer scales.  Contents are random: the work does not depend on them.
+    Reported in `detail`; the headline stays the contiguous bf16 stack."""
+    cfg, lt, dev = wl.cfg, wl.lt, wl.device
+    L, B, Hq, Hkv, D = cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    C = cfg.n_sink + cfg.n_recent
+    q, k, v = wl.step_inputs[0]
+    out = torch.zeros_like(wl.out)
+    res = {}
+
+    def time_steps(shape, tables, ws, n0, steps=16):
+        seq = torch.full((B,), n0, dtype=torch.int32, device=dev)
+        for _ in range(3):
+            lt.decode_step(shape, q, k, v, tables, mask_hybrid, seq, out, ws)
+        torch.cuda.synchronize()
+        seq.fill_(n0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            lt.decode_step(shape, q, k, v, tables, mask_hybrid, seq, out, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        assert lt.check(ws) == 0
+        return e0.elapsed_time(e1) / steps
+
+    n_mean = cfg.n_ctx + 8.5
+    # (a) paged: the benchmark's own K/V tensors viewed as page pools (same bytes, other addressing)
+    page = 128
+    cap = wl.shape.full_capacity
+    if cap % page == 0:
+        pps = cap // page
+        n_pages = B * pps
+        table = torch.randperm(n_pages, device=dev)[: B * pps].view(B, pps).to(torch.int32).contiguous()
+        shape = lt.Shape(L, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16, page_size=page,
+                         pages_per_seq=pps, n_pages=n_pages, block_table=table)
+        pools_k = [t.view(n_pages, Hkv, page, D) for t in wl.k_full]
+        pools_v = [t.view(n_pages, Hkv, page, D) for t in wl.v_full]
+        tables = lt.LayerTables(shape, pools_k, pools_v, wl.k_stream, wl.v_stream)
+        ms = time_steps(shape, tables, wl.ws, cfg.n_ctx)
+        res["paged_128"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3),
+                            "gbs": algorithmic_bytes_decode(cfg, n_mean, cfg.n_lazy) / (ms * 1e-3) / 1e9}
+    # (b) FP8 caches: byte tensors of the same geometry
+    scales = torch.full((L, 2), 0.02, dtype=torch.float32, device=dev)
+    shape8 = lt.Shape(L, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16, kv_fp8=1, kv_scales=scales)
+    mk = lambda n: [torch.randint(0, 120, (B, Hkv, n, D), dtype=torch.uint8, device=dev) for _ in range(L)]
+    k8, v8, ks8, vs8 = mk(cap), mk(cap), mk(C), mk(C)
+    tables8 = lt.LayerTables(shape8, k8, v8, ks8, vs8)
+    ws8 = torch.empty(lt.workspace_bytes(shape8), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws8)
+    ms = time_steps(shape8, tables8, ws8, cfg.n_ctx)
+    kv8 = algorithmic_bytes_decode(cfg, n_mean, cfg.n_lazy) / 2          # one byte per cached element
+    res["fp8_caches"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs_of_8bit_bytes": kv8 / (ms * 1e-3) / 1e9}
+    del k8, v8, ks8, vs8, ws8
+    return res
 
 
 def run_e2e(wl, passes):
