@@ -108,7 +108,7 @@ def test_uniform_attention_closed_form(n, S, R, T):
     K = _rng(11).standard_normal((1, n, 8))
     sc = O.lazy_scores(np.zeros((2, T, 8)), K, S, R)
     assert np.max(np.abs(sc - _uniform_mass(n, S, R, T))) < 1e-13
-    # survey formula for one row, window not overlapping the sinks:
+    # closed form for one row when the window does not overlap the sinks:
     if S <= n - R:
         i = n - 1
         assert abs(_uniform_mass(n, S, R, 1) - (min(S, i + 1) + max(0, i - max(S, n - R) + 1)) / (i + 1)) < 1e-15
