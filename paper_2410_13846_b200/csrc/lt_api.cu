@@ -43,7 +43,9 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   // Measured on B200 (32K context, whole stack and one layer per call): long chunks win, per-item
   // hand-off costs more than an uneven last round; shorter chunks only pay when a launch has very few keys.
   p.min_chunk = 512;
-  p.max_chunk = 2048;
+  // 8-bit caches: that path is bound by SM-side work, where the hand-off between items (four CTA barriers) is
+  // pure loss: 8192-key chunks measured 9 % faster than 2048-key ones; the 16-bit path is flat from 2048 to 4096.
+  p.max_chunk = s.kv_fp8 ? 8192 : 2048;
   p.target_items = 592;
   // chunk = clamp(ceil(keys / target), min, max) gives at most target + units items
   // when it is not clamped at max, and units * ceil(n_max / max) when it is
