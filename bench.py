@@ -594,6 +594,40 @@ def run_profile_case(args):
                       "pass_s": time.perf_counter() - t0, "mask": wl.mask.cpu().tolist()}))
 
 
+def run_profile_case_fp8(args):
+    """Small case of the decode step with FP8 caches for profiler captures: 4
+    layers (2 lazy) of the benchmark's stack shape, byte caches with random
+    codes (2.3 GB on the device), a few decode steps, nothing else."""
+    assert torch.cuda.is_available()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    from paper_2410_13846_b200 import build
+    build.build_library()
+    import paper_2410_13846_b200 as lt
+    from synth import CONFIGS
+    cfg = CONFIGS[WORKLOAD].scaled(n_layers=4, n_lazy=2)
+    L, B, Hq, Hkv, D = cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    C, cap = cfg.n_sink + cfg.n_recent, cfg.n_ctx + 64
+    scales = torch.full((L, 2), 0.02, dtype=torch.float32, device=dev)
+    shape = lt.Shape(L, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16, kv_fp8=1, kv_scales=scales)
+    mk = lambda n: [torch.randint(0, 120, (B, Hkv, n, D), dtype=torch.uint8, device=dev) for _ in range(L)]
+    tables = lt.LayerTables(shape, mk(cap), mk(cap), mk(C), mk(C))
+    ws = torch.empty(lt.workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws)
+    mask = torch.tensor([0, 1, 1, 0], dtype=torch.uint8, device=dev)
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
+    q = torch.randn((L, B, Hq, D), device=dev).bfloat16()
+    k = torch.randn((L, B, Hkv, D), device=dev).bfloat16()
+    out = torch.zeros_like(q)
+    t0 = time.perf_counter()
+    for _ in range(args.profile_case_fp8):
+        lt.decode_step(shape, q, k, k, tables, mask, seq, out, ws)
+    torch.cuda.synchronize()
+    assert lt.check(ws) == 0
+    print(json.dumps({"profile_case": "fp8 caches, " + cfg.name, "layers": L, "decode_steps": args.profile_case_fp8,
+                      "run_s": time.perf_counter() - t0}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -603,8 +637,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-case", type=int, default=0, metavar="DECODE_STEPS",
                     help="run the 4-layer small case with this many decode steps per pass (for ncu) and exit")
+    ap.add_argument("--profile-case-fp8", type=int, default=0, metavar="DECODE_STEPS",
+                    help="run the 4-layer small case of the decode step with FP8 caches (for ncu) and exit")
     args = ap.parse_args()
-    if args.profile_case > 0:
+    if args.profile_case_fp8 > 0:
+        run_profile_case_fp8(args)
+    elif args.profile_case > 0:
         run_profile_case(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -139,8 +139,10 @@ struct TileSrc {
 //   V: ldmatrix.trans on byte pairs hands it V[2c][2g], V[2c][2g+1], V[2c+1][2g],
 //      V[2c+1][2g+1]: bytes (0, 2) feed an MMA over the even d, bytes (1, 3) one
 //      over the odd d, so an accumulator tile owns d = 32 blk + 16 half + 2 g + parity.
-// K bytes become f16 through the conversion unit, V bytes through integer bit
-// moves that yield value / 256 (two pipes share the work).  Q and P are f16 as
+// K bytes become f16 with the conversion instruction (one per byte pair), V
+// bytes - whose pairs are not adjacent - with integer bit moves that yield
+// value / 256; both run on the integer pipe, which is what bounds this path.
+// Q and P are f16 as
 // well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
 // is folded into the softmax scale and the V scale (x 256) into the final
 // normalisation.  32-key tiles give every warp two independent MMA chains.
@@ -392,7 +394,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
             ldmatrix_x4(m, st + row * kD + ((chunk ^ (row & 7)) << 4));
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-              // K goes through the conversion unit, V (below) through integer bit moves: two pipes share the work
+              // adjacent byte pairs: one conversion instruction each
               const uint32_t af[4] = {e4m3x2_to_f16x2(m[2 * hf] & 0xffffu), e4m3x2_to_f16x2(m[2 * hf + 1] & 0xffffu),
                                       e4m3x2_to_f16x2(m[2 * hf] >> 16), e4m3x2_to_f16x2(m[2 * hf + 1] >> 16)};
               mma_f16(sc[mt], af, qf[2 * blk + hf][0], qf[2 * blk + hf][1]);
