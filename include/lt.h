@@ -13,8 +13,9 @@
  * Conventions
  *   - Every function returns an lt_status; nothing aborts, throws or traps.
  *   - The caller owns all memory.  The library allocates nothing on the
- *     device, keeps no state between calls and never synchronises the device
- *     unless a function says so.  All device work is enqueued on `stream`
+ *     device, keeps no state between calls (beyond device properties it looks
+ *     up once per device) and never synchronises the device unless a function
+ *     says so.  All device work is enqueued on `stream`
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
  *   - "dev" marks a device pointer, "host" a host pointer.
  *   - Layer tables (k_full, v_full, k_stream, v_stream) are HOST arrays of
@@ -67,6 +68,7 @@ enum { LT_F32 = 0, LT_BF16 = 1 };
 #define LT_DEVERR_LEN_CLAMPED 4u      /* attend: seq_len > full_capacity; clamped */
 #define LT_DEVERR_TIMEOUT 8u          /* scoring: a bounded wait inside a kernel expired; scores invalid */
 
+/* Zero-initialise the struct and set what you need: every field after softmax_scale has a zero default. */
 typedef struct lt_shape {
   int32_t n_layers;      /* L, 1..LT_MAX_LAYERS */
   int32_t batch;         /* B >= 1 */
@@ -160,8 +162,8 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
 
 /*
  * Lazy ratio with the denominator given (Section 5.1: FlashAttention's prefill
- * already produced the log-sum-exp of every attention row, so "we only need to
- * recompute the streaming attention score", a constant-size product; Table 1).
+ * already produced the log-sum-exp of every attention row, so only the product of
+ * the tail queries with the kept keys is left to compute, a constant-size one; Table 1).
  * Same result as lt_lazy_scores, but only the kept keys are read:
  *   lse     dev float [L][B][Hq][w_last]: natural logarithm of
  *           sum_{j <= i} exp(scale * q_i . k_j) for the tail rows
@@ -190,8 +192,8 @@ lt_status lt_select_lazy(const float* scores /* dev [L][B][Hq] */, int32_t n_lay
                          float* layer_ratio /* dev [L] or NULL */, void* stream);
 
 /*
- * Per-prompt selection (Section 4: the layers that are lazy "vary according to
- * different prompts"): for every batch row b, r = mean over [Hq] of
+ * Per-prompt selection (Section 4: which layers are lazy differs from prompt to
+ * prompt): for every batch row b, r = mean over [Hq] of
  * scores[l][b] and the n_lazy layers with the largest r become lazy for that
  * prompt.  layer_mask dev uint8 [B][L], layer_ratio dev float [B][L] or NULL.
  * Use the result with shape.per_sequence_mask = 1.
@@ -202,9 +204,8 @@ lt_status lt_select_lazy_per_seq(const float* scores /* dev [L][B][Hq] */, int32
 
 /*
  * Frequency-count choice of the lazy layers over many samples (Section 5.2,
- * LightTransfer-Train: every training sample reveals its own lazy layers, "we
- * then compute the frequency for each layer and select those with the highest
- * lazy layer counts").
+ * LightTransfer-Train: every training sample reveals its own lazy layers; the
+ * layers that are lazy in the most samples are chosen).
  *   sample_masks  dev uint8 [n_samples][L]: per-sample masks, e.g. the rows that
  *                 lt_select_lazy_per_seq wrote for successive batches
  *   layer_mask    dev uint8 [L]: 1 for the n_lazy layers with the highest counts,
@@ -236,8 +237,8 @@ lt_status lt_select_lazy_push(const float* layer_scores /* dev */, int32_t layer
                               void* stream);
 
 /*
- * Prefill -> decode compaction of the lazy layers (Section 5.1: "retain only
- * the KV caches corresponding to {X_initial, X_recent} and discard others";
+ * Prefill -> decode compaction of the lazy layers (Section 5.1: a lazy
+ * layer keeps the KV of its initial and its most recent tokens and drops the rest;
  * Fig. 3).  For every layer with mask 1 and every (b, kv head), prompt rows
  * p in {0 .. min(n_sink,n)-1} U {max(n_sink, n - n_recent) .. n-1}, n = seq_lens[b],
  * are copied bit for bit from the full cache to row lt_ring_slot(p) of the
@@ -262,7 +263,7 @@ lt_status lt_stream_init_layer(const lt_shape* shape, const uint8_t* layer_mask 
                                void* ws /* dev, for the error word; may be NULL */, void* stream);
 
 /*
- * Per-step KV append (Section 3: decoding "saves their KV cache"; Section 5.1
+ * Per-step KV append (Section 3: decoding stores the KV of every generated token; Section 5.1
  * for the lazy layers).  With p = seq_lens[b]:
  *   mask 0: k_new[l][b][h][:] -> full cache row p        (skipped and flagged
  *           LT_DEVERR_POS_OUT_OF_RANGE when p >= full_capacity)

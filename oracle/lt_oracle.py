@@ -124,8 +124,8 @@ def full_attention(q, K, V, scale=None):
 def kept_positions(n: int, n_sink: int, n_recent: int):
     """Boolean vector over positions 0..n-1: True where the key is kept by a
     lazy layer, i.e. j < n_sink or j >= n - n_recent (a set union, so an
-    overlap is not counted twice).  (Section 5.1; Appendix E, "first 4 and the
-    last 1020 tokens".)
+    overlap is not counted twice).  (Section 5.1; Appendix E: the first 4 and the last
+    1020 tokens in the paper's setting.)
     """
     j = np.arange(n)
     return (j < n_sink) | (j >= n - n_recent)
@@ -243,8 +243,8 @@ def causal_lse(Q_tail, K, scale=None):
 
 
 def lazy_scores_from_lse(Q_tail, K, lse, n_sink: int, n_recent: int, scale=None):
-    """O3 as deployed (Section 5.1, "only need to recompute the streaming
-    attention score"; Table 1): the denominator of every tail row comes in as
+    """O3 as deployed (Section 5.1: with the prefill's denominators at hand only
+    the window block is recomputed; Table 1): the denominator of every tail row comes in as
     its log-sum-exp, and only the logits of the kept keys {j < n_sink} U
     {j >= n - n_recent} (causally visible ones) are computed:
         mass_t = sum_{j kept, j <= i} exp(scale * q_t . k_j - lse[hq, t]),
@@ -271,7 +271,7 @@ def lazy_scores_from_lse(Q_tail, K, lse, n_sink: int, n_recent: int, scale=None)
 
 def lazy_scores_per_row_window(Q_tail, K, n_sink: int, n_recent: int, scale=None):
     """O3 under the other reading of X_recent (Appendix E: the mask M_lazy keeps,
-    for row i, "the first 4 and the last 1020 tokens" of [i]): the recent set of
+    for row i, the first few and the most recent tokens of [i]): the recent set of
     the tail query at position i is {i - n_recent + 1 .. i} instead of the fixed
     block {n - n_recent .. n - 1}.  Both readings agree for the last query.
     """
@@ -360,8 +360,8 @@ def select_lazy_priority_queue_trace(ratios, n_full: int):
 
 
 def select_lazy_per_sequence(scores, n_lazy: int):
-    """O4 per prompt (Section 4: the lazy layers "vary according to different
-    prompts"): row b of the result is select_lazy on that batch row's scores
+    """O4 per prompt (Section 4: which layers are lazy differs from prompt to
+    prompt): row b of the result is select_lazy on that batch row's scores
     alone.  scores [L, B, Hq] -> mask uint8 [B, L], r float64 [B, L].
     """
     scores = _f64(scores)
