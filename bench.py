@@ -455,8 +455,9 @@ def run_variants(wl, mask_hybrid):
 
 
 def run_e2e(wl, passes):
-    """Same pass through the public API with HOST buffers: every step copies its
-    inputs from pinned host memory and reads its result back."""
+    """Same pass through the C ABI with HOST buffers: every step hands pinned host
+    q / k_new / v_new to lt_decode_step_host, which copies them in, runs the step
+    and copies the output back; the caller waits for it before the next step."""
     cfg, lt = wl.cfg, wl.lt
     pin = lambda t: t.cpu().pin_memory()  # noqa: E731
     h_qtail = pin(wl.q_tail)
@@ -474,9 +475,7 @@ def run_e2e(wl, passes):
         h_mask.copy_(wl.mask, non_blocking=True)
         for i in range(cfg.steps):
             hq, hk, hv = h_steps[i % len(h_steps)]
-            d_q.copy_(hq, non_blocking=True); d_k.copy_(hk, non_blocking=True); d_v.copy_(hv, non_blocking=True)
-            lt.decode_step(wl.shape, d_q, d_k, d_v, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
-            h_out.copy_(wl.out, non_blocking=True)
+            lt.decode_step_host(wl.shape, hq, hk, hv, h_out, d_q, d_k, d_v, wl.out, wl.tables, wl.mask, wl.seq, wl.ws)
             torch.cuda.current_stream().synchronize()       # the caller consumes the step's result
 
     one_pass()

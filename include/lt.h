@@ -333,6 +333,25 @@ lt_status lt_decode_step(const lt_shape* shape, const void* q /* dev */, const v
                          void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
+ * lt_decode_step for a caller whose step inputs and outputs live in HOST
+ * memory (the same operation, Section 3; the sampler of a serving loop reads
+ * the step's result on the host).  Enqueues on `stream`: q_host, k_new_host,
+ * v_new_host -> the device staging buffers, the whole-stack lt_decode_step
+ * (all layers, seq_lens advanced), out staging -> out_host.  Does not
+ * synchronise: out_host is valid once the stream has reached this point.
+ *   q_host, k_new_host, v_new_host, out_host  host, layouts and dtypes as in
+ *       lt_decode_step; page-locked memory keeps the copies asynchronous
+ *   q_dev, k_new_dev, v_new_dev, out_dev      dev staging buffers of the same
+ *       sizes, owned by the caller
+ */
+lt_status lt_decode_step_host(const lt_shape* shape, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* out_host, void* q_dev, void* k_new_dev,
+                              void* v_new_dev, void* out_dev, void* const* k_full, void* const* v_full,
+                              void* const* k_stream, void* const* v_stream /* host tables */,
+                              const uint8_t* layer_mask /* dev */, int32_t* seq_lens /* dev [B] */,
+                              int32_t out_dtype, void* ws /* dev */, size_t ws_bytes, void* stream);
+
+/*
  * The decode-attention step for callers that cannot allocate device memory.
  * (No counterpart in the paper: this is a deployment convenience of the library.)
  *

@@ -131,6 +131,8 @@ def lib() -> C.CDLL:
     L.lt_hybrid_decode_attn.argtypes = [shp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
     L.lt_decode_step.restype = i32
     L.lt_decode_step.argtypes = [shp, vp, vp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
+    L.lt_decode_step_host.restype = i32
+    L.lt_decode_step_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, tab, tab, tab, tab, vp, vp, i32, vp, sz, vp]
     _LIB = L
     return L
 
@@ -295,6 +297,23 @@ def decode_step(shape: Shape, q, k_new, v_new, tables: LayerTables, layer_mask, 
                              tables.k_stream, tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
                              layer_begin, cnt, 1 if advance_seq_lens else 0, _ptr(ws),
                              ws.numel() * ws.element_size(), _stream(stream)), "lt_decode_step")
+
+
+def decode_step_host(shape: Shape, q_host, k_new_host, v_new_host, out_host, q_dev, k_new_dev, v_new_dev, out_dev,
+                     tables: LayerTables, layer_mask, seq_lens, ws, stream=None):
+    """lt_decode_step_host: the whole-stack step with HOST inputs and output (host tensors, ideally pinned)
+    through caller-owned device staging tensors.  Asynchronous on the stream."""
+    import torch
+    for t in (q_host, k_new_host, v_new_host, out_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    out_dtype = LT_F32 if out_dev.dtype == torch.float32 else LT_BF16
+    hp = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
+    _ok(lib().lt_decode_step_host(C.byref(shape.c()), hp(q_host), hp(k_new_host), hp(v_new_host), hp(out_host),
+                                  _ptr(q_dev), _ptr(k_new_dev), _ptr(v_new_dev), _ptr(out_dev), tables.k_full,
+                                  tables.v_full, tables.k_stream, tables.v_stream, _ptr(layer_mask), _ptr(seq_lens),
+                                  out_dtype, _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+        "lt_decode_step_host")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

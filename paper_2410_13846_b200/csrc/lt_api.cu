@@ -422,4 +422,30 @@ lt_status lt_decode_step(const lt_shape* shape, const void* q, const void* k_new
                      layer_begin, layer_count, 1, advance_seq_lens ? 1 : 0, ws, ws_bytes, stream);
 }
 
+lt_status lt_decode_step_host(const lt_shape* shape, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* out_host, void* q_dev, void* k_new_dev, void* v_new_dev,
+                              void* out_dev, void* const* k_full, void* const* v_full, void* const* k_stream,
+                              void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, int32_t out_dtype,
+                              void* ws, size_t ws_bytes, void* stream) {
+  lt_status st = validate_shape(shape);
+  if (st != LT_OK) return st;
+  if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_new_dev || !v_new_dev || !out_dev)
+    return LT_ERR_INVALID_ARG;
+  if (out_dtype != LT_F32 && out_dtype != LT_BF16) return LT_ERR_UNSUPPORTED;
+  const size_t e = elem_bytes(shape->dtype);
+  const size_t rows = (size_t)shape->n_layers * shape->batch;
+  const size_t q_bytes = rows * shape->n_q_heads * shape->head_dim * e;
+  const size_t kv_bytes = rows * shape->n_kv_heads * shape->head_dim * e;
+  const size_t out_bytes = rows * shape->n_q_heads * shape->head_dim * (out_dtype == LT_F32 ? 4 : 2);
+  cudaStream_t cs = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LT_ERR_CUDA;
+  if (cudaMemcpyAsync(k_new_dev, k_new_host, kv_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LT_ERR_CUDA;
+  if (cudaMemcpyAsync(v_new_dev, v_new_host, kv_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LT_ERR_CUDA;
+  st = lt_decode_step(shape, q_dev, k_new_dev, v_new_dev, k_full, v_full, k_stream, v_stream, layer_mask, seq_lens,
+                      out_dev, out_dtype, 0, shape->n_layers, 1, ws, ws_bytes, stream);
+  if (st != LT_OK) return st;
+  if (cudaMemcpyAsync(out_host, out_dev, out_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LT_ERR_CUDA;
+  return LT_OK;
+}
+
 }  // extern "C"

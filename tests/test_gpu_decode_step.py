@@ -153,3 +153,28 @@ def test_large_batch_is_split_into_launches_by_layers():
         lt.decode_step(fus.shape, q, k, v, fus.tables, fus.mask, fus.seq_lens, out, fus.ws)
         assert torch.equal(out, ref) and torch.equal(fus.seq_lens, sep.seq_lens)
     assert lt.check(fus.ws) == 0
+
+
+def test_host_buffer_step_equals_device_step():
+    """lt_decode_step_host: pinned host inputs in, host output back, same bits as the device-pointer call."""
+    L, B, Hq, Hkv, D, S, R = 3, 2, 8, 2, 128, 4, 12
+    lens, cap = [40, 9], 64
+    dev, host = _two_stacks(L, B, Hq, Hkv, D, S, R, cap, torch.bfloat16, lens, [0, 1, 0], seed=12)
+    g = torch.Generator().manual_seed(13)
+    d_q = torch.empty(L, B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    d_k = torch.empty(L, B, Hkv, D, dtype=torch.bfloat16, device="cuda"); d_v = torch.empty_like(d_k)
+    d_out = torch.empty(L, B, Hq, D, dtype=torch.float32, device="cuda")
+    h_out = torch.empty(L, B, Hq, D, dtype=torch.float32).pin_memory()
+    ref = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+    for step in range(5):
+        q = torch.randn(L, B, Hq, D, generator=g).bfloat16().pin_memory()
+        k = torch.randn(L, B, Hkv, D, generator=g).bfloat16().pin_memory()
+        v = torch.randn(L, B, Hkv, D, generator=g).bfloat16().pin_memory()
+        lt.decode_step(dev.shape, q.cuda(), k.cuda(), v.cuda(), dev.tables, dev.mask, dev.seq_lens, ref, dev.ws)
+        lt.decode_step_host(host.shape, q, k, v, h_out, d_q, d_k, d_v, d_out, host.tables, host.mask, host.seq_lens,
+                            host.ws)
+        torch.cuda.synchronize()
+        assert torch.equal(h_out, ref.cpu()), step
+    assert torch.equal(host.seq_lens, dev.seq_lens) and lt.check(host.ws) == 0
+    for l in range(L):
+        assert torch.equal(host.k_full[l], dev.k_full[l]) and torch.equal(host.k_stream[l], dev.k_stream[l])
