@@ -102,7 +102,8 @@ typedef struct lt_shape {
      v_new and out stay in `dtype`.  A stored byte c of layer l means E4M3(c) * kv_scales[l][0] for K and
      * kv_scales[l][1] for V; lt_kv_append / lt_decode_step store code(x) = E4M3 nearest to
      float32(x) / scale (float32 division, round to nearest even, saturating at +-448).  Needs
-     dtype = LT_BF16, head_dim = 128 and a query group of at most 8.  lt_lazy_scores and lt_lazy_scores_lse
+     dtype = LT_BF16, head_dim = 128 and a query group of at most 8; the kernels take q through f16, so
+     |q| must stay below 65504.  lt_lazy_scores and lt_lazy_scores_lse
      do not read 8-bit keys: score from the prefill's 16-bit keys with a shape whose kv_fp8 is 0. */
   int32_t kv_fp8;
   int32_t reserved2_;      /* must be 0 */
