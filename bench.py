@@ -39,7 +39,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes of one decode-kernel launch from the committed ncu capture, as a
 # ratio to the algorithmic bytes of that launch (profiles/); None until measured.
-NCU_TRAFFIC_RATIO = 1.005  # profiles/decode_mma_kernel__llama3_8b_32k_4layer_small_case.md
+NCU_TRAFFIC_RATIO = 1.004  # profiles/decode_mma_kernel__llama3_8b_32k_full_stack_dram_bytes.md (full-size launches)
 
 
 def _peaks():
