@@ -76,6 +76,12 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
   return y;
 }
+// One MUFU instruction: 2^x, relative error 2^-22, 2^(-inf) = 0, results below 2^-126 flush to zero.
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
 // lower 16 bits <- lo, upper <- hi
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -401,13 +407,18 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
             }
           }
         } else {
+          // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
+          float sc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int ks8 = 0; ks8 < 8; ++ks8) {
             uint32_t af[4];
             const int chunk = 2 * (ks8 & 3) + k_chk;
             ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
-            mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
+            if (ks8 & 1) mma_bf16(sc2, af, qf[ks8][0], qf[ks8][1]);
+            else mma_bf16(sc[mt], af, qf[ks8][0], qf[ks8][1]);
           }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) sc[mt][i] += sc2[i];
         }
       }
       // ---- scale, mask the ragged tail, tile max per head ---------------------
@@ -429,7 +440,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
       }
       const float Mn0 = fmaxf(M0, mx0), Mn1 = fmaxf(M1, mx1);
-      const float corr0 = exp2f(M0 - Mn0), corr1 = exp2f(M1 - Mn1);
+      const float corr0 = ex2(M0 - Mn0), corr1 = ex2(M1 - Mn1);
       M0 = Mn0;
       M1 = Mn1;
       l0 *= corr0;
@@ -444,8 +455,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       // ---- P = 2^(t - M), O^T += V^T P ---------------------------------------
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
-        const float p0 = exp2f(sc[mt][0] - Mn0), p1 = exp2f(sc[mt][1] - Mn1);
-        const float p2 = exp2f(sc[mt][2] - Mn0), p3 = exp2f(sc[mt][3] - Mn1);
+        const float p0 = ex2(sc[mt][0] - Mn0), p1 = ex2(sc[mt][1] - Mn1);
+        const float p2 = ex2(sc[mt][2] - Mn0), p3 = ex2(sc[mt][3] - Mn1);
         l0 += p0 + p2;
         l1 += p1 + p3;
         // P for the B operand: one f16 term with 8-bit caches, a bf16 head and a bf16 residual otherwise
