@@ -117,20 +117,21 @@ struct WorkList {
       prefix[e + 1] = items;  // turned into the prefix below
       run += items;
     }
-    __shared__ int thread_sum[256];  // blockDim.x <= 256
-    thread_sum[threadIdx.x] = run;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int acc = 0;
-      for (int t = 0; t < (int)blockDim.x; ++t) {
-        const int v = thread_sum[t];
-        thread_sum[t] = acc;
-        acc += v;
-      }
-      prefix[0] = 0;
+    // block-wide exclusive scan of the per-thread sums: shuffles inside a warp, then the warp totals
+    __shared__ int warp_total[8];  // blockDim.x <= 256
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    int incl = run;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += t;
     }
+    if (lane == 31) warp_total[wid] = incl;
+    if (threadIdx.x == 0) prefix[0] = 0;
     __syncthreads();
-    int acc = thread_sum[threadIdx.x];
+    int before = 0;
+    for (int w = 0; w < wid; ++w) before += warp_total[w];
+    int acc = before + incl - run;
     for (int e = e0; e < e1; ++e) {
       acc += prefix[e + 1];
       prefix[e + 1] = acc;
