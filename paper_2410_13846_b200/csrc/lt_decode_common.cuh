@@ -171,7 +171,7 @@ struct WorkList {
     w.c = rem - w.h * w.nc;
     w.slot0 = idx - w.c;
     int len = (w.n + w.nc - 1) / w.nc;  // balanced chunks: no tiny last chunk
-    if (s.page_size > 0) len = (len + 15) & ~15;  // paged caches: a 16-key tile never straddles two pages
+    if (s.page_size > 0) len = (len + 31) & ~31;  // paged caches: a 16- or 32-key tile never straddles two pages
     w.j0 = min(w.n, w.c * len);
     w.j1 = min(w.n, w.j0 + len);
     w.new_row = -1;

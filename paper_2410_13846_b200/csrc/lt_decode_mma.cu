@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     return t;
   };
   // copy this warp's idx-th tile of `t` into ring stage `stage` (no commit)
-  // row of key `row` relative to t.Kb / t.Vb (a paged chunk starts on a multiple of 16, so a tile has one page)
+  // row of key `row` relative to t.Kb / t.Vb (a paged chunk starts on a multiple of 32, so a tile has one page)
   auto cache_row = [&](const TileSrc& t, int row) -> long long {
     if (t.tbl_off < 0) return row;
     const int page = s.block_table[t.tbl_off + row / s.page_size];

@@ -105,3 +105,52 @@ def test_fp8_shape_is_validated_and_scoring_refuses_8bit_keys():
         lt.lazy_scores(ok, torch.zeros((2, 1, 8, 8, 128), dtype=torch.bfloat16, device="cuda"), k8, 64, 8,
                        torch.zeros((2, 1, 8), device="cuda"), ws)
     assert e.value.status == 2
+
+
+def test_fp8_with_paged_full_caches():
+    """Both options together: E4M3 pools behind a block table; 32-key tiles must not straddle pages."""
+    torch.manual_seed(35)
+    g = np.random.default_rng(35)
+    L, B, Hq, Hkv, D, S, R, page, pps = 2, 2, 8, 2, 128, 4, 28, 128, 6
+    cap = page * pps
+    lens, steps = [600, 250], 12
+    mask = np.array([0, 1], dtype=np.uint8)
+    scales = g.uniform(0.015, 0.04, size=(L, 2)).astype(np.float32)
+    n_pages = B * pps + 2
+    table = torch.randperm(n_pages)[: B * pps].view(B, pps).to(torch.int32).cuda().contiguous()
+    sc = torch.from_numpy(scales).cuda().contiguous()
+    shape = lt.Shape(L, B, Hq, Hkv, D, S, R, cap, lt.LT_BF16, 0.0, page_size=page, pages_per_seq=pps, n_pages=n_pages,
+                     block_table=table, kv_fp8=1, kv_scales=sc)
+    k_pool = [torch.zeros((n_pages, Hkv, page, D), dtype=torch.uint8, device="cuda") for _ in range(L)]
+    v_pool = [torch.zeros((n_pages, Hkv, page, D), dtype=torch.uint8, device="cuda") for _ in range(L)]
+    k_str = [torch.zeros((B, Hkv, S + R, D), dtype=torch.uint8, device="cuda") for _ in range(L)]
+    v_str = [torch.zeros((B, Hkv, S + R, D), dtype=torch.uint8, device="cuda") for _ in range(L)]
+    tables = lt.LayerTables(shape, k_pool, v_pool, k_str, v_str)
+    ws = torch.empty(lt.workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    lt.workspace_init(ws)
+    replays = [O.HybridReplay(mask, S, R) for _ in range(B)]
+    tab = table.cpu()
+    for l in range(L):
+        hk = torch.randn(B, Hkv, cap, D).bfloat16(); hv = torch.randn(B, Hkv, cap, D).bfloat16()
+        kc, kval = O.quantize_e4m3(f64(hk), scales[l, 0]); vc, vval = O.quantize_e4m3(f64(hv), scales[l, 1])
+        for b in range(B):
+            for p in range(pps):
+                sl = slice(p * page, (p + 1) * page)
+                k_pool[l][int(tab[b, p])] = torch.from_numpy(kc[b, :, sl]).cuda()
+                v_pool[l][int(tab[b, p])] = torch.from_numpy(vc[b, :, sl]).cuda()
+            replays[b].load_prompt(l, kval[b, :, :lens[b]], vval[b, :, :lens[b]])
+    dmask = torch.from_numpy(mask).cuda()
+    seq = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    lt.stream_init(shape, dmask, tables, seq, ws=ws)
+    out = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+    for step in range(steps):
+        q = torch.randn(L, B, Hq, D).bfloat16().cuda()
+        k = torch.randn(L, B, Hkv, D).bfloat16().cuda(); v = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        lt.decode_step(shape, q, k, v, tables, dmask, seq, out, ws)
+        for l in range(L):
+            _, kval = O.quantize_e4m3(f64(k[l]), scales[l, 0]); _, vval = O.quantize_e4m3(f64(v[l]), scales[l, 1])
+            for b in range(B):
+                replays[b].append(l, kval[b], vval[b])
+                mx, rel = attn_errors(f64(out[l, b]), replays[b].attend(l, f64(q[l, b])))
+                assert mx <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (step, l, b, mx, rel)
+    assert lt.check(ws) == 0 and seq.cpu().tolist() == [n + steps for n in lens]
