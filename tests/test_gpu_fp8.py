@@ -154,3 +154,47 @@ def test_fp8_with_paged_full_caches():
                 mx, rel = attn_errors(f64(out[l, b]), replays[b].attend(l, f64(q[l, b])))
                 assert mx <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (step, l, b, mx, rel)
     assert lt.check(ws) == 0 and seq.cpu().tolist() == [n + steps for n in lens]
+
+
+def test_fp8_long_context_sampled_units():
+    """Enough keys that a launch uses its longest (8192-key) chunks and several of them per unit;
+    sampled (layer, batch row, kv head) units against the oracle on the dequantised values."""
+    torch.manual_seed(37)
+    g = np.random.default_rng(37)
+    L, B, Hq, Hkv, D, S, R = 4, 4, 32, 8, 128, 4, 2044
+    n0, steps = 40000, 2
+    cap = n0 + steps
+    mask = np.array([0, 1, 0, 1], dtype=np.uint8)
+    scales = g.uniform(0.02, 0.04, size=(L, 2)).astype(np.float32)
+    st = Fp8Stack(L, B, Hq, Hkv, S, R, cap, scales)
+    table = torch.from_numpy(O.e4m3_values()).float().cuda()                 # code -> value, for the sampled read-back
+    for l in range(L):
+        st.k_full[l].copy_(torch.randint(0, 0x7F, st.k_full[l].shape, dtype=torch.uint8, device="cuda")
+                           | (torch.randint(0, 2, st.k_full[l].shape, dtype=torch.uint8, device="cuda") << 7))
+        st.v_full[l].copy_(torch.randint(0, 0x7F, st.v_full[l].shape, dtype=torch.uint8, device="cuda")
+                           | (torch.randint(0, 2, st.v_full[l].shape, dtype=torch.uint8, device="cuda") << 7))
+        st.k_full[l].clamp_(max=0xFE)                                        # keep the NaN codes out
+        st.k_full[l][st.k_full[l] == 0x7F] = 0x7E
+        st.v_full[l].clamp_(max=0xFE)
+        st.v_full[l][st.v_full[l] == 0x7F] = 0x7E
+    st.mask.copy_(torch.from_numpy(mask)); st.seq_lens.fill_(n0)
+    lt.stream_init(st.shape, st.mask, st.tables, st.seq_lens, ws=st.ws)
+    out = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+    new = []
+    for step in range(steps):
+        q = (0.05 * torch.randn(L, B, Hq, D)).bfloat16().cuda()             # codes are spread over E4M3's whole range: keep logits moderate
+        k = torch.randn(L, B, Hkv, D).bfloat16().cuda(); v = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        new.append((k, v))
+        lt.decode_step(st.shape, q, k, v, st.tables, st.mask, st.seq_lens, out, st.ws)
+    assert lt.check(st.ws) == 0 and torch.isfinite(out).all()
+    G = Hq // Hkv
+    for l, b, h in [(0, 0, 0), (1, 3, 7), (2, 1, 4), (3, 2, 5)]:
+        Kq = table[st.k_full[l][b, h, :n0].long()].double().cpu().numpy() * float(scales[l, 0])
+        Vq = table[st.v_full[l][b, h, :n0].long()].double().cpu().numpy() * float(scales[l, 1])
+        ka = np.stack([O.quantize_e4m3(f64(k_[l, b, h]), scales[l, 0])[1] for k_, _ in new])
+        va = np.stack([O.quantize_e4m3(f64(v_[l, b, h]), scales[l, 1])[1] for _, v_ in new])
+        K = np.concatenate([Kq, ka])[None]; V = np.concatenate([Vq, va])[None]
+        qh = f64(q[l, b, h * G:(h + 1) * G])
+        ref = O.streaming_attention(qh, K, V, S, R) if mask[l] else O.full_attention(qh, K, V)
+        mx, rel = attn_errors(f64(out[l, b, h * G:(h + 1) * G]), ref)
+        assert rel <= ATTN_REL_L2 and mx <= ATTN_MAX_ABS * max(1.0, float(np.abs(ref).max())), (l, b, h, mx, rel)
