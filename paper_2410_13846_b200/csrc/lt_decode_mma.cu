@@ -1,4 +1,5 @@
-// Decode step, bandwidth path: bf16, head_dim 128, GQA group <= 8.
+// Decode step, bandwidth path: bf16 activations, head_dim 128, GQA group <= 8;
+// caches in bf16 or (template branch FP8) in E4M3 bytes.
 //
 // A persistent launch (two CTAs per SM) walks the flattened work list of
 // (layer, batch row, kv head, KV chunk) items; items are handed out through a
@@ -139,7 +140,7 @@ struct TileSrc {
 // FP8 = true: the caches hold E4M3 bytes (rows of 128 B) with one scale per layer
 // for K and one for V.  A ring stage then holds the raw bytes of a tile (K rows,
 // then V rows, the 16-byte column c of row r at column c ^ (r & 7)) and the MMA
-// fragments are made from the bytes in registers, as f16 holding value / 256:
+// fragments are made from the bytes in registers, as f16:
 //   K: ldmatrix on the bytes hands thread (g, c) the four bytes d = 4c .. 4c+3 of
 //      row g - an A fragment for a d order that Q's fragments simply follow;
 //   V: ldmatrix.trans on byte pairs hands it V[2c][2g], V[2c][2g+1], V[2c+1][2g],
@@ -148,8 +149,7 @@ struct TileSrc {
 // K bytes become f16 with the conversion instruction (one per byte pair), V
 // bytes - whose pairs are not adjacent - with integer bit moves that yield
 // value / 256; both run on the integer pipe, which is what bounds this path.
-// Q and P are f16 as
-// well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
+// Q and P are f16 as well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
 // is folded into the softmax scale and the V scale (x 256) into the final
 // normalisation.  32-key tiles give every warp two independent MMA chains.
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
