@@ -13,10 +13,14 @@
  * Conventions
  *   - Every function returns an lt_status; nothing aborts, throws or traps.
  *   - The caller owns all memory.  The library allocates nothing on the
- *     device, keeps no state between calls (beyond device properties it looks
- *     up once per device) and never synchronises the device unless a function
- *     says so.  All device work is enqueued on `stream`
- *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     device and never synchronises the device unless a function says so.  All
+ *     device work is enqueued on `stream` (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream).
+ *   - State between calls: none that belongs to a caller.  The library caches,
+ *     per device and behind locks, what it looks up on first use (SM count,
+ *     kernel attributes and occupancy, the driver's tensor-map encoder), so any
+ *     number of host threads may call it, first calls included.  Two calls that
+ *     share a workspace must still be ordered by the caller.
  *   - "dev" marks a device pointer, "host" a host pointer.
  *   - Layer tables (k_full, v_full, k_stream, v_stream) are HOST arrays of
  *     n_layers DEVICE pointers, read during the call only.  An entry may be
@@ -54,8 +58,9 @@ enum {
   LT_ERR_UNSUPPORTED = 2, /* head_dim not in {64,128}, unknown dtype, too many layers */
   LT_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
   LT_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error) */
-  LT_ERR_TIMEOUT = 5,     /* reserved: no kernel of this library waits on another */
-  LT_ERR_DEVICE_RANGE = 6 /* reported by lt_check: a position left its cache */
+  LT_ERR_TIMEOUT = 5,     /* reported by lt_check: a bounded wait inside the scoring kernel (on its copy engine
+                             or tensor-core barriers) ran out; that call's scores are invalid */
+  LT_ERR_DEVICE_RANGE = 6 /* reported by lt_check: a position left its cache, or a selected layer's table entry was NULL */
 };
 
 enum { LT_F32 = 0, LT_BF16 = 1 };
@@ -141,7 +146,8 @@ lt_status lt_workspace_init(void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
  * Copy the device error word to *flags_out and clear it.  SYNCHRONISES the
- * stream.  Returns LT_ERR_DEVICE_RANGE when any bit is set, LT_OK otherwise.
+ * stream.  Returns LT_ERR_TIMEOUT when LT_DEVERR_TIMEOUT is set (whatever else
+ * is), LT_ERR_DEVICE_RANGE when any other bit is set, LT_OK when the word is 0.
  */
 lt_status lt_check(void* ws /* dev */, uint32_t* flags_out /* host, may be NULL */, void* stream);
 
@@ -150,16 +156,24 @@ lt_status lt_check(void* ws /* dev */, uint32_t* flags_out /* host, may be NULL 
  *   q_tail  dev [L][B][Hq][w_last][D]: queries of prompt positions
  *           n_ctx - w_last .. n_ctx - 1
  *   k_full  host table of dev pointers; rows 0 .. n_ctx-1 of every (b, kv head)
- *           hold the prompt keys.  Every entry must be non-NULL.
+ *           hold the prompt keys.  Entries of the scored layers must be
+ *           non-NULL; the others are not looked at.
+ *   layers [layer_begin, layer_begin + layer_count) are scored (0 and n_layers
+ *           for the whole stack).  Scoring one layer at a time, right after its
+ *           prefill, is what Figure 3's queue needs: the keys of a layer that
+ *           was popped and compacted are never read again, so its full cache
+ *           can be freed and its table entry set to NULL.
  *   scores  dev float [L][B][Hq]: for each query head the mean over the w_last
  *           tail queries of the causal-softmax mass on keys j < n_sink or
  *           j >= n_ctx - n_recent (a set union; 1.0 when the window covers all).
+ *           Only the scored layers' slices are written.
  * The mean over heads and batch rows that completes Eq. 1 is taken by
  * lt_select_lazy.  Requires 1 <= w_last <= n_ctx <= full_capacity.
  */
 lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
                          const void* const* k_full /* host table */, int32_t n_ctx, int32_t w_last,
-                         float* scores /* dev */, void* ws /* dev */, size_t ws_bytes, void* stream);
+                         int32_t layer_begin, int32_t layer_count, float* scores /* dev */, void* ws /* dev */,
+                         size_t ws_bytes, void* stream);
 
 /*
  * Lazy ratio with the denominator given (Section 5.1: FlashAttention's prefill
@@ -173,12 +187,12 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
  *           read; the rest of the prompt keys is not touched.
  *   scores[l][b][hq] = mean over the tail rows of
  *           sum_{j kept, j <= i} exp(scale * q_i . k_j - lse_i).
- * Cost is independent of n_ctx.  Same workspace as lt_lazy_scores.
+ * Cost is independent of n_ctx.  Same workspace and layer range as lt_lazy_scores.
  */
 lt_status lt_lazy_scores_lse(const lt_shape* shape, const void* q_tail /* dev */,
                              const void* const* k_full /* host table */, const float* lse /* dev */,
-                             int32_t n_ctx, int32_t w_last, float* scores /* dev */, void* ws /* dev */,
-                             size_t ws_bytes, void* stream);
+                             int32_t n_ctx, int32_t w_last, int32_t layer_begin, int32_t layer_count,
+                             float* scores /* dev */, void* ws /* dev */, size_t ws_bytes, void* stream);
 
 /*
  * Selection (Section 5.1, the max-priority queue of size P = L - n_lazy; Fig. 3):
@@ -365,12 +379,17 @@ lt_status lt_decode_step_host(const lt_shape* shape, const void* q_host, const v
  * exits.  The call allocates and frees nothing.
  *
  *   - Same arguments, layouts and result as lt_hybrid_decode_attn.
- *   - dev_error (dev, may be NULL): receives this call's error word (the
- *     LT_DEVERR_* bits), stream-ordered; there is no workspace to lt_check.
+ *   - dev_error (dev, 4-byte aligned, may be NULL): receives this call's error
+ *     word (the LT_DEVERR_* bits), stream-ordered; there is no workspace to
+ *     lt_check.  It is written only by a call that returns LT_OK: a call refused
+ *     on the host enqueues nothing and leaves both *dev_error and the shared
+ *     array as they were.
  *   - A shape whose lt_workspace_bytes(shape, 0, 0, ..) exceeds
  *     LT_STATIC_SCRATCH_BYTES returns LT_ERR_WORKSPACE before any device work.
  *   - The first call on each device looks up the array's device address; make
- *     that call before beginning any stream capture.
+ *     that call before beginning any stream capture.  The address is kept for
+ *     the life of the process, which assumes that the device's primary context
+ *     is not reset in between.
  *   - All calls on a device share the array, which still holds the previous
  *     call's partials.  The error word is cleared at the start of every call and
  *     partials are written before they are read, so calls in stream order are

@@ -110,9 +110,9 @@ def lib() -> C.CDLL:
     L.lt_check.restype = i32
     L.lt_check.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     L.lt_lazy_scores.restype = i32
-    L.lt_lazy_scores.argtypes = [shp, vp, tab, i32, i32, vp, vp, sz, vp]
+    L.lt_lazy_scores.argtypes = [shp, vp, tab, i32, i32, i32, i32, vp, vp, sz, vp]
     L.lt_lazy_scores_lse.restype = i32
-    L.lt_lazy_scores_lse.argtypes = [shp, vp, tab, vp, i32, i32, vp, vp, sz, vp]
+    L.lt_lazy_scores_lse.argtypes = [shp, vp, tab, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.lt_select_lazy.restype = i32
     L.lt_select_lazy.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
     L.lt_select_lazy_per_seq.restype = i32
@@ -212,22 +212,27 @@ def workspace_init(ws, stream=None):
 def check(ws, stream=None, raise_on_error: bool = True) -> int:
     flags = C.c_uint32(0)
     st = lib().lt_check(_ptr(ws), C.byref(flags), _stream(stream))
-    if st != 0 and (raise_on_error or st != 6):
+    if st != 0 and (raise_on_error or st not in (5, 6)):
         raise LtError(st, f"lt_check (flags={flags.value:#x})")
     return int(flags.value)
 
 
-def lazy_scores(shape: Shape, q_tail, k_full, n_ctx: int, w_last: int, scores, ws, stream=None):
+def lazy_scores(shape: Shape, q_tail, k_full, n_ctx: int, w_last: int, scores, ws, layer_begin: int = 0,
+                layer_count: int | None = None, stream=None):
     tab = k_full.k_full if isinstance(k_full, LayerTables) else _table(k_full, shape.n_layers)
-    _ok(lib().lt_lazy_scores(C.byref(shape.c()), _ptr(q_tail), tab, n_ctx, w_last, _ptr(scores), _ptr(ws),
-                             ws.numel() * ws.element_size(), _stream(stream)), "lt_lazy_scores")
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_lazy_scores(C.byref(shape.c()), _ptr(q_tail), tab, n_ctx, w_last, layer_begin, cnt, _ptr(scores),
+                             _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "lt_lazy_scores")
 
 
-def lazy_scores_lse(shape: Shape, q_tail, k_full, lse, n_ctx: int, w_last: int, scores, ws, stream=None):
+def lazy_scores_lse(shape: Shape, q_tail, k_full, lse, n_ctx: int, w_last: int, scores, ws, layer_begin: int = 0,
+                    layer_count: int | None = None, stream=None):
     """lt_lazy_scores_lse: Eq. 1 from the prefill's log-sum-exp and the kept keys only."""
     tab = k_full.k_full if isinstance(k_full, LayerTables) else _table(k_full, shape.n_layers)
-    _ok(lib().lt_lazy_scores_lse(C.byref(shape.c()), _ptr(q_tail), tab, _ptr(lse), n_ctx, w_last, _ptr(scores),
-                                 _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "lt_lazy_scores_lse")
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_lazy_scores_lse(C.byref(shape.c()), _ptr(q_tail), tab, _ptr(lse), n_ctx, w_last, layer_begin, cnt,
+                                 _ptr(scores), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+        "lt_lazy_scores_lse")
 
 
 def select_lazy(scores, n_layers: int, batch: int, n_q_heads: int, n_lazy: int, layer_mask, layer_ratio=None,

@@ -1,9 +1,13 @@
 // C-ABI entry points of liblt: argument validation, workspace carving and
-// stream-ordered launches.  No device memory is allocated here and no state
-// survives a call.
+// stream-ordered launches.  No device memory is allocated here.  The only state
+// that survives a call is what the library looks up once per device (SM count,
+// kernel attributes, the driver's tensor-map encoder), each behind a lock, so
+// calls from several host threads are safe.
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
+
+#include <mutex>
 
 #include "lt_internal.h"
 
@@ -88,17 +92,23 @@ size_t ws_prefix_bytes(const lt_shape& s) {
   return kWsHeaderBytes + round_up(counters, kWsAlign);
 }
 
-int persistent_grid(const DecodeArgs& a, int ctas_per_sm) {
+int sm_count_of_current_device() {
+  static std::mutex mu;
   static int sm_count[64] = {0};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  std::lock_guard<std::mutex> lock(mu);
   if (sm_count[dev] == 0) {
     int n = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
     sm_count[dev] = n;
   }
+  return sm_count[dev];
+}
+
+int persistent_grid(const DecodeArgs& a, int ctas_per_sm) {
   const long long most = a.items_cap;
-  long long grid = (long long)sm_count[dev] * ctas_per_sm;
+  long long grid = (long long)sm_count_of_current_device() * ctas_per_sm;
   if (grid > most) grid = most;
   return (int)(grid < 1 ? 1 : grid);
 }
@@ -110,6 +120,17 @@ static lt_status fill_table(LayerTable* t, const void* const* host, int L, bool 
     t->p[l] = host[l];
     if (require_all && !host[l]) return LT_ERR_INVALID_ARG;
     if (((uintptr_t)host[l] & 15u) != 0) return LT_ERR_INVALID_ARG;
+  }
+  return LT_OK;
+}
+
+// Entries of [begin, begin + count) must be present; the rest of the table is not looked at.
+static lt_status fill_table_range(LayerTable* t, const void* const* host, int begin, int count) {
+  memset(t, 0, sizeof(*t));
+  if (!host) return LT_ERR_INVALID_ARG;
+  for (int l = begin; l < begin + count; ++l) {
+    if (!host[l] || ((uintptr_t)host[l] & 15u) != 0) return LT_ERR_INVALID_ARG;
+    t->p[l] = host[l];
   }
   return LT_OK;
 }
@@ -179,13 +200,14 @@ lt_status lt_check(void* ws, uint32_t* flags_out, void* stream) {
   if (cudaMemsetAsync(ws, 0, sizeof(flags), st) != cudaSuccess) return LT_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LT_ERR_CUDA;
   if (flags_out) *flags_out = flags;
+  if (flags & LT_DEVERR_TIMEOUT) return LT_ERR_TIMEOUT;  // the scores of that call are invalid
   return flags ? LT_ERR_DEVICE_RANGE : LT_OK;
 }
 
 // Shared body of lt_lazy_scores (lse == NULL) and lt_lazy_scores_lse.
 static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,
-                             int window_only, int32_t n_ctx, int32_t w_last, float* scores, void* ws, size_t ws_bytes,
-                             void* stream) {
+                             int window_only, int32_t n_ctx, int32_t w_last, int32_t layer_begin,
+                             int32_t layer_count, float* scores, void* ws, size_t ws_bytes, void* stream) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
@@ -193,8 +215,9 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   if (shape->kv_fp8) return LT_ERR_UNSUPPORTED;  // scoring reads 16- or 32-bit keys only
   if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
   if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0) return LT_ERR_INVALID_ARG;
+  if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
   LayerTable kf;
-  if ((st = fill_table(&kf, k_full, shape->n_layers, true)) != LT_OK) return st;
+  if ((st = fill_table_range(&kf, k_full, layer_begin, layer_count)) != LT_OK) return st;
   const ScorePlan sp = make_score_plan(*shape, n_ctx, w_last, window_only != 0);
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   const size_t prefix = ws_prefix_bytes(*shape);
@@ -205,6 +228,8 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   a.lse = lse;
   a.n_ctx = n_ctx;
   a.w_last = w_last;
+  a.layer_begin = layer_begin;
+  a.layer_count = layer_count;
   a.window_only = window_only;
   a.n_splits = sp.n_splits;
   a.split_len = sp.split_len;
@@ -221,13 +246,17 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
 }
 
 lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* const* k_full, int32_t n_ctx,
-                         int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
-  return scores_impl(shape, q_tail, k_full, nullptr, 0, n_ctx, w_last, scores, ws, ws_bytes, stream);
+                         int32_t w_last, int32_t layer_begin, int32_t layer_count, float* scores, void* ws,
+                         size_t ws_bytes, void* stream) {
+  return scores_impl(shape, q_tail, k_full, nullptr, 0, n_ctx, w_last, layer_begin, layer_count, scores, ws, ws_bytes,
+                     stream);
 }
 
 lt_status lt_lazy_scores_lse(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,
-                             int32_t n_ctx, int32_t w_last, float* scores, void* ws, size_t ws_bytes, void* stream) {
-  return scores_impl(shape, q_tail, k_full, lse, 1, n_ctx, w_last, scores, ws, ws_bytes, stream);
+                             int32_t n_ctx, int32_t w_last, int32_t layer_begin, int32_t layer_count, float* scores,
+                             void* ws, size_t ws_bytes, void* stream) {
+  return scores_impl(shape, q_tail, k_full, lse, 1, n_ctx, w_last, layer_begin, layer_count, scores, ws, ws_bytes,
+                     stream);
 }
 
 lt_status lt_select_lazy(const float* scores, int32_t n_layers, int32_t batch, int32_t n_q_heads, int32_t n_lazy,
@@ -332,12 +361,15 @@ lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask, const v
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 
-// Shared body of lt_hybrid_decode_attn (k_new == NULL) and lt_decode_step.
-static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+}  // extern "C"
+
+// Shared body of lt_hybrid_decode_attn (k_new == NULL) and lt_decode_step, in two halves: every check that
+// the host can make (nothing is enqueued), then the launches.
+lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
                              const void* const* k_full, const void* const* v_full, const void* const* k_stream,
                              const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
                              int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
-                             void* ws, size_t ws_bytes, void* stream) {
+                             void* ws, size_t ws_bytes) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q || !layer_mask || !seq_lens || !out) return LT_ERR_INVALID_ARG;
@@ -349,12 +381,11 @@ static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k
   if ((((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15u) != 0) return LT_ERR_INVALID_ARG;
   if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
   if (shape->batch > kMaxWorkEntries) return LT_ERR_UNSUPPORTED;
-  LayerTable kf, vf, ks, vs;
   const int L = shape->n_layers;
-  if ((st = fill_table(&kf, k_full, L, false)) != LT_OK) return st;
-  if ((st = fill_table(&vf, v_full, L, false)) != LT_OK) return st;
-  if ((st = fill_table(&ks, k_stream, L, false)) != LT_OK) return st;
-  if ((st = fill_table(&vs, v_stream, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&c->kf, k_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&c->vf, v_full, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&c->ks, k_stream, L, false)) != LT_OK) return st;
+  if ((st = fill_table(&c->vs, v_stream, L, false)) != LT_OK) return st;
 
   DecodePlan dp = make_decode_plan(*shape);
   const size_t prefix = ws_prefix_bytes(*shape);
@@ -363,7 +394,7 @@ static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   if (ws_bytes < prefix + ml_bytes + o_bytes) return LT_ERR_WORKSPACE;
 
-  DecodeArgs a;
+  DecodeArgs& a = c->a;
   a.s = *shape;
   a.q = q;
   a.k_new = k_new;
@@ -378,6 +409,9 @@ static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k
   a.target_items = dp.target_items;
   a.items_cap = dp.items_cap;
   a.fused = fused;
+  a.advance = advance;
+  a.layer_begin = layer_begin;
+  a.layer_count = layer_count;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
   a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;
   a.work_counter = a.done_counter + 1;
@@ -385,21 +419,40 @@ static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k
   a.part_o = reinterpret_cast<float*>((char*)ws + prefix + ml_bytes);
   a.dev_err = err_word(ws);
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
+  return LT_OK;
+}
 
+lt_status lt::decode_launch(const DecodeCall& c, void* stream) {
   // One launch takes at most kMaxWorkEntries (layer, batch row) pairs; a larger
   // stack goes in consecutive launches by layers (only the last one advances).
+  DecodeArgs a = c.a;
   cudaStream_t cs = (cudaStream_t)stream;
-  const int layers_per_launch = kMaxWorkEntries / shape->batch;
-  const bool mma = decode_mma_supported(*shape);
+  const int layer_begin = c.a.layer_begin, layer_count = c.a.layer_count;
+  const int layers_per_launch = kMaxWorkEntries / a.s.batch;
+  const bool mma = decode_mma_supported(a.s);
   for (int done = 0; done < layer_count; done += layers_per_launch) {
     a.layer_begin = layer_begin + done;
     a.layer_count = layer_count - done < layers_per_launch ? layer_count - done : layers_per_launch;
-    a.advance = (advance && done + a.layer_count == layer_count) ? 1 : 0;
-    cudaError_t e = mma ? launch_decode_mma(a, kf, vf, ks, vs, cs) : launch_decode_generic(a, kf, vf, ks, vs, cs);
+    a.advance = (c.a.advance && done + a.layer_count == layer_count) ? 1 : 0;
+    cudaError_t e = mma ? launch_decode_mma(a, c.kf, c.vf, c.ks, c.vs, cs) : launch_decode_generic(a, c.kf, c.vf, c.ks, c.vs, cs);
     if (e != cudaSuccess) return LT_ERR_CUDA;
   }
   return LT_OK;
 }
+
+static lt_status decode_impl(const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+                             const void* const* k_full, const void* const* v_full, const void* const* k_stream,
+                             const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
+                             int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
+                             void* ws, size_t ws_bytes, void* stream) {
+  DecodeCall c;
+  const lt_status st = decode_prepare(&c, shape, q, k_new, v_new, k_full, v_full, k_stream, v_stream, layer_mask,
+                                      seq_lens, out, out_dtype, layer_begin, layer_count, fused, advance, ws, ws_bytes);
+  if (st != LT_OK) return st;
+  return decode_launch(c, stream);
+}
+
+extern "C" {
 
 lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q, const void* const* k_full,
                                 const void* const* v_full, const void* const* k_stream, const void* const* v_stream,

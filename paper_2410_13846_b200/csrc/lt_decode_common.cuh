@@ -37,7 +37,7 @@ struct WorkItem {
 __device__ __forceinline__ int ring_slot_of(int p, int S, int R) { return p < S ? p : S + (p - S) % R; }
 
 // Shared-memory footprint of the work list (bytes) for `entries` (layer, b) pairs.
-__host__ __device__ inline int worklist_smem_bytes(int entries, int batch) {
+__host__ __device__ constexpr inline int worklist_smem_bytes(int entries, int batch) {
   return ((entries + 1 + batch) * 4 + entries + 15) / 16 * 16;
 }
 

@@ -32,6 +32,8 @@
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 
+#include <mutex>
+
 #include "lt_decode_common.cuh"
 #include "lt_internal.h"
 
@@ -662,21 +664,38 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
   static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
   auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8>;
-  // attribute and occupancy are looked up once per shared-memory size (host time matters for per-layer callers)
-  static int cached_smem_of[64], cached_per_sm_of[64];  // per device; zero = not looked up yet
+  // Per device, behind a lock (host threads may issue their first calls concurrently): the dynamic
+  // shared-memory limit is raised once to the largest size any launch of this variant can ask for, and
+  // the occupancy of each shared-memory size met so far is remembered (host time matters for per-layer callers).
+  constexpr int kSmemMax = ring + merge + worklist_smem_bytes(kMaxWorkEntries, kMaxWorkEntries);
+  constexpr int kSizes = 8;
+  struct PerDevice {
+    bool attr_set;
+    int n, smem[kSizes], per_sm[kSizes];
+  };
+  static std::mutex mu;
+  static PerDevice cache[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  int& cached_smem = cached_smem_of[dev];
-  int& cached_per_sm = cached_per_sm_of[dev];
-  int per_sm = cached_per_sm;
-  if (smem != cached_smem) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, WARPS * 32, smem);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-    cached_smem = smem;
-    cached_per_sm = per_sm;
+  int per_sm = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    PerDevice& c = cache[dev];
+    if (!c.attr_set) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+      if (e != cudaSuccess) return e;
+      c.attr_set = true;
+    }
+    for (int i = 0; i < c.n; ++i)
+      if (c.smem[i] == smem) per_sm = c.per_sm[i];
+    if (per_sm == 0) {
+      cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, WARPS * 32, smem);
+      if (e != cudaSuccess) return e;
+      if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+      const int slot = c.n < kSizes ? c.n++ : 0;  // a caller that cycles through many sizes just looks up again
+      c.smem[slot] = smem;
+      c.per_sm[slot] = per_sm;
+    }
   }
   const int grid = persistent_grid(a, per_sm);
   kern<<<grid, WARPS * 32, smem, st>>>(a, kf, vf, ks, vs);

@@ -105,6 +105,8 @@ constexpr int kMaxWorkEntries = 2048;
 // CTAs of a persistent decode launch: per_sm * SM count, but no more than the
 // most items the launch can have.
 int persistent_grid(const DecodeArgs& a, int ctas_per_sm);
+// SM count of the current device (looked up once per device, behind a lock).
+int sm_count_of_current_device();
 cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 // bf16, head_dim 128, group size <= 8: tensor-core path.
@@ -112,11 +114,26 @@ bool decode_mma_supported(const lt_shape& s);
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                               const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 
+// A validated decode call, ready to launch: the two halves of lt_hybrid_decode_attn / lt_decode_step,
+// split so that a caller can put its own stream work between the host-side checks and the launches.
+struct DecodeCall {
+  DecodeArgs a;
+  LayerTable kf, vf, ks, vs;
+};
+// Every check the host can make; enqueues nothing.  `ws` only has its address and size looked at.
+lt_status decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+                         const void* const* k_full, const void* const* v_full, const void* const* k_stream,
+                         const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
+                         int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
+                         void* ws, size_t ws_bytes);
+lt_status decode_launch(const DecodeCall& c, void* stream);
+
 struct ScoreArgs {
   lt_shape s;
   const void* q_tail;
   const float* lse;  // window_only: natural-log denominators [L][B][Hq][T]
   int n_ctx, w_last;
+  int layer_begin, layer_count;  // layers scored by this call; q_tail, stats and scores keep their whole-stack indexing
   int window_only;
   int n_splits, split_len;
   float cs;      // softmax scale * log2(e)

@@ -29,7 +29,7 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
   const lt_shape& s = a.s;
   const int t = blockIdx.x / a.n_splits, sp = blockIdx.x % a.n_splits;
   const int b = blockIdx.y / s.n_q_heads, hq = blockIdx.y % s.n_q_heads;
-  const int l = blockIdx.z;
+  const int l = a.layer_begin + blockIdx.z;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int h = hq / G;
   __shared__ float qs[D];
@@ -80,7 +80,7 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
 }
 
 cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
-  dim3 grid(a.w_last * a.n_splits, a.s.batch * a.s.n_q_heads, a.s.n_layers);
+  dim3 grid(a.w_last * a.n_splits, a.s.batch * a.s.n_q_heads, a.layer_count);
   const bool bf = a.s.dtype == LT_BF16;
   if (a.s.head_dim == 128) {
     if (bf) scores_generic_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(a, kf);
@@ -96,9 +96,10 @@ cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cuda
 // row's mass W/A, average over the w_last rows in row order.
 __global__ void scores_finish_kernel(ScoreArgs a) {
   const lt_shape& s = a.s;
-  const long long total = (long long)s.n_layers * s.batch * s.n_q_heads;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= total) return;
+  const long long per_layer = (long long)s.batch * s.n_q_heads;
+  const long long rel = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (rel >= a.layer_count * per_layer) return;
+  const long long idx = a.layer_begin * per_layer + rel;
   float sum = 0.f;
   for (int t = 0; t < a.w_last; ++t) {
     const float* st = a.stats + ((idx * a.w_last + t) * a.n_splits) * 3;
@@ -124,7 +125,7 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
 }
 
 cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st) {
-  const long long total = (long long)a.s.n_layers * a.s.batch * a.s.n_q_heads;
+  const long long total = (long long)a.layer_count * a.s.batch * a.s.n_q_heads;
   scores_finish_kernel<<<(unsigned)((total + 127) / 128), 128, 0, st>>>(a);
   return cudaGetLastError();
 }

@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int M = G * T;
   const int sp = blockIdx.x % a.n_splits, rb = blockIdx.x / a.n_splits;
   const int b = blockIdx.y / s.n_kv_heads, h = blockIdx.y % s.n_kv_heads;
-  const int l = blockIdx.z;
+  const int l = a.layer_begin + blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_ctx = a.n_ctx;
   int k0, k1;
@@ -454,16 +454,16 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 // The driver's tensor-map encoder, looked up through the runtime (no link-time dependency on libcuda).
+EncodeTiledFn lookup_encode_tiled() {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  return reinterpret_cast<EncodeTiledFn>(p);
+}
 EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+  static const EncodeTiledFn fn = lookup_encode_tiled();  // initialised once, thread-safe
   return fn;
 }
 }  // namespace
@@ -481,16 +481,18 @@ cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStr
   const cuuint32_t box[2] = {64u, (cuuint32_t)kBlockN};
   const cuuint32_t estride[2] = {1u, 1u};
   KeyMaps local;
-  for (int l = 0; l < a.s.n_layers; ++l) {
+  const int l_end = a.layer_begin + a.layer_count;
+  for (int l = a.layer_begin; l < l_end; ++l) {
     const CUresult r = encode(&local.m[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kf.p[l]), gdim,
                               gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
-  for (int l = a.s.n_layers; l < LT_MAX_LAYERS; ++l) local.m[l] = local.m[0];
+  for (int l = 0; l < LT_MAX_LAYERS; ++l)
+    if (l < a.layer_begin || l >= l_end) local.m[l] = local.m[a.layer_begin];
   cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  dim3 grid(a.n_splits * row_blocks, a.s.batch * a.s.n_kv_heads, a.s.n_layers);
+  dim3 grid(a.n_splits * row_blocks, a.s.batch * a.s.n_kv_heads, a.layer_count);
   scores_umma_kernel<<<grid, kThreads, kSmemBytes, st>>>(a, local);
   return cudaGetLastError();
 }

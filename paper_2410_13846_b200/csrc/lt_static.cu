@@ -71,14 +71,27 @@ extern "C" lt_status lt_hybrid_decode_attn_static(const lt_shape* shape, const v
   if (st != LT_OK) return st;
   if (need > (size_t)LT_STATIC_SCRATCH_BYTES) return LT_ERR_WORKSPACE;
 
+  // Every check the host can make comes before any CUDA call and before anything is enqueued: a refused
+  // call touches neither the shared array nor *dev_error.  (The checks only look at the workspace's address
+  // and size, so they can run against a stand-in address before the array's own is known.)
+  (void)max_seq_len_hint;  // ignored, as in lt_hybrid_decode_attn
+  DecodeCall call;
+  st = decode_prepare(&call, shape, q, nullptr, nullptr, k_full, v_full, k_stream, v_stream, layer_mask,
+                      const_cast<int32_t*>(seq_lens), out, out_dtype, layer_begin, layer_count, 0, 0,
+                      reinterpret_cast<void*>(kWsAlign), (size_t)LT_STATIC_SCRATCH_BYTES);
+  if (st != LT_OK) return st;
+  if (dev_error && ((uintptr_t)dev_error & 3u) != 0) return LT_ERR_INVALID_ARG;
+
   void* scratch = nullptr;
   if (scratch_for_current_device(&scratch) != cudaSuccess) return LT_ERR_CUDA;
+  st = decode_prepare(&call, shape, q, nullptr, nullptr, k_full, v_full, k_stream, v_stream, layer_mask,
+                      const_cast<int32_t*>(seq_lens), out, out_dtype, layer_begin, layer_count, 0, 0, scratch,
+                      (size_t)LT_STATIC_SCRATCH_BYTES);
+  if (st != LT_OK) return st;
   cudaStream_t cs = (cudaStream_t)stream;
   // The header holds the error word and the merge counters; start every call from zero.
   if (cudaMemsetAsync(scratch, 0, ws_prefix_bytes(*shape), cs) != cudaSuccess) return LT_ERR_CUDA;
-  st = lt_hybrid_decode_attn(shape, q, k_full, v_full, k_stream, v_stream, layer_mask, seq_lens, out, out_dtype,
-                             max_seq_len_hint, layer_begin, layer_count, scratch, (size_t)LT_STATIC_SCRATCH_BYTES,
-                             stream);
+  st = decode_launch(call, stream);
   if (st != LT_OK) return st;
   if (dev_error) {
     // hand the step's error word to the caller's own device word (stream-ordered, 4 bytes)

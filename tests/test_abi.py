@@ -71,12 +71,17 @@ def test_host_side_errors_come_before_any_launch():
     assert L.lt_select_lazy(fake, 2, 1, 4, -1, fake, None, None) == 1
     assert L.lt_select_lazy(None, 2, 1, 4, 1, fake, None, None) == 1
     assert L.lt_select_lazy(fake, 200, 1, 4, 1, fake, None, None) == 2      # too many layers
-    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 513, fake, fake, 1 << 20, None) == 1   # w_last > n_ctx
-    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 600, 16, fake, fake, 1 << 20, None) == 1    # n_ctx > capacity
-    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, fake, None, 0, None) == 3          # no workspace
-    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, fake, C.c_void_p(0x1000), 300, None) == 3  # too small
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 513, 0, 2, fake, fake, 1 << 20, None) == 1   # w_last > n_ctx
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 600, 16, 0, 2, fake, fake, 1 << 20, None) == 1    # n_ctx > capacity
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, 0, 2, fake, None, 0, None) == 3          # no workspace
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, 0, 2, fake, C.c_void_p(0x1000), 300, None) == 3  # too small
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, 1, 2, fake, fake, 1 << 20, None) == 1    # layer range
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab, 512, 16, 0, 0, fake, fake, 1 << 20, None) == 1
     tab_null = (C.c_void_p * 2)(0x1000, None)
-    assert L.lt_lazy_scores(C.byref(cs), fake, tab_null, 512, 16, fake, fake, 1 << 20, None) == 1
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab_null, 512, 16, 0, 2, fake, fake, 1 << 20, None) == 1   # scored layer missing
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab_null, 512, 16, 1, 1, fake, fake, 1 << 20, None) == 1
+    # a missing entry outside the scored range is fine: the call gets past the table check (and stops at the workspace)
+    assert L.lt_lazy_scores(C.byref(cs), fake, tab_null, 512, 16, 0, 1, fake, None, 0, None) == 3
     tab_misaligned = (C.c_void_p * 2)(0x1004, 0x2000)
     assert L.lt_hybrid_decode_attn(C.byref(cs), fake, tab_misaligned, tab, None, None, fake, fake, fake, 0, 0, 0, 2,
                                    fake, 1 << 20, None) == 1

@@ -70,17 +70,22 @@ def test_llama3_8b_32k_sampled_units():
     st, q_tail, planted = _build(cfg, steps)
     s = st.shape
     L, B, Hkv, G, n0 = cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.group, cfg.n_ctx
-    g = np.random.default_rng(11)
     # ---- scoring + selection --------------------------------------------------
     scores = torch.zeros((L, B, cfg.n_q_heads), dtype=torch.float32, device="cuda")
     lt.lazy_scores(s, q_tail, st.tables, n0, cfg.w_last, scores, st.ws)
     sc = f64(scores)
     assert np.isfinite(sc).all() and sc.min() >= 0 and sc.max() <= 1 + 1e-6
-    for _ in range(6):                                        # sampled (layer, b, kv head) units, all G heads
-        l, b, h = int(g.integers(L)), int(g.integers(B)), int(g.integers(Hkv))
+    # scoring units (layer, b, kv head; all G heads of each): a fixed sample that covers every kv head, the
+    # first and the last batch row, and planted as well as unplanted layers (first, middle, last of each)
+    unplanted = [l for l in range(L) if l not in planted]
+    score_units = [(planted[0], 0, 0), (unplanted[0], B - 1, 1), (planted[-1], B - 1, 2), (unplanted[-1], 0, 3),
+                   (planted[len(planted) // 2], B // 2, 4), (unplanted[len(unplanted) // 2], 1, 5),
+                   (planted[1], B - 1, 6), (unplanted[1], 0, 7)]
+    assert {u[2] for u in score_units} == set(range(Hkv))
+    for l, b, h in score_units:
         ref = O.lazy_scores(f64(q_tail[l, b, h * G:(h + 1) * G]), f64(st.k_full[l][b, h:h + 1, :n0]), cfg.n_sink,
                             cfg.n_recent)
-        assert np.max(np.abs(sc[l, b, h * G:(h + 1) * G] - ref)) <= SCORE_ABS
+        assert np.max(np.abs(sc[l, b, h * G:(h + 1) * G] - ref)) <= SCORE_ABS, (l, b, h)
     lt.select_lazy(scores, L, B, cfg.n_q_heads, cfg.n_lazy, st.mask)
     mask = st.mask.cpu().numpy()
     r = O.layer_ratios(sc)
@@ -100,9 +105,11 @@ def test_llama3_8b_32k_sampled_units():
     assert torch.isfinite(out).all()
     n = n0 + steps
     lazy_layers, full_layers = np.nonzero(mask)[0], np.nonzero(mask == 0)[0]
-    units = [(int(full_layers[0]), 0, 0), (int(full_layers[-1]), B - 1, Hkv - 1), (int(lazy_layers[0]), 0, 1),
-             (int(lazy_layers[-1]), B - 1, Hkv - 2)]
-    units += [(int(g.integers(L)), int(g.integers(B)), int(g.integers(Hkv))) for _ in range(4)]
+    # decode units: a fixed sample with every kv head at least once and the first and last batch row of both layer kinds
+    fl, lz = [int(x) for x in full_layers], [int(x) for x in lazy_layers]
+    units = [(fl[0], 0, 0), (fl[-1], B - 1, Hkv - 1), (lz[0], 0, 1), (lz[-1], B - 1, Hkv - 2),
+             (fl[len(fl) // 2], B // 2, 2), (lz[len(lz) // 2], 1, 3), (fl[1], B - 1, 4), (lz[1], 0, 5)]
+    assert {u[2] for u in units} == set(range(Hkv))
     for l, b, h in units:
         # logical history of this unit: prompt rows (still in the full cache of every layer) + appended rows
         K = np.concatenate([f64(st.k_full[l][b, h, :n0]), np.stack([f64(x[l, b, h]) for x in new_k])])[None]
