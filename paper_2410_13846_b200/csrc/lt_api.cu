@@ -62,9 +62,9 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   return p;
 }
 
-ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only) {
-  ScorePlan p;
-  const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
+// Host-side key splits of one (layer, batch row, kv head) when `layers` layers are scored by one call.
+static int host_score_splits(const lt_shape& s, int n_ctx, int w_last, bool window_only, int layers, int* split_len) {
+  const int64_t units = (int64_t)layers * s.batch * s.n_kv_heads;
   int64_t want = (148 * 4 + units - 1) / units;  // a few CTAs per SM even for small stacks
   int span = n_ctx;                              // keys that are divided among the splits
   if (window_only) {
@@ -79,11 +79,41 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
   int len = (int)((span + want - 1) / want);
   len = (len + 63) / 64 * 64;
   if (len < 64) len = 64;
-  p.split_len = len;
-  p.n_splits = (int)((span + len - 1) / len);
-  if (p.n_splits < 1) p.n_splits = 1;
-  if (window_only && s.n_sink > 0) p.n_splits += 1;
-  p.stat_floats = (size_t)s.n_layers * s.batch * s.n_q_heads * w_last * p.n_splits * 3;
+  *split_len = len;
+  int n = (int)((span + len - 1) / len);
+  if (n < 1) n = 1;
+  if (window_only && s.n_sink > 0) n += 1;
+  return n;
+}
+
+ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only, int layer_count) {
+  ScorePlan p;
+  const size_t rows_per_layer = (size_t)s.batch * s.n_q_heads * w_last;
+  if (layer_count > 0) {
+    p.n_splits = host_score_splits(s, n_ctx, w_last, window_only, layer_count, &p.split_len);
+    p.stat_floats = (size_t)layer_count * rows_per_layer * p.n_splits * 3;
+    return p;
+  }
+  // Workspace query: room for a call over any layer range with any prompt length up to n_ctx and any
+  // tail length up to w_last, through either kernel.  The persistent tensor-core kernel cuts a unit into at
+  // most (CTAs / units) + 2 pieces, never more than it has tiles.
+  const bool umma = !window_only && scores_umma_supported(s, w_last);
+  const int64_t tiles = (n_ctx + kScoreBlockN - 1) / kScoreBlockN;
+  size_t most_slots = 0;  // max over c of c * slots(c)
+  p.n_splits = 1;
+  p.split_len = 64;
+  for (int c = 1; c <= s.n_layers; ++c) {
+    int len = 0;
+    int64_t slots = host_score_splits(s, n_ctx, w_last, window_only, c, &len) + 1;  // + 1: rounding of shorter prompts
+    if (umma) {
+      int64_t pieces = kScoreMaxCtas / ((int64_t)c * s.batch * s.n_kv_heads) + 2;
+      if (pieces > tiles) pieces = tiles;
+      if (pieces > slots) slots = pieces;
+    }
+    if ((size_t)(c * slots) > most_slots) most_slots = (size_t)(c * slots);
+    if (slots > p.n_splits) p.n_splits = (int)slots;
+  }
+  p.stat_floats = rows_per_layer * most_slots * 3;
   return p;
 }
 
@@ -218,11 +248,33 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
   LayerTable kf;
   if ((st = fill_table_range(&kf, k_full, layer_begin, layer_count)) != LT_OK) return st;
-  const ScorePlan sp = make_score_plan(*shape, n_ctx, w_last, window_only != 0);
+  const bool umma = scores_umma_supported(*shape, w_last);
+  ScorePlan sp = make_score_plan(*shape, n_ctx, w_last, window_only != 0, layer_count);
+  ScoreArgs a;
+  memset(&a, 0, sizeof(a));
+  if (umma) {
+    // the persistent launch: one CTA per SM; with the whole prompt scored the CTAs own contiguous tile ranges
+    a.row_blocks = ((shape->n_q_heads / shape->n_kv_heads) * w_last + kScoreBlockM - 1) / kScoreBlockM;
+    a.n_units = layer_count * shape->batch * shape->n_kv_heads * a.row_blocks;
+    a.streamk = window_only ? 0 : 1;
+    a.tiles_per_unit = (n_ctx + kScoreBlockN - 1) / kScoreBlockN;
+    a.total_tiles = (long long)a.n_units * a.tiles_per_unit;
+    const long long work = a.streamk ? a.total_tiles : (long long)a.n_units * sp.n_splits;
+    int grid = sm_count_of_current_device();
+    if (grid > kScoreMaxCtas) grid = kScoreMaxCtas;
+    if (grid > work) grid = (int)work;
+    a.grid = grid < 1 ? 1 : grid;
+    if (a.streamk) {
+      // most pieces any unit is cut into under this grid: owner(last tile) - owner(first tile) + 1
+      long long pieces = ((long long)(a.tiles_per_unit - 1) * a.grid) / a.total_tiles + 2;
+      if (pieces > a.tiles_per_unit) pieces = a.tiles_per_unit;
+      sp.n_splits = (int)pieces;
+      sp.stat_floats = (size_t)layer_count * shape->batch * shape->n_q_heads * w_last * sp.n_splits * 3;
+    }
+  }
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   const size_t prefix = ws_prefix_bytes(*shape);
   if (ws_bytes < prefix + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
-  ScoreArgs a;
   a.s = *shape;
   a.q_tail = q_tail;
   a.lse = lse;
@@ -238,8 +290,7 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
   a.dev_err = err_word(ws);
   cudaStream_t cs = (cudaStream_t)stream;
-  cudaError_t e = scores_umma_supported(*shape, w_last) ? launch_scores_umma(a, kf, cs)
-                                                        : launch_scores_generic(a, kf, cs);
+  cudaError_t e = umma ? launch_scores_umma(a, kf, cs) : launch_scores_generic(a, kf, cs);
   if (e != cudaSuccess) return LT_ERR_CUDA;
   e = launch_scores_finish(a, cs);
   return e == cudaSuccess ? LT_OK : LT_ERR_CUDA;

@@ -38,11 +38,27 @@ DecodePlan make_decode_plan(const lt_shape& s);
 // only the kept keys are visited: split 0 is the sink range when n_sink > 0,
 // the other splits are equal parts of the recent range.
 struct ScorePlan {
-  int n_splits;        // key-range splits per (layer, batch row, kv head)
+  int n_splits;        // statistics slots per tail row: key-range splits of its (layer, batch row, kv head), or
+                       // the pieces that the persistent tensor-core kernel may cut its unit into
   int split_len;       // keys per split (of the whole prompt, or of the recent range)
-  size_t stat_floats;  // [L][B][Hq][T][n_splits][3] partial (max, sum_all, sum_window)
+  size_t stat_floats;  // [L][B][Hq][T][n_splits][3] partial (reference exponent, sum_all, sum_window)
 };
-ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only);
+// layer_count: layers scored by one call; 0 = the bound that holds for any layer range (workspace query).
+ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_only, int layer_count = 0);
+
+// Geometry of the tensor-core scoring kernel.
+constexpr int kScoreBlockM = 256;   // query rows per unit
+constexpr int kScoreBlockN = 128;   // keys per tile
+constexpr int kScoreMaxCtas = 192;  // the persistent launch never has more CTAs than this (one per SM)
+// The persistent launch cuts the sequence of all tiles, [0, total), into `grid` contiguous ranges:
+// tile g belongs to CTA g * grid / total.
+__host__ __device__ inline int score_tile_owner(long long total, int grid, long long g) {
+  return (int)((g * grid) / total);
+}
+__host__ __device__ inline void score_cta_tiles(long long total, int grid, int cta, long long* g0, long long* g1) {
+  *g0 = ((long long)cta * total + grid - 1) / grid;
+  *g1 = ((long long)(cta + 1) * total + grid - 1) / grid;
+}
 
 // Index of (layer l, batch row b) in layer_mask.
 __host__ __device__ inline int mask_index(const lt_shape& s, int l, int b) {
@@ -136,6 +152,13 @@ struct ScoreArgs {
   int layer_begin, layer_count;  // layers scored by this call; q_tail, stats and scores keep their whole-stack indexing
   int window_only;
   int n_splits, split_len;
+  // tensor-core path only: the persistent launch
+  int streamk;             // 1: CTAs own contiguous tile ranges and n_splits counts the pieces of a unit; 0: host splits
+  int grid;                // CTAs
+  int row_blocks;          // blocks of kScoreBlockM query rows per (layer, b, kv head)
+  int n_units;             // layer_count * B * Hkv * row_blocks
+  int tiles_per_unit;      // streamk: ceil(n_ctx / kScoreBlockN)
+  long long total_tiles;   // streamk: n_units * tiles_per_unit
   float cs;      // softmax scale * log2(e)
   float* stats;  // workspace
   float* scores;

@@ -72,7 +72,7 @@ __global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
       }
     }
     float* st = a.stats +
-                ((((((long long)l * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * a.n_splits) + sp) * 3;
+                ((((((long long)blockIdx.z * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * a.n_splits) + sp) * 3;
     st[0] = Mx;
     st[1] = As;
     st[2] = Ws;
@@ -92,28 +92,43 @@ cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cuda
   return cudaGetLastError();
 }
 
-// One thread per (layer, b, hq): merge the splits of every tail row, take the
-// row's mass W/A, average over the w_last rows in row order.
+// One thread per (layer, b, hq): merge the statistics slots of every tail row, take the
+// row's mass W/A, average over the w_last rows in row order.  The statistics are indexed by the
+// layer's position in the scored range.
 __global__ void scores_finish_kernel(ScoreArgs a) {
   const lt_shape& s = a.s;
   const long long per_layer = (long long)s.batch * s.n_q_heads;
   const long long rel = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (rel >= a.layer_count * per_layer) return;
   const long long idx = a.layer_begin * per_layer + rel;
+  const int T = a.w_last;
   float sum = 0.f;
-  for (int t = 0; t < a.w_last; ++t) {
-    const float* st = a.stats + ((idx * a.w_last + t) * a.n_splits) * 3;
+  for (int t = 0; t < T; ++t) {
+    const float* st = a.stats + ((rel * T + t) * a.n_splits) * 3;
+    int n_slots = a.n_splits;
+    if (a.streamk) {
+      // the persistent kernel wrote one slot per piece of this row's unit: the CTAs from the owner of the
+      // unit's first tile to the owner of its last one
+      const int G = s.n_q_heads / s.n_kv_heads;
+      const int hq = (int)(rel % s.n_q_heads);
+      const long long lb = rel / s.n_q_heads;  // (layer in range) * B + b
+      const int r = (hq % G) * T + t;          // row among the kv head's G * T query rows
+      const long long unit = (lb * s.n_kv_heads + hq / G) * a.row_blocks + r / kScoreBlockM;
+      const long long g0 = unit * a.tiles_per_unit;
+      n_slots = score_tile_owner(a.total_tiles, a.grid, g0 + a.tiles_per_unit - 1) -
+                score_tile_owner(a.total_tiles, a.grid, g0) + 1;
+    }
     float Mx = -INFINITY;
-    for (int sp = 0; sp < a.n_splits; ++sp) Mx = fmaxf(Mx, st[sp * 3]);
+    for (int sp = 0; sp < n_slots; ++sp) Mx = fmaxf(Mx, st[sp * 3]);
     if (a.window_only) {
       // denominator given: mass = sum over splits of W * 2^(M - lse * log2(e))
-      const float lse2 = a.lse[idx * a.w_last + t] * 1.4426950408889634f;
+      const float lse2 = a.lse[idx * T + t] * 1.4426950408889634f;
       float W = 0.f;
-      for (int sp = 0; sp < a.n_splits; ++sp) W += st[sp * 3 + 2] * exp2f(st[sp * 3] - lse2);
+      for (int sp = 0; sp < n_slots; ++sp) W += st[sp * 3 + 2] * exp2f(st[sp * 3] - lse2);
       sum += W;
     } else {
       float A = 0.f, W = 0.f;
-      for (int sp = 0; sp < a.n_splits; ++sp) {
+      for (int sp = 0; sp < n_slots; ++sp) {
         const float w = exp2f(st[sp * 3] - Mx);
         A += w * st[sp * 3 + 1];
         W += w * st[sp * 3 + 2];
@@ -121,7 +136,7 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
       sum += W / A;
     }
   }
-  a.scores[idx] = sum / (float)a.w_last;
+  a.scores[idx] = sum / (float)T;
 }
 
 cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st) {

@@ -3,26 +3,44 @@
 // S = Q K^T is a real dense contraction here (G * w_last query rows against
 // every prompt key), so it runs on the 5th-generation tensor cores:
 // tcgen05.mma (M = 128, N = 128, K = 16 per instruction, bf16 in, fp32 out)
-// issued by one thread, operands in shared memory in the 128-byte-swizzled
-// K-major layout, accumulators in tensor memory (TMEM).
+// issued by one thread.  The stationary operand, the block of up to 256 query
+// rows, lives in tensor memory (TMEM) as the A operand; only the streamed K
+// tiles come from shared memory (128-byte-swizzled K-major layout, written by
+// TMA), which halves the shared-memory traffic of an instruction compared with
+// both operands in shared memory.  Accumulators are three 128 x 128 fp32 slots
+// in TMEM that rotate between the MMA issuer and the statistics warps.
 //
-// One CTA per (layer, batch row, kv head, key split, block of 256 query rows),
-// three warpgroups with fixed roles:
-//   warp 0      producer: one lane streams 128-key K tiles into a 4-stage ring
-//               with TMA (cp.async.bulk.tensor, two 64-column boxes per tile, the
-//               128-byte swizzle applied by the copy engine), completion counted
-//               in bytes on full[s];
-//   warp 1      allocates TMEM; lane 0 issues the MMAs of a tile (2 row blocks x
-//               8 k-steps) into one of two accumulator buffers and commits to
-//               empty[s] (stage may be refilled) and sfull[t] (scores ready);
+// The launch is persistent: one CTA per SM.  With the whole prompt scored
+// (lt_lazy_scores) the 128-key tiles of all (layer, batch row, kv head, block of
+// 256 query rows) units form one sequence that is cut into equal contiguous
+// ranges, one per CTA, so every SM gets the same number of tiles whatever the
+// unit count; a unit that straddles a cut gets one statistics slot per piece.
+// With the denominator given (lt_lazy_scores_lse) the work items are the host's
+// key splits of the kept ranges, dealt round-robin.
+//
+// Roles (three warpgroups):
+//   warp 0      producer: one lane streams K tiles into a ring with TMA
+//               (cp.async.bulk.tensor, two 64-column boxes per tile), completion
+//               counted in bytes on full[s]; the ring never drains between pieces;
+//   warp 1      allocates TMEM; lane 0 issues the MMAs of a tile (8 k-steps per row
+//               block) into the next accumulator slot and commits to slot_full and,
+//               after the tile's last row block, to empty[s];
 //   warps 2-3   fill up the first warpgroup (register hand-over is per warpgroup);
-//   warps 4-11  statistics: thread = one query row (TMEM lane), reads its row of
-//               the 128 x 128 score block with tcgen05.ld and keeps only the
-//               running max, sum exp and windowed sum exp - no shuffles, no
-//               shared memory, nothing written until the end.  The exponentials
-//               (one MUFU instruction each) are the floor of this kernel, so
-//               these warps take the registers the first warpgroup gives up and
-//               hold a whole 128-column row in flight.
+//   warps 4-11  statistics: thread = one query row (one TMEM lane).  At a change of
+//               unit the thread writes its query row into TMEM (tcgen05.st).  It reads
+//               its row of every 128 x 128 score block with tcgen05.ld and keeps only a
+//               reference exponent, sum exp and windowed sum exp - no shuffles, no
+//               shared memory, nothing written until the end of the piece.
+//
+// Exponentials.  One ex2 per score on the special-function unit (16 per clock per
+// SM) would bound the kernel at twice the tensor-core time, so a fixed share of
+// the columns takes 2^x on the FMA pipe instead: the reference of a row is an
+// INTEGER M >= max (log2 domain), so x = t - M splits exactly into round(x) and
+// a remainder f in [-1/2, 1/2]; 2^f is a cubic (relative error 7.5e-5, far inside
+// the 1e-3 absolute tolerance of a ratio of sums) and round(x) goes into the
+// exponent field with one integer add.  The FMA-pipe work uses the packed
+// two-lane fp32 instructions (fma / add .f32x2).
+//
 // Every wait on an mbarrier is bounded in time; on expiry the kernel raises
 // LT_DEVERR_TIMEOUT in the workspace header, all roles leave their loops, TMEM
 // is freed and the kernel returns.
@@ -31,37 +49,33 @@
 
 #include "lt_internal.h"
 
+#ifndef LT_SCORES_POLY_OF8
+#define LT_SCORES_POLY_OF8 3  // of every 8 column pairs, this many take 2^x on the FMA pipe
+#endif
+
 namespace lt {
 
 namespace {
 
 constexpr int kD = 128;  // head_dim
 constexpr int kRowBytes = 256;
-constexpr int kBlockM = 256;   // query rows per CTA (2 UMMA row blocks)
-constexpr int kBlockN = 128;   // keys per tile
-constexpr int kStages = 4;
-constexpr int kQHalfBytes = kBlockM * 128;        // one d-half of Q: [256 rows][128 B]
-constexpr int kQBytes = 2 * kQHalfBytes;          // 64 KB
+constexpr int kBlockM = kScoreBlockM;  // query rows per unit (2 UMMA row blocks)
+constexpr int kBlockN = kScoreBlockN;  // keys per tile
+constexpr int kStages = 6;
 constexpr int kKHalfBytes = kBlockN * 128;        // one d-half of a K tile
 constexpr int kStageBytes = 2 * kKHalfBytes;      // 32 KB
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
 constexpr int kThreads = 384;
 constexpr int kRegsLight = 56;   // producer / MMA warpgroup after setmaxnreg.dec
 constexpr int kRegsStats = 224;  // statistics warpgroups after setmaxnreg.inc
 constexpr int kTmemCols = 512;
+constexpr int kSlots = 3;        // accumulator slots of 128 columns: TMEM columns [0, 384)
+constexpr int kQCol = 384;       // query rows (A operand): 64 columns per row block, [384, 512)
+constexpr int kPolyOf8 = LT_SCORES_POLY_OF8;
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 1.9 GHz
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 
@@ -106,7 +120,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-
 // Bounded wait that ignores the abort flag: used to let copies in flight land before the CTA exits.
 __device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity) {
   const long long t0 = clock64();
@@ -128,12 +141,14 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) | ((128u >> 4) << 24);
 
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] . B[smem]^T: A is 128 lanes x 8 columns (16 bf16 of one query row per lane, two per
+// 32-bit column, the lower d in the lower half), B a 128-key x 16-d slice of the K tile.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -156,26 +171,128 @@ __device__ __forceinline__ void tmem_ld32_at(uint32_t taddr, uint32_t (&v)[N]) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+// v[OFF .. OFF+31] into 32 consecutive columns of this thread's TMEM lane (asynchronous until tmem_st_wait)
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_st32_at(uint32_t taddr, const uint32_t (&v)[N]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n" ::"r"(taddr),
+      "r"(v[OFF + 0]), "r"(v[OFF + 1]), "r"(v[OFF + 2]), "r"(v[OFF + 3]), "r"(v[OFF + 4]), "r"(v[OFF + 5]),
+      "r"(v[OFF + 6]), "r"(v[OFF + 7]), "r"(v[OFF + 8]), "r"(v[OFF + 9]), "r"(v[OFF + 10]), "r"(v[OFF + 11]),
+      "r"(v[OFF + 12]), "r"(v[OFF + 13]), "r"(v[OFF + 14]), "r"(v[OFF + 15]), "r"(v[OFF + 16]), "r"(v[OFF + 17]),
+      "r"(v[OFF + 18]), "r"(v[OFF + 19]), "r"(v[OFF + 20]), "r"(v[OFF + 21]), "r"(v[OFF + 22]), "r"(v[OFF + 23]),
+      "r"(v[OFF + 24]), "r"(v[OFF + 25]), "r"(v[OFF + 26]), "r"(v[OFF + 27]), "r"(v[OFF + 28]), "r"(v[OFF + 29]),
+      "r"(v[OFF + 30]), "r"(v[OFF + 31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+
 // One MUFU instruction: 2^x, relative error 2^-22, results below 2^-126 flush to zero.
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
-// max of 64 values: four interleaved chains, then a small tree (short dependency depth)
+// Three-input maximum (one instruction on sm_100).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Packed two-lane fp32 arithmetic (one instruction per pair).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// max of 64 values: four interleaved chains of three-input maxima, then a small tree
 __device__ __forceinline__ float max64(const uint32_t (&v)[64]) {
-  float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]), m2 = __uint_as_float(v[2]),
-        m3 = __uint_as_float(v[3]);
+  float m0 = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+  float m1 = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+  float m2 = max3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+  float m3 = max3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
 #pragma unroll
-  for (int i = 4; i < 64; i += 4) {
-    m0 = fmaxf(m0, __uint_as_float(v[i]));
-    m1 = fmaxf(m1, __uint_as_float(v[i + 1]));
-    m2 = fmaxf(m2, __uint_as_float(v[i + 2]));
-    m3 = fmaxf(m3, __uint_as_float(v[i + 3]));
+  for (int i = 12; i < 60; i += 8) {
+    m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+    m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+    m2 = max3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+    m3 = max3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
   }
+  m0 = max3(m0, __uint_as_float(v[60]), __uint_as_float(v[61]));
+  m1 = max3(m1, __uint_as_float(v[62]), __uint_as_float(v[63]));
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
-// sum_i 2^(v_i * cs + off): four accumulators
+
+// 2^f on [-1/2, 1/2] as a cubic: least maximum relative error (7.5e-5), from a weighted least-squares
+// (Lawson) fit of p(f) / 2^f to 1 on 4001 Chebyshev nodes, coefficients rounded to float.
+constexpr float kP0 = 0.9999280571937561f, kP1 = 0.6932609677314758f, kP2 = 0.2426111251115799f,
+                kP3 = 0.0551716685295105f;
+constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round-to-nearest(x) in the low mantissa bits
+constexpr float kMinX = -125.0f;       // 2^x below this is treated as 2^-125 (keeps the exponent field positive)
+
+// sum_i 2^(v_i * cs - M) over the 64 values, M an integer (as a float): MUFU for most column pairs, the
+// FMA-pipe polynomial for kPolyOf8 of every 8 pairs.
+__device__ __forceinline__ float sum_ex2_64_mixed(const uint32_t (&v)[64], float cs, float M) {
+  const f32x2 cs2 = pack2(cs, cs), nM2 = pack2(-M, -M);
+  const f32x2 magic2 = pack2(kMagic, kMagic), mone2 = pack2(-1.f, -1.f);
+  const f32x2 p3 = pack2(kP3, kP3), p2 = pack2(kP2, kP2), p1 = pack2(kP1, kP1), p0 = pack2(kP0, kP0);
+  f32x2 acc0 = pack2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {  // pair i = columns 2i, 2i + 1
+    const f32x2 x2 = fma2(pack2u(v[2 * i], v[2 * i + 1]), cs2, nM2);
+    float xl, xh;
+    unpack2(x2, xl, xh);
+    f32x2 e2;
+    // the polynomial pairs are spread over the group of 8 so that both pipes stay fed
+    const bool poly = ((i & 7) * kPolyOf8) / 8 != (((i & 7) + 1) * kPolyOf8) / 8;
+    if (poly) {
+      const f32x2 xc = pack2(fmaxf(xl, kMinX), fmaxf(xh, kMinX));
+      const f32x2 t2 = add2(xc, magic2);                     // magic + round(x)
+      const f32x2 f2 = add2(xc, fma2(t2, mone2, magic2));    // x - round(x), exact
+      f32x2 p = fma2(p3, f2, p2);
+      p = fma2(p, f2, p1);
+      p = fma2(p, f2, p0);
+      float pl, ph, tl, th;
+      unpack2(p, pl, ph);
+      unpack2(t2, tl, th);
+      // 2^round(x): the integer sits in the low bits of t; shifted into the exponent field it adds to p's exponent
+      const float rl = __int_as_float(__float_as_int(pl) + (__float_as_int(tl) << 23));
+      const float rh = __int_as_float(__float_as_int(ph) + (__float_as_int(th) << 23));
+      e2 = pack2(rl, rh);
+    } else {
+      e2 = pack2(ex2(xl), ex2(xh));
+    }
+    if ((i & 3) == 0) acc0 = add2(acc0, e2);
+    else if ((i & 3) == 1) acc1 = add2(acc1, e2);
+    else if ((i & 3) == 2) acc2 = add2(acc2, e2);
+    else acc3 = add2(acc3, e2);
+  }
+  float a, b;
+  unpack2(add2(add2(acc0, acc1), add2(acc2, acc3)), a, b);
+  return a + b;
+}
+// The same sum with every exponential on the MUFU; -inf entries (masked columns) contribute 0.
 __device__ __forceinline__ float sum_ex2_64(const uint32_t (&v)[64], float cs, float off) {
   float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
@@ -190,55 +307,103 @@ __device__ __forceinline__ float sum_ex2_64(const uint32_t (&v)[64], float cs, f
 
 }  // namespace
 
-// grid (n_splits * row_blocks, B * Hkv, L); block 384.
 struct KeyMaps {
   CUtensorMap m[LT_MAX_LAYERS];  // layer l's K cache as a [B * Hkv * capacity][128] bf16 matrix, box 64 x 128
 };
+
+// One contiguous run of tiles of one unit, handled by one CTA.
+struct Piece {
+  int l, b, h, rb;  // the unit: layer, batch row, kv head, block of 256 query rows
+  int unit;         // its index (changes <=> the query rows in TMEM must be replaced)
+  int k0, k1;       // keys of the piece: statistics cover [k0, k1)
+  int ts0;          // first key of the piece's first tile
+  int n_tiles;
+  int slot;         // statistics slot of the piece within its rows
+};
+
+// The pieces of this CTA, in order.  `cursor` starts at 0 (every role walks the same list on its own).
+__device__ __forceinline__ bool next_piece(const ScoreArgs& a, long long& cursor, Piece& p) {
+  const lt_shape& s = a.s;
+  int unit, k0, k1, ts0, n_tiles, slot;
+  if (a.streamk) {
+    long long g_begin, g_end;
+    score_cta_tiles(a.total_tiles, gridDim.x, blockIdx.x, &g_begin, &g_end);
+    const long long g = g_begin + cursor;
+    if (g >= g_end) return false;
+    const int TU = a.tiles_per_unit;
+    unit = (int)(g / TU);
+    const int ta = (int)(g - (long long)unit * TU);
+    const int tb = (int)min((long long)TU, ta + (g_end - g));
+    k0 = ta * kBlockN;
+    k1 = min(tb * kBlockN, a.n_ctx);
+    ts0 = k0;
+    n_tiles = tb - ta;
+    slot = (int)blockIdx.x - score_tile_owner(a.total_tiles, gridDim.x, (long long)unit * TU);
+    cursor += n_tiles;
+  } else {
+    const long long n_items = (long long)a.n_units * a.n_splits;
+    const long long item = (long long)blockIdx.x + cursor * gridDim.x;
+    if (item >= n_items) return false;
+    unit = (int)(item / a.n_splits);
+    slot = (int)(item - (long long)unit * a.n_splits);
+    score_split_range(a, slot, &k0, &k1);
+    // Paged caches: tiles start on multiples of 128 keys so that none straddles two pages (the page size
+    // is a multiple of 128); the keys before k0 in the first tile are masked by the statistics warps.
+    ts0 = s.page_size > 0 ? (k0 & ~(kBlockN - 1)) : k0;
+    n_tiles = k1 > k0 ? (k1 - ts0 + kBlockN - 1) / kBlockN : 0;
+    cursor += 1;
+  }
+  p.unit = unit;
+  p.rb = unit % a.row_blocks;
+  int x = unit / a.row_blocks;
+  p.h = x % s.n_kv_heads;
+  x /= s.n_kv_heads;
+  p.b = x % s.batch;
+  p.l = a.layer_begin + x / s.batch;
+  p.k0 = k0;
+  p.k1 = k1;
+  p.ts0 = ts0;
+  p.n_tiles = n_tiles;
+  p.slot = slot;
+  return true;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
     scores_umma_kernel(ScoreArgs a, const __grid_constant__ KeyMaps maps) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern of the MMA is a function of address bits 4..9
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const uint32_t sQ = smem_u32(smem);
-  const uint32_t sK = sQ + kQBytes;
-  uint8_t* bar_mem = smem + kQBytes + kStages * kStageBytes;
+  const uint32_t sK = smem_u32(smem);
+  uint8_t* bar_mem = smem + kStages * kStageBytes;
   const uint32_t bar0 = smem_u32(bar_mem);
-  const uint32_t bar_full = bar0;                      // [kStages]
-  const uint32_t bar_empty = bar0 + 8 * kStages;       // [kStages]
-  const uint32_t bar_sfull = bar0 + 16 * kStages;      // [2]
-  const uint32_t bar_sempty = bar_sfull + 16;          // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 16 * kStages + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * kStages + 40);
+  const uint32_t bar_full = bar0;                          // [kStages]   K tile landed
+  const uint32_t bar_empty = bar0 + 8 * kStages;           // [kStages]   K tile consumed by the MMAs
+  const uint32_t bar_sfull = bar0 + 16 * kStages;          // [kSlots]    accumulator slot holds a score block
+  const uint32_t bar_sempty = bar_sfull + 8 * kSlots;      // [kSlots]    score block is in registers
+  const uint32_t bar_qready = bar_sempty + 8 * kSlots;     // [2]         query rows of a row block are in TMEM
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 16 * kStages + 16 * kSlots + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * kStages + 16 * kSlots + 24);
+  static_assert(16 * kStages + 16 * kSlots + 32 <= kBarBytes, "barrier area too small");
 
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int T = a.w_last;
   const int M = G * T;
-  const int sp = blockIdx.x % a.n_splits, rb = blockIdx.x / a.n_splits;
-  const int b = blockIdx.y / s.n_kv_heads, h = blockIdx.y % s.n_kv_heads;
-  const int l = a.layer_begin + blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_ctx = a.n_ctx;
-  int k0, k1;
-  score_split_range(a, sp, &k0, &k1);
-  // Paged caches: tiles start on multiples of 128 keys so that none straddles two pages (the page size
-  // is a multiple of 128); the keys before k0 in the first tile are masked by the statistics warps.
-  const int ts0 = s.page_size > 0 ? (k0 & ~(kBlockN - 1)) : k0;
-  const int n_tiles = k1 > k0 ? (k1 - ts0 + kBlockN - 1) / kBlockN : 0;
-  const int rows_here = min(kBlockM, M - rb * kBlockM);  // valid query rows of this CTA
-  const int n_mb = (rows_here + 127) / 128;              // UMMA row blocks in use
 
-  // ---- set-up: barriers, TMEM, Q tile ------------------------------------------
+  // ---- set-up: barriers, TMEM ----------------------------------------------------
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_full + 8 * i, 1);
       mbar_init(bar_empty + 8 * i, 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kSlots; ++i) {
       mbar_init(bar_sfull + 8 * i, 1);
-      mbar_init(bar_sempty + 8 * i, 256);
+      mbar_init(bar_sempty + 8 * i, 128);
     }
+    mbar_init(bar_qready, 128);
+    mbar_init(bar_qready + 8, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -248,189 +413,251 @@ __global__ void __launch_bounds__(kThreads, 1)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
-  {
-    const uint8_t* qb = (const uint8_t*)a.q_tail +
-                        ((((long long)l * s.batch + b) * s.n_q_heads + (long long)h * G) * T + (long long)rb * kBlockM) *
-                            kRowBytes;
-    for (int idx = threadIdx.x; idx < kBlockM * 16; idx += kThreads) {
-      const int r = idx >> 4, p = idx & 15;
-      const bool valid = r < rows_here;
-      cp_async16(sQ + (p >> 3) * kQHalfBytes + r * 128 + (((p & 7) ^ (r & 7)) << 4),
-                 qb + (long long)(valid ? r : 0) * kRowBytes + p * 16, valid ? 16 : 0);
-    }
-    cp_async_commit();
-    cp_async_wait<0>();
-    fence_proxy_async();
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // tensor-map row of key j of this (b, kv head); j is a tile start
-  auto map_row = [&](int j) {
-    if (s.page_size <= 0) return (b * s.n_kv_heads + h) * s.full_capacity + j;
-    const int page = s.block_table[(long long)b * s.pages_per_seq + j / s.page_size];
-    return (page * s.n_kv_heads + h) * s.page_size + j % s.page_size;
-  };
+  // rows of query block rb that exist, and the UMMA row blocks they fill
+  auto rows_of = [&](int rb) { return min(kBlockM, M - rb * kBlockM); };
+  auto mbs_of = [&](int rb) { return (rows_of(rb) + 127) / 128; };
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsLight));
-  if (warp == 0) {
-    // ===== producer =====
-    // Rows past the split end are real cache rows (or zero past the end of the
-    // cache): the statistics warps never look at those columns.
-    if (lane == 0) {
-      const CUtensorMap* map = &maps.m[l];
-      bool ok = true;
-      int issued = 0;
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int st = it % kStages;
-        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * st, ((it / kStages) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        const uint32_t dst = sK + st * kStageBytes;
-        const uint32_t bar = bar_full + 8 * st;
-        mbar_expect_tx(bar, kStageBytes);
-        const int y = map_row(ts0 + it * kBlockN);
-        tma_load_2d(dst, map, 0, y, bar);
-        tma_load_2d(dst + kKHalfBytes, map, 64, y, bar);
-        issued = it + 1;
-      }
-      if (!ok) {
-        // gave up: let the copies already issued land before the shared memory goes away
-        for (int j = max(0, issued - kStages); j < issued; ++j)
-          mbar_wait_quiet(bar_full + 8 * (j % kStages), (j / kStages) & 1);
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ===== MMA issuer =====
-    if (lane == 0) {
-      bool ok = true;
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int st = it % kStages, t = it & 1;
-        if (it >= 2) ok = mbar_wait(bar_sempty + 8 * t, ((it >> 1) & 1) ^ 1, abort_flag);
-        if (ok) ok = mbar_wait(bar_full + 8 * st, (it / kStages) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        fence_proxy_async();
-        for (int mb = 0; mb < n_mb; ++mb) {
-          const uint32_t d_tmem = tmem_base + t * 256 + mb * 128;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + mb * (128 * 128) + (ks & 3) * 32;
-            const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
-            umma_bf16(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
+    if (warp == 0) {
+      // ===== producer =====
+      // Rows past the piece's last key are real cache rows (or zero past the end of the
+      // cache): the statistics warps never look at those columns.
+      if (lane == 0) {
+        bool ok = true;
+        long long cursor = 0;
+        int kt = 0;  // tiles issued by this CTA so far: stage kt % kStages, use kt / kStages of that stage
+        Piece p;
+        while (ok && next_piece(a, cursor, p)) {
+          const CUtensorMap* map = &maps.m[p.l];
+          for (int it = 0; it < p.n_tiles; ++it, ++kt) {
+            const int st = kt % kStages;
+            if (kt >= kStages) ok = mbar_wait(bar_empty + 8 * st, ((kt / kStages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            const uint32_t dst = sK + st * kStageBytes;
+            const uint32_t bar = bar_full + 8 * st;
+            mbar_expect_tx(bar, kStageBytes);
+            const int j = p.ts0 + it * kBlockN;
+            int y;
+            if (s.page_size <= 0) {
+              y = (p.b * s.n_kv_heads + p.h) * s.full_capacity + j;
+            } else {
+              const int page = s.block_table[(long long)p.b * s.pages_per_seq + j / s.page_size];
+              y = (page * s.n_kv_heads + p.h) * s.page_size + j % s.page_size;
+            }
+            tma_load_2d(dst, map, 0, y, bar);
+            tma_load_2d(dst + kKHalfBytes, map, 64, y, bar);
           }
         }
-        umma_commit(bar_empty + 8 * st);
-        umma_commit(bar_sfull + 8 * t);
+        if (!ok) {
+          // gave up: let the copies already issued land before the shared memory goes away
+          for (int j = max(0, kt - kStages); j < kt; ++j)
+            mbar_wait_quiet(bar_full + 8 * (j % kStages), (j / kStages) & 1);
+        }
       }
+      __syncwarp();
+    } else if (warp == 1) {
+      // ===== MMA issuer =====
+      if (lane == 0) {
+        bool ok = true;
+        long long cursor = 0;
+        int kt = 0;          // tiles consumed so far
+        int uc = 0;          // score blocks issued so far: slot uc % kSlots, use uc / kSlots of that slot
+        int q_uses0 = 0, q_uses1 = 0;
+        int prev_unit = -1;
+        Piece p;
+        while (ok && next_piece(a, cursor, p)) {
+          const int n_mb = mbs_of(p.rb);
+          if (p.unit != prev_unit && p.n_tiles > 0) {
+            // the statistics warps replace the query rows in TMEM (after the last MMAs that read the old ones)
+            ok = mbar_wait(bar_qready, q_uses0 & 1, abort_flag);
+            ++q_uses0;
+            if (ok && n_mb > 1) {
+              ok = mbar_wait(bar_qready + 8, q_uses1 & 1, abort_flag);
+              ++q_uses1;
+            }
+            if (!ok) break;
+            tc_fence_after();
+            prev_unit = p.unit;
+          }
+          for (int it = 0; it < p.n_tiles && ok; ++it, ++kt) {
+            const int st = kt % kStages;
+            ok = mbar_wait(bar_full + 8 * st, (kt / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            for (int mb = 0; mb < n_mb; ++mb, ++uc) {
+              const int slot = uc % kSlots, use = uc / kSlots;
+              if (use > 0) {
+                ok = mbar_wait(bar_sempty + 8 * slot, (use - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+              }
+              const uint32_t d_tmem = tmem_base + slot * 128;
+              const uint32_t a_tmem = tmem_base + kQCol + mb * 64;
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
+                umma_bf16_ts(d_tmem, a_tmem + ks * 8, umma_desc(b_addr), ks > 0 ? 1u : 0u);
+              }
+              umma_commit(bar_sfull + 8 * slot);
+            }
+            if (!ok) break;
+            umma_commit(bar_empty + 8 * st);
+          }
+        }
+      }
+      __syncwarp();
     }
-    __syncwarp();
-  }
   } else {
     // ===== statistics =====
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsStats));
-    // A tile's 128 columns are taken in two halves of 64 registers.  The load of
+    // A score block's 128 columns are taken in two halves of 64 registers.  The load of
     // one half is in flight while the exponentials of the other half run, and
-    // the accumulator buffer is handed back to the MMA warp as soon as both
+    // the accumulator slot is handed back to the MMA warp as soon as both
     // halves sit in registers.
-    const int sw = warp - 4;
-    const int mb = sw >> 2;          // row block of this warp
-    const int quad = warp & 3;       // TMEM lane quadrant this warp may read
-    const int r_local = mb * 128 + quad * 32 + lane;
-    const int r = rb * kBlockM + r_local;
-    const bool row_valid = r_local < rows_here;
-    const int vis = n_ctx - T + (r % T);  // last visible key of this row
+    const int mb = (warp - 4) >> 2;  // row block of this warp
+    const int quad = warp & 3;       // TMEM lane quadrant this warp may access
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float cs = a.cs;
     const int S = s.n_sink;
-    const int win_lo = s.recent_per_row ? vis - s.n_recent + 1 : n_ctx - s.n_recent;  // first recent key of this row
-    const int lim = min(vis, k1 - 1);     // last key of this split that the row may see
-    float m = -INFINITY, sA = 0.f, sWn = 0.f;
-    const bool active = mb < n_mb;
-    const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + mb * 128;
-
-    // statistics of one half (64 keys from jb) already in registers
-    auto half_stats = [&](uint32_t (&v)[64], int jb) {
-      const int jend = jb + 64;
-      const bool all_win = (jend <= S) || (jb >= win_lo);
-      const bool no_win = (jb >= S) && (jend <= win_lo);
-      if ((jb >= k0) && (jend - 1 <= lim) && (all_win || no_win)) {
-        const float mn = fmaxf(m, max64(v));
-        const float corr = ex2((m - mn) * cs);
-        const float ps = sum_ex2_64(v, cs, -mn * cs);
-        sA = fmaf(sA, corr, ps);
-        sWn = fmaf(sWn, corr, all_win ? ps : 0.f);
-        m = mn;
-      } else if (max(jb, k0) <= min(jend - 1, lim)) {
-        // boundary half (split start, causal tail, split end or window edge): mask in place.
-        // 2^(-inf) = 0, and at least one key is visible, so the maximum is finite.
-#pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (jb + i > lim || jb + i < k0) v[i] = 0xff800000u;
-        const float mn = fmaxf(m, max64(v));
-        const float corr = ex2((m - mn) * cs);
-        const float off = -mn * cs;
-        const float ps = sum_ex2_64(v, cs, off);
-#pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          const int j = jb + i;
-          if (!(j < S || j >= win_lo)) v[i] = 0xff800000u;
-        }
-        const float pw = sum_ex2_64(v, cs, off);
-        sA = fmaf(sA, corr, ps);
-        sWn = fmaf(sWn, corr, pw);
-        m = mn;
-      }
-    };
 
     bool ok = true;
+    long long cursor = 0;
+    int uc = 0;  // score blocks issued by the MMA warp before the current piece
+    int prev_unit = -1;
+    Piece p;
     uint32_t va[64], vb[64];
-    if (n_tiles > 0) {
-      ok = mbar_wait(bar_sfull, 0, abort_flag);
-      tc_fence_after();
-      if (ok && active) {
-        tmem_ld32_at<0>(lane_base, va);
-        tmem_ld32_at<32>(lane_base + 32, va);
+    while (ok && next_piece(a, cursor, p)) {
+      const int rows_here = rows_of(p.rb);
+      const int n_mb = (rows_here + 127) / 128;
+      const bool active = mb < n_mb;
+      const int r_local = mb * 128 + quad * 32 + lane;
+      const int r = p.rb * kBlockM + r_local;   // row of the kv head's G * T query rows
+      const bool row_valid = r_local < rows_here;
+      const int g = r / T, tq = r - g * T;
+      const long long rowid =
+          (((long long)(p.l - a.layer_begin) * s.batch + p.b) * s.n_q_heads + p.h * G + g) * T + tq;
+      float* stp = a.stats + (rowid * a.n_splits + p.slot) * 3;
+      if (!active || p.n_tiles == 0) {
+        // nothing to read: an idle row block, or an empty key range (its slot still gets neutral statistics)
+        if (active && row_valid) {
+          stp[0] = -INFINITY;
+          stp[1] = 0.f;
+          stp[2] = 0.f;
+        }
+        uc += p.n_tiles * n_mb;
+        continue;
       }
-    }
-    for (int it = 0; it < n_tiles && ok; ++it) {
-      const int t = it & 1;
-      const int kb = ts0 + it * kBlockN;
-      const uint32_t taddr = lane_base + t * 256;
-      // first half is (being) loaded; start the second half, then work on the first
-      tmem_ld_wait();
-      if (active) {
+      if (p.unit != prev_unit) {
+        // this thread's query row -> TMEM (the A operand of its row block).  Every MMA that read the old
+        // rows of this block has completed: its score block was consumed by this warpgroup.
+        const uint4* qrow = reinterpret_cast<const uint4*>(
+            (const uint8_t*)a.q_tail +
+            ((((long long)p.l * s.batch + p.b) * s.n_q_heads + (long long)p.h * G) * T + (row_valid ? r : 0)) *
+                kRowBytes);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const uint4 x = row_valid ? __ldg(qrow + i) : make_uint4(0u, 0u, 0u, 0u);
+          va[4 * i] = x.x;
+          va[4 * i + 1] = x.y;
+          va[4 * i + 2] = x.z;
+          va[4 * i + 3] = x.w;
+        }
+        tmem_st32_at<0>(lane_addr + kQCol + mb * 64, va);
+        tmem_st32_at<32>(lane_addr + kQCol + mb * 64 + 32, va);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bar_qready + 8 * mb);
+        prev_unit = p.unit;
+      }
+      const int k0 = p.k0, k1 = p.k1;
+      const int vis = n_ctx - T + tq;  // last visible key of this row
+      const int win_lo = s.recent_per_row ? vis - s.n_recent + 1 : n_ctx - s.n_recent;  // first recent key of this row
+      const int lim = min(vis, k1 - 1);     // last key of this piece that the row may see
+      float Mr = -INFINITY, sA = 0.f, sWn = 0.f;  // reference exponent (an integer), sum, windowed sum
+
+      // statistics of one half (64 keys from jb) already in registers
+      auto half_stats = [&](uint32_t (&v)[64], int jb) {
+        const int jend = jb + 64;
+        const bool all_win = (jend <= S) || (jb >= win_lo);
+        const bool no_win = (jb >= S) && (jend <= win_lo);
+        if ((jb >= k0) && (jend - 1 <= lim) && (all_win || no_win)) {
+          const float Mn = fmaxf(Mr, ceilf(max64(v) * cs));
+          const float corr = ex2(Mr - Mn);
+          const float ps = sum_ex2_64_mixed(v, cs, Mn);
+          sA = fmaf(sA, corr, ps);
+          sWn = fmaf(sWn, corr, all_win ? ps : 0.f);
+          Mr = Mn;
+        } else if (max(jb, k0) <= min(jend - 1, lim)) {
+          // boundary half (piece start, causal tail, piece end or window edge): mask in place.
+          // 2^(-inf) = 0, and at least one key is visible, so the maximum is finite.
+#pragma unroll
+          for (int i = 0; i < 64; ++i)
+            if (jb + i > lim || jb + i < k0) v[i] = 0xff800000u;
+          const float Mn = fmaxf(Mr, ceilf(max64(v) * cs));
+          const float corr = ex2(Mr - Mn);
+          const float ps = sum_ex2_64(v, cs, -Mn);
+#pragma unroll
+          for (int i = 0; i < 64; ++i) {
+            const int j = jb + i;
+            if (!(j < S || j >= win_lo)) v[i] = 0xff800000u;
+          }
+          const float pw = sum_ex2_64(v, cs, -Mn);
+          sA = fmaf(sA, corr, ps);
+          sWn = fmaf(sWn, corr, pw);
+          Mr = Mn;
+        }
+      };
+
+      // score block `it` of this row block is block uc + it * n_mb + mb of the CTA
+      {
+        const int u = uc + mb;
+        const int sl = u % kSlots;
+        ok = mbar_wait(bar_sfull + 8 * sl, (u / kSlots) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        tmem_ld32_at<0>(lane_addr + sl * 128, va);
+        tmem_ld32_at<32>(lane_addr + sl * 128 + 32, va);
+      }
+      for (int it = 0; it < p.n_tiles; ++it) {
+        const int u = uc + it * n_mb + mb;
+        const int sl = u % kSlots;
+        const int kb = p.ts0 + it * kBlockN;
+        const uint32_t taddr = lane_addr + sl * 128;
+        // first half is (being) loaded; start the second half, then work on the first
+        tmem_ld_wait();
         tmem_ld32_at<0>(taddr + 64, vb);
         tmem_ld32_at<32>(taddr + 96, vb);
         half_stats(va, kb);
-      }
-      tmem_ld_wait();
-      // both halves are in registers: the accumulator buffer may be overwritten
-      tc_fence_before();
-      mbar_arrive(bar_sempty + 8 * t);
-      if (it + 1 < n_tiles) {
-        const int tn = (it + 1) & 1;
-        ok = mbar_wait(bar_sfull + 8 * tn, ((it + 1) >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        if (active) {
-          tmem_ld32_at<0>(lane_base + tn * 256, va);
-          tmem_ld32_at<32>(lane_base + tn * 256 + 32, va);
+        tmem_ld_wait();
+        // both halves are in registers: the accumulator slot may be overwritten
+        tc_fence_before();
+        mbar_arrive(bar_sempty + 8 * sl);
+        if (it + 1 < p.n_tiles) {
+          const int un = u + n_mb;
+          const int sn = un % kSlots;
+          ok = mbar_wait(bar_sfull + 8 * sn, (un / kSlots) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          tmem_ld32_at<0>(lane_addr + sn * 128, va);
+          tmem_ld32_at<32>(lane_addr + sn * 128 + 32, va);
         }
+        half_stats(vb, kb + 64);
       }
-      if (active) half_stats(vb, kb + 64);
+      if (!ok) break;
+      if (row_valid) {
+        stp[0] = Mr;
+        stp[1] = sA;
+        stp[2] = sWn;
+      }
+      uc += p.n_tiles * n_mb;
     }
     tmem_ld_wait();
-    if (ok && row_valid) {
-      const int g = r / T, tq = r - g * T;
-      const long long rowid = (((long long)l * s.batch + b) * s.n_q_heads + h * G + g) * T + tq;
-      float* stp = a.stats + (rowid * a.n_splits + sp) * 3;
-      stp[0] = m * cs;
-      stp[1] = sA;
-      stp[2] = sWn;
-    }
   }
 
   // ---- teardown ------------------------------------------------------------------
@@ -468,10 +695,8 @@ EncodeTiledFn encode_tiled_fn() {
 }
 }  // namespace
 
+// grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 384.
 cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
-  const int G = a.s.n_q_heads / a.s.n_kv_heads;
-  const int M = G * a.w_last;
-  const int row_blocks = (M + kBlockM - 1) / kBlockM;
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return cudaErrorNotSupported;
   const cuuint64_t rows_total = a.s.page_size > 0 ? (cuuint64_t)a.s.n_pages * a.s.n_kv_heads * a.s.page_size
@@ -492,8 +717,7 @@ cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStr
     if (l < a.layer_begin || l >= l_end) local.m[l] = local.m[a.layer_begin];
   cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  dim3 grid(a.n_splits * row_blocks, a.s.batch * a.s.n_kv_heads, a.layer_count);
-  scores_umma_kernel<<<grid, kThreads, kSmemBytes, st>>>(a, local);
+  scores_umma_kernel<<<a.grid, kThreads, kSmemBytes, st>>>(a, local);
   return cudaGetLastError();
 }
 
