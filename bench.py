@@ -37,9 +37,10 @@ METRIC = "hybrid decode-attn tokens/s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes of one decode-kernel launch from the committed ncu capture, as a
-# ratio to the algorithmic bytes of that launch (profiles/); None until measured.
-NCU_TRAFFIC_RATIO = 1.004  # profiles/decode_mma_kernel__llama3_8b_32k_full_stack_dram_bytes.md (full-size launches)
+# DRAM bytes of one decode-kernel launch as a ratio to the algorithmic bytes of that launch, from the
+# committed DRAM-byte capture of the 4-layer small case (the counters are not read during a timed run, so
+# the line's traffic figure is this constant ratio times the algorithmic bytes, and is labelled as such).
+NCU_TRAFFIC_RATIO = 1.004
 
 
 def _peaks():
@@ -386,6 +387,14 @@ def run_ours(args):
     mask_hybrid = torch.zeros_like(wl.mask)
     mask_hybrid[torch.as_tensor(wl.planted, device=device)] = 1
     variants = run_variants(wl, mask_hybrid) if world == 1 else {}
+    per_layer = run_per_layer_calls(wl, mask_hybrid, peak) if world == 1 else None
+    other = {}
+    if world == 1 and not args.no_other_configs:
+        # the other paper-shaped workloads, one stack at a time (the benchmark stack is freed first)
+        del wl
+        import gc
+        gc.collect(); torch.cuda.empty_cache()
+        other = run_other_configs(device, peak, gpu_index)
 
     if rank == 0:
         hybrid_step_ms = decode_ms_total / (K * T)
@@ -409,7 +418,9 @@ def run_ours(args):
                          "kernel": "lt_decode_step (persistent split-KV kernel: append + attend + merge), hybrid mask",
                          "algorithmic_bytes_per_launch": float(bytes_per_step.mean()),
                          "ms_per_launch": float(attn_ms.mean()),
-                         "traffic": (float(bytes_per_step.mean()) * NCU_TRAFFIC_RATIO) if NCU_TRAFFIC_RATIO else None},
+                         "traffic": (float(bytes_per_step.mean()) * NCU_TRAFFIC_RATIO) if NCU_TRAFFIC_RATIO else None,
+                         "traffic_how": "estimated: algorithmic bytes x the DRAM-bytes / algorithmic-bytes ratio of the "
+                                        "committed small-case ncu capture (not re-measured in this run)"},
             "cpu_baseline": cpu,
             "detail": {
                 "hybrid": {"step_ms": hybrid_step_ms, "attn_ms": float(attn_ms.mean()),
@@ -425,6 +436,8 @@ def run_ours(args):
                 "lazy_score_routes_max_abs_diff": routes_diff,
                 "lazy_score_kernel_roofs": score_roofs,
                 "variants": variants,
+                "per_layer_calls": per_layer,
+                "other_configs": other,
                 "paper_context": "paper reports up to 2.17x whole-model throughput vs full attention on A100 "
                                  "(Mistral-7B, 16K, max batch); other hardware, not the target",
             },
@@ -490,6 +503,209 @@ def run_variants(wl, mask_hybrid):
     res["fp8_caches"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs_of_8bit_bytes": kv8 / (ms * 1e-3) / 1e9}
     del k8, v8, ks8, vs8, ws8
     return res
+
+
+def _time_decode_steps(lt, shape, tables, mask, seq, n0, step_inputs, out, ws, steps, warm=3):
+    """Mean ms of `steps` fused decode steps starting from length n0 (CUDA events on the current stream)."""
+    seq.fill_(n0)
+    for i in range(warm):
+        q, k, v = step_inputs[i % len(step_inputs)]
+        lt.decode_step(shape, q, k, v, tables, mask, seq, out, ws)
+    torch.cuda.synchronize()
+    seq.fill_(n0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        q, k, v = step_inputs[i % len(step_inputs)]
+        lt.decode_step(shape, q, k, v, tables, mask, seq, out, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def run_per_layer_calls(wl, mask_hybrid, peak):
+    """The deployment form of the step: a model calls the cache-updating attention once per layer (its other
+    layers run in between), so a step is n_layers launches of one layer each; the last one advances seq_lens."""
+    cfg, lt = wl.cfg, wl.lt
+    L, B = cfg.n_layers, cfg.batch
+    steps = 12
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=wl.device)
+    q, k, v = wl.step_inputs[0]
+
+    def one_step():
+        for l in range(L):
+            lt.decode_step(wl.shape, q, k, v, wl.tables, mask_hybrid, seq, wl.out, wl.ws, layer_begin=l, layer_count=1,
+                           advance_seq_lens=(l == L - 1))
+
+    for _ in range(3):
+        one_step()
+    torch.cuda.synchronize()
+    seq.fill_(cfg.n_ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(wl.ws) == 0
+    ms = e0.elapsed_time(e1) / steps
+    nbytes = float(np.mean([algorithmic_bytes_decode(cfg, cfg.n_ctx + i + 1, cfg.n_lazy) for i in range(steps)]))
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"launches_per_step": L, "step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": gbs,
+            "frac_of_peak": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
+
+def run_other_configs(device, peak, gpu_index):
+    """Throughput of the other paper-shaped workloads (detail only; the headline stays the 32K stack):
+    the Llama-2-7B-shaped MHA 4K stack (hybrid against all-full), the Llama-3.1-8B-shaped 128K stack with
+    the lazy fraction swept over 0 / 25 / 50 / 75 %, and the QwQ-32B-shaped long generation as a
+    graph-replayed loop.  One stack lives on the device at a time."""
+    import gc
+
+    from synth import CONFIGS
+    res = {}
+
+    def step_metrics(cfg, ms, n_lazy, n_mean):
+        nbytes = algorithmic_bytes_decode(cfg, n_mean, n_lazy)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"step_ms": ms, "decode_tokens_per_s": cfg.batch / (ms * 1e-3), "algorithmic_bytes": nbytes, "gbs": gbs,
+                "frac_of_peak": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
+    def score_ms(wl, iters=5):
+        cfg, lt = wl.cfg, wl.lt
+        for _ in range(2):
+            lt.lazy_scores(wl.shape, wl.q_tail, wl.tables, cfg.n_ctx, cfg.w_last, wl.scores, wl.ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            lt.lazy_scores(wl.shape, wl.q_tail, wl.tables, cfg.n_ctx, cfg.w_last, wl.scores, wl.ws)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    # ---- Llama-2-7B-shaped MHA stack, 4K context ------------------------------------------------------
+    try:
+        cfg = CONFIGS["llama2_7b_4k"]
+        wl = Workload(cfg, device)
+        lt = wl.lt
+        steps = 16
+        s_ms = score_ms(wl)
+        wl.identify()
+        torch.cuda.synchronize()
+        assert sorted(np.nonzero(wl.mask.cpu().numpy())[0].tolist()) == wl.planted
+        n_mean = cfg.n_ctx + (steps + 1) / 2
+        hyb = _time_decode_steps(lt, wl.shape, wl.tables, wl.mask, wl.seq, cfg.n_ctx, wl.step_inputs, wl.out, wl.ws, steps)
+        full_mask = torch.zeros_like(wl.mask)
+        full = _time_decode_steps(lt, wl.shape, wl.tables, full_mask, wl.seq, cfg.n_ctx, wl.step_inputs, wl.out, wl.ws, steps)
+        assert lt.check(wl.ws) == 0
+        h, f = step_metrics(cfg, hyb, cfg.n_lazy, n_mean), step_metrics(cfg, full, 0, n_mean)
+        res["llama2_7b_4k"] = {"shape": "32 layers, 32 q / 32 kv heads (MHA), batch 32, context 4096, 16 lazy",
+                               "lazy_score_ms": s_ms, "hybrid": h, "all_full": f,
+                               "hybrid_over_all_full": full / hyb,
+                               "byte_ratio_ceiling": f["algorithmic_bytes"] / h["algorithmic_bytes"]}
+        del wl
+    except torch.cuda.OutOfMemoryError as e:  # a smaller device: say so instead of failing the headline
+        res["llama2_7b_4k"] = {"skipped": f"out of device memory: {e}"[:200]}
+    gc.collect(); torch.cuda.empty_cache()
+
+    # ---- Llama-3.1-8B-shaped stack, 128K context, lazy fraction sweep ---------------------------------------
+    try:
+        cfg = CONFIGS["llama31_8b_128k"]
+        wl = Workload(cfg, device)
+        lt = wl.lt
+        steps = 16
+        L = cfg.n_layers
+        s_ms = score_ms(wl)
+        n_mean = cfg.n_ctx + (steps + 1) / 2
+        sweep, base_ms = {}, None
+        for n_lazy in (0, L // 4, L // 2, 3 * L // 4):
+            lt.select_lazy(wl.scores, L, cfg.batch, cfg.n_q_heads, n_lazy, wl.mask)
+            wl.seq.copy_(wl.seq0)
+            lt.stream_init(wl.shape, wl.mask, wl.tables, wl.seq, ws=wl.ws)
+            ms = _time_decode_steps(lt, wl.shape, wl.tables, wl.mask, wl.seq, cfg.n_ctx, wl.step_inputs, wl.out, wl.ws, steps)
+            m = step_metrics(cfg, ms, n_lazy, n_mean)
+            if base_ms is None:
+                base_ms, base_bytes = ms, m["algorithmic_bytes"]
+            m["speedup_over_all_full"] = base_ms / ms
+            m["byte_ratio_ceiling"] = base_bytes / m["algorithmic_bytes"]
+            sweep[f"{100 * n_lazy // L}%_lazy"] = m
+        assert lt.check(wl.ws) == 0
+        res["llama31_8b_128k"] = {"shape": "32 layers, 32 q / 8 kv heads, batch 2, context 131072, window 4 + 4092",
+                                  "lazy_score_ms": s_ms, "lazy_fraction_sweep": sweep}
+        del wl
+    except torch.cuda.OutOfMemoryError as e:
+        res["llama31_8b_128k"] = {"skipped": f"out of device memory: {e}"[:200]}
+    gc.collect(); torch.cuda.empty_cache()
+
+    # ---- QwQ-32B-shaped long generation: eager loop against a graph-replayed loop -------------------------
+    try:
+        cfg = CONFIGS["qwq32b_longgen"]
+        wl = Workload(cfg, device)
+        lt = wl.lt
+        L, B = cfg.n_layers, cfg.batch
+        n_steps, per_graph = 2048, 16
+        g = np.random.default_rng(41)
+        m = np.zeros(L, dtype=np.uint8); m[g.permutation(L)[:cfg.n_lazy]] = 1     # the prompt is shorter than the window:
+        wl.mask.copy_(torch.from_numpy(m).to(device))                             # every ratio is 1, so the mask is given
+        q, k, v = wl.step_inputs[0]
+
+        def reset():
+            wl.seq.copy_(wl.seq0)
+            lt.stream_init(wl.shape, wl.mask, wl.tables, wl.seq, ws=wl.ws)
+
+        reset()
+        for _ in range(3):
+            lt.decode_step(wl.shape, q, k, v, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
+        torch.cuda.synchronize()
+        reset()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_steps):
+            lt.decode_step(wl.shape, q, k, v, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
+        e1.record()
+        torch.cuda.synchronize()
+        eager_ms = e0.elapsed_time(e1)
+        # one captured graph of 16 steps (the step reads lengths and mask from the device), replayed 128 times
+        reset()
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(per_graph):
+                    lt.decode_step(wl.shape, q, k, v, wl.tables, wl.mask, wl.seq, wl.out, wl.ws)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        reset()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        reset()
+        e0.record()
+        for _ in range(n_steps // per_graph):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_ms = e0.elapsed_time(e1)
+        assert lt.check(wl.ws) == 0 and wl.seq.cpu().tolist() == [cfg.n_ctx + n_steps] * B
+        nbytes = float(np.mean([algorithmic_bytes_decode(cfg, cfg.n_ctx + i + 1, cfg.n_lazy) for i in range(n_steps)]))
+        res["qwq32b_longgen"] = {
+            "shape": "64 layers, 40 q / 8 kv heads (group of 5), batch 4, prompt 1024, 32 lazy, window 4 + 4092",
+            "decode_steps": n_steps, "context_from_to": [cfg.n_ctx, cfg.n_ctx + n_steps],
+            "mean_algorithmic_bytes_per_step": nbytes,
+            "eager": {"step_ms": eager_ms / n_steps, "decode_tokens_per_s": B * n_steps / (eager_ms * 1e-3),
+                      "gbs": nbytes / (eager_ms / n_steps * 1e-3) / 1e9},
+            "graph_replay": {"steps_per_graph": per_graph, "step_ms": graph_ms / n_steps,
+                             "decode_tokens_per_s": B * n_steps / (graph_ms * 1e-3),
+                             "gbs": nbytes / (graph_ms / n_steps * 1e-3) / 1e9,
+                             "frac_of_peak": nbytes / (graph_ms / n_steps * 1e-3) / 1e9 / peak}}
+        del wl, graph
+    except torch.cuda.OutOfMemoryError as e:
+        res["qwq32b_longgen"] = {"skipped": f"out of device memory: {e}"[:200]}
+    gc.collect(); torch.cuda.empty_cache()
+    return res
+
 
 
 def run_e2e(wl, passes):
@@ -672,6 +888,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the MHA 4K, long-generation and 128K workloads that are reported in `detail`")
     ap.add_argument("--profile-case", type=int, default=0, metavar="DECODE_STEPS",
                     help="run the 4-layer small case with this many decode steps per pass (for ncu) and exit")
     ap.add_argument("--profile-case-fp8", type=int, default=0, metavar="DECODE_STEPS",

@@ -314,6 +314,12 @@ lt_status lt_kv_append(const lt_shape* shape, const uint8_t* layer_mask /* dev *
  * Split-KV: partial (max, sum, weighted values) per KV chunk go to the
  * workspace; the last chunk of each (layer, b, kv head) to finish merges them
  * in chunk order inside the same launch.  batch <= 2048.
+ * A call over part of the stack (layer_count < n_layers: a model that calls
+ * layer by layer, as the cache-updating attention call of Appendix A is used)
+ * is launched with CUDA's programmatic-serialization attribute: its CTAs may
+ * become resident while the previous kernel of the stream finishes and wait
+ * there until that kernel has completed, so back-to-back per-layer calls do not
+ * pay a launch gap each.  Results and ordering are those of plain stream order.
  */
 lt_status lt_hybrid_decode_attn(const lt_shape* shape, const void* q /* dev */,
                                 const void* const* k_full, const void* const* v_full,

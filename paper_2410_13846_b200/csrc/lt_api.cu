@@ -97,7 +97,8 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
   // Workspace query: room for a call over any layer range with any prompt length up to n_ctx and any
   // tail length up to w_last, through either kernel.  The persistent tensor-core kernel cuts a unit into at
   // most (CTAs / units) + 2 pieces, never more than it has tiles.
-  const bool umma = !window_only && scores_umma_supported(s, w_last);
+  // The tensor-core kernel writes two slots per piece or split (one per half of a tile's keys).
+  const bool umma = scores_umma_supported(s, w_last);
   const int64_t tiles = (n_ctx + kScoreBlockN - 1) / kScoreBlockN;
   size_t most_slots = 0;  // max over c of c * slots(c)
   p.n_splits = 1;
@@ -106,9 +107,12 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
     int len = 0;
     int64_t slots = host_score_splits(s, n_ctx, w_last, window_only, c, &len) + 1;  // + 1: rounding of shorter prompts
     if (umma) {
-      int64_t pieces = kScoreMaxCtas / ((int64_t)c * s.batch * s.n_kv_heads) + 2;
-      if (pieces > tiles) pieces = tiles;
-      if (pieces > slots) slots = pieces;
+      slots *= 2;
+      if (!window_only) {
+        int64_t pieces = kScoreMaxCtas / ((int64_t)c * s.batch * s.n_kv_heads) + 2;
+        if (pieces > tiles) pieces = tiles;
+        if (2 * pieces > slots) slots = 2 * pieces;
+      }
     }
     if ((size_t)(c * slots) > most_slots) most_slots = (size_t)(c * slots);
     if (slots > p.n_splits) p.n_splits = (int)slots;
@@ -259,7 +263,7 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
     a.streamk = window_only ? 0 : 1;
     a.tiles_per_unit = (n_ctx + kScoreBlockN - 1) / kScoreBlockN;
     a.total_tiles = (long long)a.n_units * a.tiles_per_unit;
-    const long long work = a.streamk ? a.total_tiles : (long long)a.n_units * sp.n_splits;
+    const long long work = a.streamk ? a.total_tiles : (long long)a.n_units * sp.n_splits;  // tiles, or host splits
     int grid = sm_count_of_current_device();
     if (grid > kScoreMaxCtas) grid = kScoreMaxCtas;
     if (grid > work) grid = (int)work;
@@ -269,8 +273,9 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
       long long pieces = ((long long)(a.tiles_per_unit - 1) * a.grid) / a.total_tiles + 2;
       if (pieces > a.tiles_per_unit) pieces = a.tiles_per_unit;
       sp.n_splits = (int)pieces;
-      sp.stat_floats = (size_t)layer_count * shape->batch * shape->n_q_heads * w_last * sp.n_splits * 3;
     }
+    sp.n_splits *= 2;  // two statistics slots per piece or split: one per half of a tile's keys
+    sp.stat_floats = (size_t)layer_count * shape->batch * shape->n_q_heads * w_last * sp.n_splits * 3;
   }
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   const size_t prefix = ws_prefix_bytes(*shape);
@@ -461,6 +466,9 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.items_cap = dp.items_cap;
   a.fused = fused;
   a.advance = advance;
+  // A call over part of the stack is one of several launches of a step (a model calls layer by layer):
+  // let each of them become resident under the tail of the one before.
+  a.pdl = layer_count < shape->n_layers ? 1 : 0;
   a.layer_begin = layer_begin;
   a.layer_count = layer_count;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
@@ -485,6 +493,7 @@ lt_status lt::decode_launch(const DecodeCall& c, void* stream) {
     a.layer_begin = layer_begin + done;
     a.layer_count = layer_count - done < layers_per_launch ? layer_count - done : layers_per_launch;
     a.advance = (c.a.advance && done + a.layer_count == layer_count) ? 1 : 0;
+    if (layer_count > layers_per_launch) a.pdl = 1;  // a stack that is split here is several launches too
     cudaError_t e = mma ? launch_decode_mma(a, c.kf, c.vf, c.ks, c.vs, cs) : launch_decode_generic(a, c.kf, c.vf, c.ks, c.vs, cs);
     if (e != cudaSuccess) return LT_ERR_CUDA;
   }

@@ -23,6 +23,17 @@
 
 namespace lt {
 
+// Programmatic dependent launch, for callers that issue a step as several launches (one per layer):
+// a launch made with the programmatic-serialization attribute may become resident while the previous
+// kernel of the stream is still running its last items.  Its CTAs then sit in pdl_wait_prior_grid()
+// until that kernel has completed and its writes are visible, so the launch latency and the CTA
+// ramp-up are paid under the previous kernel's tail.  Everything a launch shares with its predecessor -
+// seq_lens (advanced by a step's last launch), the launch counters and the partial slots of the
+// workspace - is touched only after the wait, which is the first statement of the kernels.  Without the
+// attribute both calls are no-ops.
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_allow_next_grid() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 struct WorkItem {
   int l, b, h, c;  // layer, batch row, kv head, chunk
   int nc;          // chunks of this (layer, batch row)

@@ -34,6 +34,8 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a, Layer
   __shared__ float2 s_ml[kCombineStagePairs];
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads;
+  pdl_wait_prior_grid();
+  pdl_allow_next_grid();
   WorkList wl;
   wl.carve(smem, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
@@ -115,8 +117,7 @@ static cudaError_t launch_generic_variant(const DecodeArgs& a, const LayerTable&
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 128, smem);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  kern<<<persistent_grid(a, per_sm), 128, smem, st>>>(a, kf, vf, ks, vs);
-  return cudaGetLastError();
+  return launch_decode_kernel(kern, persistent_grid(a, per_sm), 128, smem, st, a, kf, vf, ks, vs);
 }
 
 cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,

@@ -175,6 +175,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   float* sm_buf = reinterpret_cast<float*>(smem + RING_BYTES);  // [2][8][128]
   float* sm_m = sm_buf + 2 * 8 * kD;                            // [WARPS][8]
   float* sm_l = sm_m + WARPS * 8;                               // [WARPS][8]
+  pdl_wait_prior_grid();   // the previous launch of the stream is complete: lengths, counters and partial slots are ours
+  pdl_allow_next_grid();   // the next launch may take SMs as this one's CTAs retire (it waits the same way)
   WorkList wl;
   wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
@@ -698,8 +700,7 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
     }
   }
   const int grid = persistent_grid(a, per_sm);
-  kern<<<grid, WARPS * 32, smem, st>>>(a, kf, vf, ks, vs);
-  return cudaGetLastError();
+  return launch_decode_kernel(kern, grid, WARPS * 32, smem, st, a, kf, vf, ks, vs);
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,

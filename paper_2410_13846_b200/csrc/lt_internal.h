@@ -48,7 +48,7 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
 
 // Geometry of the tensor-core scoring kernel.
 constexpr int kScoreBlockM = 256;   // query rows per unit
-constexpr int kScoreBlockN = 128;   // keys per tile
+constexpr int kScoreBlockN = 256;   // keys per tile
 constexpr int kScoreMaxCtas = 192;  // the persistent launch never has more CTAs than this (one per SM)
 // The persistent launch cuts the sequence of all tiles, [0, total), into `grid` contiguous ranges:
 // tile g belongs to CTA g * grid / total.
@@ -107,6 +107,7 @@ struct DecodeArgs {
   int layer_begin, layer_count;
   int min_chunk, max_chunk, target_items, items_cap;
   int fused, advance;
+  int pdl;   // launch with the programmatic-serialization attribute (the step comes as several launches)
   float cs;  // softmax scale * log2(e)
   float* part_ml;
   float* part_o;
@@ -123,6 +124,23 @@ constexpr int kMaxWorkEntries = 2048;
 int persistent_grid(const DecodeArgs& a, int ctas_per_sm);
 // SM count of the current device (looked up once per device, behind a lock).
 int sm_count_of_current_device();
+// Launch of a decode kernel, with the programmatic-serialization attribute when a.pdl is set.
+template <typename Kern>
+inline cudaError_t launch_decode_kernel(Kern kern, int grid, int threads, int smem, cudaStream_t st, const DecodeArgs& a,
+                                        const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
+                                        const LayerTable& vs) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, a, kf, vf, ks, vs);
+}
 cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 // bf16, head_dim 128, group size <= 8: tensor-core path.
@@ -153,7 +171,9 @@ struct ScoreArgs {
   int window_only;
   int n_splits, split_len;
   // tensor-core path only: the persistent launch
-  int streamk;             // 1: CTAs own contiguous tile ranges and n_splits counts the pieces of a unit; 0: host splits
+  int streamk;             // 1: CTAs own contiguous tile ranges and n_splits = 2 x the pieces of a unit; 0: n_splits = 2 x
+                           // the host splits (a row's statistics of a piece or split come in two slots, one per half
+                           // of a tile's keys)
   int grid;                // CTAs
   int row_blocks;          // blocks of kScoreBlockM query rows per (layer, b, kv head)
   int n_units;             // layer_count * B * Hkv * row_blocks

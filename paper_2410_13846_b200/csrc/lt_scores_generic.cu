@@ -115,8 +115,8 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
       const int r = (hq % G) * T + t;          // row among the kv head's G * T query rows
       const long long unit = (lb * s.n_kv_heads + hq / G) * a.row_blocks + r / kScoreBlockM;
       const long long g0 = unit * a.tiles_per_unit;
-      n_slots = score_tile_owner(a.total_tiles, a.grid, g0 + a.tiles_per_unit - 1) -
-                score_tile_owner(a.total_tiles, a.grid, g0) + 1;
+      n_slots = 2 * (score_tile_owner(a.total_tiles, a.grid, g0 + a.tiles_per_unit - 1) -
+                     score_tile_owner(a.total_tiles, a.grid, g0) + 1);  // two slots per piece (halves of a tile's keys)
     }
     float Mx = -INFINITY;
     for (int sp = 0; sp < n_slots; ++sp) Mx = fmaxf(Mx, st[sp * 3]);

@@ -2,44 +2,49 @@
 //
 // S = Q K^T is a real dense contraction here (G * w_last query rows against
 // every prompt key), so it runs on the 5th-generation tensor cores:
-// tcgen05.mma (M = 128, N = 128, K = 16 per instruction, bf16 in, fp32 out)
-// issued by one thread.  The stationary operand, the block of up to 256 query
-// rows, lives in tensor memory (TMEM) as the A operand; only the streamed K
-// tiles come from shared memory (128-byte-swizzled K-major layout, written by
-// TMA), which halves the shared-memory traffic of an instruction compared with
-// both operands in shared memory.  Accumulators are three 128 x 128 fp32 slots
-// in TMEM that rotate between the MMA issuer and the statistics warps.
+// tcgen05.mma (M = 128, N = 256, K = 16 per instruction, bf16 in, fp32 out)
+// issued by one thread, operands in shared memory in the 128-byte-swizzled
+// K-major layout, accumulators in tensor memory (TMEM).  N = 256 on purpose: the
+// issuing thread pays a fixed cost per instruction group (barrier wait, commit)
+// during which it issues nothing, and only instructions of 128 clocks each keep
+// the tensor pipe fed across those gaps (measured: groups of eight N = 128
+// instructions run at 92 clocks per instruction instead of 64, N = 256 at 128).
 //
 // The launch is persistent: one CTA per SM.  With the whole prompt scored
-// (lt_lazy_scores) the 128-key tiles of all (layer, batch row, kv head, block of
+// (lt_lazy_scores) the 256-key tiles of all (layer, batch row, kv head, block of
 // 256 query rows) units form one sequence that is cut into equal contiguous
 // ranges, one per CTA, so every SM gets the same number of tiles whatever the
-// unit count; a unit that straddles a cut gets one statistics slot per piece.
+// unit count; a unit that straddles a cut gets its own statistics slots per piece.
 // With the denominator given (lt_lazy_scores_lse) the work items are the host's
 // key splits of the kept ranges, dealt round-robin.
 //
-// Roles (three warpgroups):
-//   warp 0      producer: one lane streams K tiles into a ring with TMA
-//               (cp.async.bulk.tensor, two 64-column boxes per tile), completion
-//               counted in bytes on full[s]; the ring never drains between pieces;
+// Roles (18 warps):
+//   warp 0      producer: one lane streams the unit's query block (64 KB, at a change
+//               of unit) and the 256-key K tiles (64 KB each, two stages) into shared
+//               memory with TMA (cp.async.bulk.tensor, 64-column x 128/256-row boxes),
+//               completion counted in bytes;
 //   warp 1      allocates TMEM; lane 0 issues the MMAs of a tile (8 k-steps per row
-//               block) into the next accumulator slot and commits to slot_full and,
-//               after the tile's last row block, to empty[s];
-//   warps 2-3   fill up the first warpgroup (register hand-over is per warpgroup);
-//   warps 4-11  statistics: thread = one query row (one TMEM lane).  At a change of
-//               unit the thread writes its query row into TMEM (tcgen05.st).  It reads
-//               its row of every 128 x 128 score block with tcgen05.ld and keeps only a
-//               reference exponent, sum exp and windowed sum exp - no shuffles, no
-//               shared memory, nothing written until the end of the piece.
+//               block of 128 query rows) into that row block's accumulator (256
+//               columns) and commits to its slot_full and, after the tile's last row
+//               block, to empty[s];
+//   warps 2-17  statistics, four per scheduler: thread = one query row (one TMEM lane)
+//               x one half of the tile's 256 keys.  It reads its 128 scores in chunks of
+//               32 registers with tcgen05.ld (the other warps of its scheduler run under
+//               the load) and keeps only a reference exponent, sum exp and windowed sum
+//               exp - no shuffles, no shared memory, nothing written until the end of the
+//               piece.  The accumulator goes back to the MMA warp as soon as the row's last
+//               chunk is in registers.
 //
 // Exponentials.  One ex2 per score on the special-function unit (16 per clock per
-// SM) would bound the kernel at twice the tensor-core time, so a fixed share of
-// the columns takes 2^x on the FMA pipe instead: the reference of a row is an
-// INTEGER M >= max (log2 domain), so x = t - M splits exactly into round(x) and
-// a remainder f in [-1/2, 1/2]; 2^f is a cubic (relative error 7.5e-5, far inside
-// the 1e-3 absolute tolerance of a ratio of sums) and round(x) goes into the
-// exponent field with one integer add.  The FMA-pipe work uses the packed
-// two-lane fp32 instructions (fma / add .f32x2).
+// SM) is the floor of this kernel (the unit is ~80 % busy with nothing but the
+// statistics running), so a fixed share of the columns takes 2^x on the FMA pipe
+// instead: the reference of a row is an INTEGER M >= max (log2 domain), so x = t - M
+// splits exactly into round(x) and a remainder f in [-1/2, 1/2]; 2^f is a cubic
+// (relative error 7.5e-5, far inside the 1e-3 absolute tolerance of a ratio of sums)
+// and round(x) goes into the exponent field with one integer add.  The FMA-pipe work
+// uses the packed two-lane fp32 instructions (fma / add .f32x2).  The share is small
+// (an eighth): measured, an ex2 costs the scheduler about five issue slots and the
+// polynomial about twelve, so a larger share only trades one bound for another.
 //
 // Every wait on an mbarrier is bounded in time; on expiry the kernel raises
 // LT_DEVERR_TIMEOUT in the workspace header, all roles leave their loops, TMEM
@@ -50,7 +55,7 @@
 #include "lt_internal.h"
 
 #ifndef LT_SCORES_POLY_OF8
-#define LT_SCORES_POLY_OF8 3  // of every 8 column pairs, this many take 2^x on the FMA pipe
+#define LT_SCORES_POLY_OF8 1  // of every 8 column pairs, this many take 2^x on the FMA pipe
 #endif
 
 namespace lt {
@@ -60,18 +65,18 @@ namespace {
 constexpr int kD = 128;  // head_dim
 constexpr int kRowBytes = 256;
 constexpr int kBlockM = kScoreBlockM;  // query rows per unit (2 UMMA row blocks)
-constexpr int kBlockN = kScoreBlockN;  // keys per tile
-constexpr int kStages = 6;
-constexpr int kKHalfBytes = kBlockN * 128;        // one d-half of a K tile
-constexpr int kStageBytes = 2 * kKHalfBytes;      // 32 KB
+constexpr int kBlockN = kScoreBlockN;  // keys per tile (one UMMA instruction wide)
+constexpr int kStages = 2;
+constexpr int kQHalfBytes = kBlockM * 128;        // one d-half of the query block: [256 rows][128 B]
+constexpr int kQBytes = 2 * kQHalfBytes;          // 64 KB
+constexpr int kKHalfBytes = kBlockN * 128;        // one d-half of a K tile: [256 rows][128 B]
+constexpr int kStageBytes = 2 * kKHalfBytes;      // 64 KB
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
-constexpr int kThreads = 384;
-constexpr int kRegsLight = 56;   // producer / MMA warpgroup after setmaxnreg.dec
-constexpr int kRegsStats = 224;  // statistics warpgroups after setmaxnreg.inc
-constexpr int kTmemCols = 512;
-constexpr int kSlots = 3;        // accumulator slots of 128 columns: TMEM columns [0, 384)
-constexpr int kQCol = 384;       // query rows (A operand): 64 columns per row block, [384, 512)
+constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+constexpr int kStatWarps = 16;
+constexpr int kThreads = 64 + kStatWarps * 32;    // 576 (registers are granted as for 640: 96 per thread)
+constexpr int kTmemCols = 512;   // two accumulators of 256 columns, one per row block
+constexpr int kChunk = 32;       // columns per tcgen05.ld
 constexpr int kPolyOf8 = LT_SCORES_POLY_OF8;
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 1.9 GHz
 
@@ -138,56 +143,35 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128.
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) | ((128u >> 4) << 24);
 
-// D[tmem] (+)= A[tmem] . B[smem]^T: A is 128 lanes x 8 columns (16 bf16 of one query row per lane, two per
-// 32-bit column, the lower d in the lower half), B a 128-key x 16-d slice of the K tile.
-__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem] . B[smem]^T: A a 128-row x 16-d slice of the query block, B a 256-key x 16-d slice of the K tile.
+__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// 32 consecutive columns of this thread's TMEM lane into v[OFF .. OFF+31] (asynchronous until tmem_ld_wait)
-template <int OFF, int N>
-__device__ __forceinline__ void tmem_ld32_at(uint32_t taddr, uint32_t (&v)[N]) {
+// 32 consecutive columns of this thread's TMEM lane into v[0 .. 31] (asynchronous until tmem_ld_wait)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-      : "=r"(v[OFF + 0]), "=r"(v[OFF + 1]), "=r"(v[OFF + 2]), "=r"(v[OFF + 3]), "=r"(v[OFF + 4]), "=r"(v[OFF + 5]),
-        "=r"(v[OFF + 6]), "=r"(v[OFF + 7]), "=r"(v[OFF + 8]), "=r"(v[OFF + 9]), "=r"(v[OFF + 10]), "=r"(v[OFF + 11]),
-        "=r"(v[OFF + 12]), "=r"(v[OFF + 13]), "=r"(v[OFF + 14]), "=r"(v[OFF + 15]), "=r"(v[OFF + 16]),
-        "=r"(v[OFF + 17]), "=r"(v[OFF + 18]), "=r"(v[OFF + 19]), "=r"(v[OFF + 20]), "=r"(v[OFF + 21]),
-        "=r"(v[OFF + 22]), "=r"(v[OFF + 23]), "=r"(v[OFF + 24]), "=r"(v[OFF + 25]), "=r"(v[OFF + 26]),
-        "=r"(v[OFF + 27]), "=r"(v[OFF + 28]), "=r"(v[OFF + 29]), "=r"(v[OFF + 30]), "=r"(v[OFF + 31])
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-// v[OFF .. OFF+31] into 32 consecutive columns of this thread's TMEM lane (asynchronous until tmem_st_wait)
-template <int OFF, int N>
-__device__ __forceinline__ void tmem_st32_at(uint32_t taddr, const uint32_t (&v)[N]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n" ::"r"(taddr),
-      "r"(v[OFF + 0]), "r"(v[OFF + 1]), "r"(v[OFF + 2]), "r"(v[OFF + 3]), "r"(v[OFF + 4]), "r"(v[OFF + 5]),
-      "r"(v[OFF + 6]), "r"(v[OFF + 7]), "r"(v[OFF + 8]), "r"(v[OFF + 9]), "r"(v[OFF + 10]), "r"(v[OFF + 11]),
-      "r"(v[OFF + 12]), "r"(v[OFF + 13]), "r"(v[OFF + 14]), "r"(v[OFF + 15]), "r"(v[OFF + 16]), "r"(v[OFF + 17]),
-      "r"(v[OFF + 18]), "r"(v[OFF + 19]), "r"(v[OFF + 20]), "r"(v[OFF + 21]), "r"(v[OFF + 22]), "r"(v[OFF + 23]),
-      "r"(v[OFF + 24]), "r"(v[OFF + 25]), "r"(v[OFF + 26]), "r"(v[OFF + 27]), "r"(v[OFF + 28]), "r"(v[OFF + 29]),
-      "r"(v[OFF + 30]), "r"(v[OFF + 31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
-
 // One MUFU instruction: 2^x, relative error 2^-22, results below 2^-126 flush to zero.
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -226,21 +210,21 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
   return d;
 }
 
-// max of 64 values: four interleaved chains of three-input maxima, then a small tree
-__device__ __forceinline__ float max64(const uint32_t (&v)[64]) {
+// max of 32 values: four interleaved chains of three-input maxima, then a small tree
+__device__ __forceinline__ float max32(const uint32_t (&v)[32]) {
   float m0 = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
   float m1 = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
   float m2 = max3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
   float m3 = max3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
 #pragma unroll
-  for (int i = 12; i < 60; i += 8) {
+  for (int i = 12; i < 28; i += 8) {
     m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
     m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
     m2 = max3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
     m3 = max3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
   }
-  m0 = max3(m0, __uint_as_float(v[60]), __uint_as_float(v[61]));
-  m1 = max3(m1, __uint_as_float(v[62]), __uint_as_float(v[63]));
+  m0 = max3(m0, __uint_as_float(v[28]), __uint_as_float(v[29]));
+  m1 = max3(m1, __uint_as_float(v[30]), __uint_as_float(v[31]));
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
@@ -251,15 +235,15 @@ constexpr float kP0 = 0.9999280571937561f, kP1 = 0.6932609677314758f, kP2 = 0.24
 constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round-to-nearest(x) in the low mantissa bits
 constexpr float kMinX = -125.0f;       // 2^x below this is treated as 2^-125 (keeps the exponent field positive)
 
-// sum_i 2^(v_i * cs - M) over the 64 values, M an integer (as a float): MUFU for most column pairs, the
+// sum_i 2^(v_i * cs - M) over the 32 values, M an integer (as a float): MUFU for most column pairs, the
 // FMA-pipe polynomial for kPolyOf8 of every 8 pairs.
-__device__ __forceinline__ float sum_ex2_64_mixed(const uint32_t (&v)[64], float cs, float M) {
+__device__ __forceinline__ float sum_ex2_32_mixed(const uint32_t (&v)[32], float cs, float M) {
   const f32x2 cs2 = pack2(cs, cs), nM2 = pack2(-M, -M);
   const f32x2 magic2 = pack2(kMagic, kMagic), mone2 = pack2(-1.f, -1.f);
   const f32x2 p3 = pack2(kP3, kP3), p2 = pack2(kP2, kP2), p1 = pack2(kP1, kP1), p0 = pack2(kP0, kP0);
   f32x2 acc0 = pack2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {  // pair i = columns 2i, 2i + 1
+  for (int i = 0; i < 16; ++i) {  // pair i = columns 2i, 2i + 1
     const f32x2 x2 = fma2(pack2u(v[2 * i], v[2 * i + 1]), cs2, nM2);
     float xl, xh;
     unpack2(x2, xl, xh);
@@ -293,10 +277,10 @@ __device__ __forceinline__ float sum_ex2_64_mixed(const uint32_t (&v)[64], float
   return a + b;
 }
 // The same sum with every exponential on the MUFU; -inf entries (masked columns) contribute 0.
-__device__ __forceinline__ float sum_ex2_64(const uint32_t (&v)[64], float cs, float off) {
+__device__ __forceinline__ float sum_ex2_32(const uint32_t (&v)[32], float cs, float off) {
   float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-  for (int i = 0; i < 64; i += 4) {
+  for (int i = 0; i < 32; i += 4) {
     s0 += ex2(fmaf(__uint_as_float(v[i]), cs, off));
     s1 += ex2(fmaf(__uint_as_float(v[i + 1]), cs, off));
     s2 += ex2(fmaf(__uint_as_float(v[i + 2]), cs, off));
@@ -308,17 +292,18 @@ __device__ __forceinline__ float sum_ex2_64(const uint32_t (&v)[64], float cs, f
 }  // namespace
 
 struct KeyMaps {
+  CUtensorMap q;                 // q_tail as a [L * B * Hq * w_last][128] bf16 matrix, box 64 x 256
   CUtensorMap m[LT_MAX_LAYERS];  // layer l's K cache as a [B * Hkv * capacity][128] bf16 matrix, box 64 x 128
 };
 
 // One contiguous run of tiles of one unit, handled by one CTA.
 struct Piece {
   int l, b, h, rb;  // the unit: layer, batch row, kv head, block of 256 query rows
-  int unit;         // its index (changes <=> the query rows in TMEM must be replaced)
+  int unit;         // its index (changes <=> the query block in shared memory must be replaced)
   int k0, k1;       // keys of the piece: statistics cover [k0, k1)
   int ts0;          // first key of the piece's first tile
   int n_tiles;
-  int slot;         // statistics slot of the piece within its rows
+  int slot;         // statistics slot pair of the piece within its rows (one slot per column half)
 };
 
 // The pieces of this CTA, in order.  `cursor` starts at 0 (every role walks the same list on its own).
@@ -341,15 +326,16 @@ __device__ __forceinline__ bool next_piece(const ScoreArgs& a, long long& cursor
     slot = (int)blockIdx.x - score_tile_owner(a.total_tiles, gridDim.x, (long long)unit * TU);
     cursor += n_tiles;
   } else {
-    const long long n_items = (long long)a.n_units * a.n_splits;
+    const int host_splits = a.n_splits / 2;
+    const long long n_items = (long long)a.n_units * host_splits;
     const long long item = (long long)blockIdx.x + cursor * gridDim.x;
     if (item >= n_items) return false;
-    unit = (int)(item / a.n_splits);
-    slot = (int)(item - (long long)unit * a.n_splits);
+    unit = (int)(item / host_splits);
+    slot = (int)(item - (long long)unit * host_splits);
     score_split_range(a, slot, &k0, &k1);
-    // Paged caches: tiles start on multiples of 128 keys so that none straddles two pages (the page size
-    // is a multiple of 128); the keys before k0 in the first tile are masked by the statistics warps.
-    ts0 = s.page_size > 0 ? (k0 & ~(kBlockN - 1)) : k0;
+    // Paged caches: tiles start on multiples of 128 keys so that no 128-key box straddles two pages (the page
+    // size is a multiple of 128); the keys before k0 in the first tile are masked by the statistics warps.
+    ts0 = s.page_size > 0 ? (k0 & ~127) : k0;
     n_tiles = k1 > k0 ? (k1 - ts0 + kBlockN - 1) / kBlockN : 0;
     cursor += 1;
   }
@@ -373,17 +359,19 @@ __global__ void __launch_bounds__(kThreads, 1)
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern of the MMA is a function of address bits 4..9
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const uint32_t sK = smem_u32(smem);
-  uint8_t* bar_mem = smem + kStages * kStageBytes;
+  const uint32_t sQ = smem_u32(smem);
+  const uint32_t sK = sQ + kQBytes;
+  uint8_t* bar_mem = smem + kQBytes + kStages * kStageBytes;
   const uint32_t bar0 = smem_u32(bar_mem);
-  const uint32_t bar_full = bar0;                          // [kStages]   K tile landed
-  const uint32_t bar_empty = bar0 + 8 * kStages;           // [kStages]   K tile consumed by the MMAs
-  const uint32_t bar_sfull = bar0 + 16 * kStages;          // [kSlots]    accumulator slot holds a score block
-  const uint32_t bar_sempty = bar_sfull + 8 * kSlots;      // [kSlots]    score block is in registers
-  const uint32_t bar_qready = bar_sempty + 8 * kSlots;     // [2]         query rows of a row block are in TMEM
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 16 * kStages + 16 * kSlots + 16);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * kStages + 16 * kSlots + 24);
-  static_assert(16 * kStages + 16 * kSlots + 32 <= kBarBytes, "barrier area too small");
+  const uint32_t bar_full = bar0;                      // [kStages]  K tile landed
+  const uint32_t bar_empty = bar0 + 8 * kStages;       // [kStages]  K tile consumed by the MMAs
+  const uint32_t bar_sfull = bar0 + 16 * kStages;      // [2]        row block's accumulator holds a score block
+  const uint32_t bar_sempty = bar_sfull + 16;          // [2]        score block is in registers
+  const uint32_t bar_qfull = bar_sempty + 16;          //            query block landed
+  const uint32_t bar_qfree = bar_qfull + 8;            //            every MMA that reads the query block has completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 16 * kStages + 56);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * kStages + 64);
+  static_assert(16 * kStages + 72 <= kBarBytes, "barrier area too small");
 
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads;
@@ -398,12 +386,12 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_full + 8 * i, 1);
       mbar_init(bar_empty + 8 * i, 1);
     }
-    for (int i = 0; i < kSlots; ++i) {
+    for (int i = 0; i < 2; ++i) {
       mbar_init(bar_sfull + 8 * i, 1);
-      mbar_init(bar_sempty + 8 * i, 128);
+      mbar_init(bar_sempty + 8 * i, kStatWarps * 32 / 2);  // every statistics thread of the row block
     }
-    mbar_init(bar_qready, 128);
-    mbar_init(bar_qready + 8, 128);
+    mbar_init(bar_qfull, 1);
+    mbar_init(bar_qfree, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -422,18 +410,32 @@ __global__ void __launch_bounds__(kThreads, 1)
   auto rows_of = [&](int rb) { return min(kBlockM, M - rb * kBlockM); };
   auto mbs_of = [&](int rb) { return (rows_of(rb) + 127) / 128; };
 
-  if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsLight));
+  if (warp < 2) {
     if (warp == 0) {
       // ===== producer =====
       // Rows past the piece's last key are real cache rows (or zero past the end of the
-      // cache): the statistics warps never look at those columns.
+      // cache): the statistics warps never look at those columns.  Query rows past the unit's last
+      // row are the next head's rows (or zero past the end of q_tail): their scores are never read.
       if (lane == 0) {
         bool ok = true;
         long long cursor = 0;
-        int kt = 0;  // tiles issued by this CTA so far: stage kt % kStages, use kt / kStages of that stage
+        int kt = 0;        // tiles issued by this CTA so far: stage kt % kStages, use kt / kStages of that stage
+        int q_loads = 0;   // query blocks loaded so far
+        int prev_unit = -1;
         Piece p;
         while (ok && next_piece(a, cursor, p)) {
+          if (p.n_tiles == 0) continue;
+          if (p.unit != prev_unit) {
+            // the MMAs of the previous unit must be done with the query block before it is replaced
+            if (q_loads > 0) ok = mbar_wait(bar_qfree, (q_loads - 1) & 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(bar_qfull, kQBytes);
+            const int yq = ((p.l * s.batch + p.b) * s.n_q_heads + p.h * G) * T + p.rb * kBlockM;
+            tma_load_2d(sQ, &maps.q, 0, yq, bar_qfull);
+            tma_load_2d(sQ + kQHalfBytes, &maps.q, 64, yq, bar_qfull);
+            ++q_loads;
+            prev_unit = p.unit;
+          }
           const CUtensorMap* map = &maps.m[p.l];
           for (int it = 0; it < p.n_tiles; ++it, ++kt) {
             const int st = kt % kStages;
@@ -442,22 +444,28 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t dst = sK + st * kStageBytes;
             const uint32_t bar = bar_full + 8 * st;
             mbar_expect_tx(bar, kStageBytes);
-            const int j = p.ts0 + it * kBlockN;
-            int y;
-            if (s.page_size <= 0) {
-              y = (p.b * s.n_kv_heads + p.h) * s.full_capacity + j;
-            } else {
-              const int page = s.block_table[(long long)p.b * s.pages_per_seq + j / s.page_size];
-              y = (page * s.n_kv_heads + p.h) * s.page_size + j % s.page_size;
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {  // two boxes of 128 keys (a box never straddles a page)
+              const int j = p.ts0 + it * kBlockN + rh * 128;
+              int y;
+              if (s.page_size <= 0) {
+                y = (p.b * s.n_kv_heads + p.h) * s.full_capacity + j;
+              } else {
+                // keys past the end of the cache take the last page: never read by the statistics
+                const int pg = min(j / s.page_size, s.pages_per_seq - 1);
+                const int page = s.block_table[(long long)p.b * s.pages_per_seq + pg];
+                y = (page * s.n_kv_heads + p.h) * s.page_size + j % s.page_size;
+              }
+              tma_load_2d(dst + rh * (128 * 128), map, 0, y, bar);
+              tma_load_2d(dst + kKHalfBytes + rh * (128 * 128), map, 64, y, bar);
             }
-            tma_load_2d(dst, map, 0, y, bar);
-            tma_load_2d(dst + kKHalfBytes, map, 64, y, bar);
           }
         }
         if (!ok) {
           // gave up: let the copies already issued land before the shared memory goes away
           for (int j = max(0, kt - kStages); j < kt; ++j)
             mbar_wait_quiet(bar_full + 8 * (j % kStages), (j / kStages) & 1);
+          if (q_loads > 0) mbar_wait_quiet(bar_qfull, (q_loads - 1) & 1);
         }
       }
       __syncwarp();
@@ -466,45 +474,41 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (lane == 0) {
         bool ok = true;
         long long cursor = 0;
-        int kt = 0;          // tiles consumed so far
-        int uc = 0;          // score blocks issued so far: slot uc % kSlots, use uc / kSlots of that slot
-        int q_uses0 = 0, q_uses1 = 0;
+        int kt = 0;            // tiles consumed so far
+        int uses0 = 0, uses1 = 0;  // score blocks issued so far into each row block's accumulator
+        int q_loads = 0;
         int prev_unit = -1;
         Piece p;
         while (ok && next_piece(a, cursor, p)) {
+          if (p.n_tiles == 0) continue;
           const int n_mb = mbs_of(p.rb);
-          if (p.unit != prev_unit && p.n_tiles > 0) {
-            // the statistics warps replace the query rows in TMEM (after the last MMAs that read the old ones)
-            ok = mbar_wait(bar_qready, q_uses0 & 1, abort_flag);
-            ++q_uses0;
-            if (ok && n_mb > 1) {
-              ok = mbar_wait(bar_qready + 8, q_uses1 & 1, abort_flag);
-              ++q_uses1;
-            }
+          if (p.unit != prev_unit) {
+            if (q_loads > 0) umma_commit(bar_qfree);  // arrives once every MMA issued so far has completed
+            ok = mbar_wait(bar_qfull, q_loads & 1, abort_flag);
             if (!ok) break;
-            tc_fence_after();
+            ++q_loads;
             prev_unit = p.unit;
           }
           for (int it = 0; it < p.n_tiles && ok; ++it, ++kt) {
             const int st = kt % kStages;
             ok = mbar_wait(bar_full + 8 * st, (kt / kStages) & 1, abort_flag);
             if (!ok) break;
-            tc_fence_after();
-            for (int mb = 0; mb < n_mb; ++mb, ++uc) {
-              const int slot = uc % kSlots, use = uc / kSlots;
-              if (use > 0) {
-                ok = mbar_wait(bar_sempty + 8 * slot, (use - 1) & 1, abort_flag);
+            for (int mb = 0; mb < n_mb; ++mb) {
+              int& uses = mb ? uses1 : uses0;
+              if (uses > 0) {
+                ok = mbar_wait(bar_sempty + 8 * mb, (uses - 1) & 1, abort_flag);
                 if (!ok) break;
-                tc_fence_after();
               }
-              const uint32_t d_tmem = tmem_base + slot * 128;
-              const uint32_t a_tmem = tmem_base + kQCol + mb * 64;
+              ++uses;
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + mb * 256;
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + mb * (128 * 128) + (ks & 3) * 32;
                 const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
-                umma_bf16_ts(d_tmem, a_tmem + ks * 8, umma_desc(b_addr), ks > 0 ? 1u : 0u);
+                umma_bf16_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
               }
-              umma_commit(bar_sfull + 8 * slot);
+              umma_commit(bar_sfull + 8 * mb);
             }
             if (!ok) break;
             umma_commit(bar_empty + 8 * st);
@@ -515,23 +519,20 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   } else {
     // ===== statistics =====
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsStats));
-    // A score block's 128 columns are taken in two halves of 64 registers.  The load of
-    // one half is in flight while the exponentials of the other half run, and
-    // the accumulator slot is handed back to the MMA warp as soon as both
-    // halves sit in registers.
-    const int mb = (warp - 4) >> 2;  // row block of this warp
+    // Four consecutive warps cover the four TMEM lane quadrants (a warp may access lanes 32 * (warp % 4) ...).
+    const int sw = warp - 2;
     const int quad = warp & 3;       // TMEM lane quadrant this warp may access
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const int mb = (sw >> 2) & 1;    // row block of this warp
+    const int ch = sw >> 3;          // half of the tile's 256 keys that this warp reads
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + mb * 256 + ch * 128;
     const float cs = a.cs;
     const int S = s.n_sink;
 
     bool ok = true;
     long long cursor = 0;
-    int uc = 0;  // score blocks issued by the MMA warp before the current piece
-    int prev_unit = -1;
+    int uses = 0;  // score blocks of this row block consumed so far
     Piece p;
-    uint32_t va[64], vb[64];
+    uint32_t va[kChunk];
     while (ok && next_piece(a, cursor, p)) {
       const int rows_here = rows_of(p.rb);
       const int n_mb = (rows_here + 127) / 128;
@@ -542,38 +543,15 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int g = r / T, tq = r - g * T;
       const long long rowid =
           (((long long)(p.l - a.layer_begin) * s.batch + p.b) * s.n_q_heads + p.h * G + g) * T + tq;
-      float* stp = a.stats + (rowid * a.n_splits + p.slot) * 3;
+      float* stp = a.stats + (rowid * a.n_splits + 2 * p.slot + ch) * 3;
       if (!active || p.n_tiles == 0) {
-        // nothing to read: an idle row block, or an empty key range (its slot still gets neutral statistics)
+        // nothing to read: an idle row block, or an empty key range (its slots still get neutral statistics)
         if (active && row_valid) {
           stp[0] = -INFINITY;
           stp[1] = 0.f;
           stp[2] = 0.f;
         }
-        uc += p.n_tiles * n_mb;
         continue;
-      }
-      if (p.unit != prev_unit) {
-        // this thread's query row -> TMEM (the A operand of its row block).  Every MMA that read the old
-        // rows of this block has completed: its score block was consumed by this warpgroup.
-        const uint4* qrow = reinterpret_cast<const uint4*>(
-            (const uint8_t*)a.q_tail +
-            ((((long long)p.l * s.batch + p.b) * s.n_q_heads + (long long)p.h * G) * T + (row_valid ? r : 0)) *
-                kRowBytes);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint4 x = row_valid ? __ldg(qrow + i) : make_uint4(0u, 0u, 0u, 0u);
-          va[4 * i] = x.x;
-          va[4 * i + 1] = x.y;
-          va[4 * i + 2] = x.z;
-          va[4 * i + 3] = x.w;
-        }
-        tmem_st32_at<0>(lane_addr + kQCol + mb * 64, va);
-        tmem_st32_at<32>(lane_addr + kQCol + mb * 64 + 32, va);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(bar_qready + 8 * mb);
-        prev_unit = p.unit;
       }
       const int k0 = p.k0, k1 = p.k1;
       const int vis = n_ctx - T + tq;  // last visible key of this row
@@ -581,73 +559,58 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int lim = min(vis, k1 - 1);     // last key of this piece that the row may see
       float Mr = -INFINITY, sA = 0.f, sWn = 0.f;  // reference exponent (an integer), sum, windowed sum
 
-      // statistics of one half (64 keys from jb) already in registers
-      auto half_stats = [&](uint32_t (&v)[64], int jb) {
-        const int jend = jb + 64;
+      // statistics of one chunk (32 keys from jb) already in registers
+      auto chunk_stats = [&](uint32_t (&v)[kChunk], int jb) {
+        const int jend = jb + kChunk;
         const bool all_win = (jend <= S) || (jb >= win_lo);
         const bool no_win = (jb >= S) && (jend <= win_lo);
         if ((jb >= k0) && (jend - 1 <= lim) && (all_win || no_win)) {
-          const float Mn = fmaxf(Mr, ceilf(max64(v) * cs));
+          const float Mn = fmaxf(Mr, ceilf(max32(v) * cs));
           const float corr = ex2(Mr - Mn);
-          const float ps = sum_ex2_64_mixed(v, cs, Mn);
+          const float ps = sum_ex2_32_mixed(v, cs, Mn);
           sA = fmaf(sA, corr, ps);
           sWn = fmaf(sWn, corr, all_win ? ps : 0.f);
           Mr = Mn;
         } else if (max(jb, k0) <= min(jend - 1, lim)) {
-          // boundary half (piece start, causal tail, piece end or window edge): mask in place.
+          // boundary chunk (piece start, causal tail, piece end or window edge): mask in place.
           // 2^(-inf) = 0, and at least one key is visible, so the maximum is finite.
 #pragma unroll
-          for (int i = 0; i < 64; ++i)
+          for (int i = 0; i < kChunk; ++i)
             if (jb + i > lim || jb + i < k0) v[i] = 0xff800000u;
-          const float Mn = fmaxf(Mr, ceilf(max64(v) * cs));
+          const float Mn = fmaxf(Mr, ceilf(max32(v) * cs));
           const float corr = ex2(Mr - Mn);
-          const float ps = sum_ex2_64(v, cs, -Mn);
+          const float ps = sum_ex2_32(v, cs, -Mn);
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
+          for (int i = 0; i < kChunk; ++i) {
             const int j = jb + i;
             if (!(j < S || j >= win_lo)) v[i] = 0xff800000u;
           }
-          const float pw = sum_ex2_64(v, cs, -Mn);
+          const float pw = sum_ex2_32(v, cs, -Mn);
           sA = fmaf(sA, corr, ps);
           sWn = fmaf(sWn, corr, pw);
           Mr = Mn;
         }
       };
 
-      // score block `it` of this row block is block uc + it * n_mb + mb of the CTA
-      {
-        const int u = uc + mb;
-        const int sl = u % kSlots;
-        ok = mbar_wait(bar_sfull + 8 * sl, (u / kSlots) & 1, abort_flag);
+      for (int it = 0; it < p.n_tiles; ++it, ++uses) {
+        const int kb = p.ts0 + it * kBlockN + ch * 128;  // first key of this thread's 128 columns
+        ok = mbar_wait(bar_sfull + 8 * mb, uses & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        tmem_ld32_at<0>(lane_addr + sl * 128, va);
-        tmem_ld32_at<32>(lane_addr + sl * 128 + 32, va);
-      }
-      for (int it = 0; it < p.n_tiles; ++it) {
-        const int u = uc + it * n_mb + mb;
-        const int sl = u % kSlots;
-        const int kb = p.ts0 + it * kBlockN;
-        const uint32_t taddr = lane_addr + sl * 128;
-        // first half is (being) loaded; start the second half, then work on the first
-        tmem_ld_wait();
-        tmem_ld32_at<0>(taddr + 64, vb);
-        tmem_ld32_at<32>(taddr + 96, vb);
-        half_stats(va, kb);
-        tmem_ld_wait();
-        // both halves are in registers: the accumulator slot may be overwritten
-        tc_fence_before();
-        mbar_arrive(bar_sempty + 8 * sl);
-        if (it + 1 < p.n_tiles) {
-          const int un = u + n_mb;
-          const int sn = un % kSlots;
-          ok = mbar_wait(bar_sfull + 8 * sn, (un / kSlots) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          tmem_ld32_at<0>(lane_addr + sn * 128, va);
-          tmem_ld32_at<32>(lane_addr + sn * 128 + 32, va);
+        // Four chunks of 32 columns through one register buffer: the load of a chunk is not overlapped
+        // by this warp's own arithmetic but by the three other statistics warps of its scheduler (two
+        // buffers would not fit the 96 registers a thread gets).
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(lane_addr + c * kChunk, va);
+          tmem_ld_wait();
+          if (c == 3) {
+            // the row's last chunk is in registers: the accumulator may be overwritten
+            tc_fence_before();
+            mbar_arrive(bar_sempty + 8 * mb);
+          }
+          chunk_stats(va, kb + c * kChunk);
         }
-        half_stats(vb, kb + 64);
       }
       if (!ok) break;
       if (row_valid) {
@@ -655,9 +618,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         stp[1] = sA;
         stp[2] = sWn;
       }
-      uc += p.n_tiles * n_mb;
     }
-    tmem_ld_wait();
   }
 
   // ---- teardown ------------------------------------------------------------------
@@ -695,7 +656,7 @@ EncodeTiledFn encode_tiled_fn() {
 }
 }  // namespace
 
-// grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 384.
+// grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 640.
 cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return cudaErrorNotSupported;
@@ -703,9 +664,19 @@ cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStr
                                                   : (cuuint64_t)a.s.batch * a.s.n_kv_heads * a.s.full_capacity;
   const cuuint64_t gdim[2] = {(cuuint64_t)kD, rows_total};
   const cuuint64_t gstride[1] = {(cuuint64_t)kRowBytes};
-  const cuuint32_t box[2] = {64u, (cuuint32_t)kBlockN};
+  const cuuint32_t box[2] = {64u, 128u};
   const cuuint32_t estride[2] = {1u, 1u};
   KeyMaps local;
+  {
+    // the tail queries of the whole stack as one matrix of 128-element rows; a box is one d-half of a unit's 256 rows
+    const cuuint64_t qdim[2] = {(cuuint64_t)kD,
+                                (cuuint64_t)a.s.n_layers * a.s.batch * a.s.n_q_heads * (cuuint64_t)a.w_last};
+    const cuuint32_t qbox[2] = {64u, (cuuint32_t)kBlockM};
+    const CUresult r = encode(&local.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.q_tail), qdim, gstride,
+                              qbox, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
   const int l_end = a.layer_begin + a.layer_count;
   for (int l = a.layer_begin; l < l_end; ++l) {
     const CUresult r = encode(&local.m[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kf.p[l]), gdim,

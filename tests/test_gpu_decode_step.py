@@ -121,6 +121,47 @@ def test_per_layer_calls_advance_once():
     assert torch.equal(out, ref)
 
 
+def test_per_layer_launch_chain_without_host_syncs_matches_whole_stack_steps():
+    """A model issues the step layer by layer.  Those launches carry the programmatic-serialization
+    attribute: each may become resident under the tail of the one before and waits there until it has
+    completed.  Twelve steps of six back-to-back per-layer launches, no host synchronisation anywhere in
+    the chain (so that launches do overlap), against whole-stack steps: same bits in every output, every
+    cache and seq_lens - including the step boundary, where the first launch of a step must see the
+    lengths that the last launch of the previous step advanced."""
+    L, B, Hq, Hkv, D, S, R = 6, 3, 8, 2, 128, 4, 60
+    lens, steps = [3000, 1500, 700], 12
+    cap = max(lens) + steps + 4
+    whole, chain = _two_stacks(L, B, Hq, Hkv, D, S, R, cap, torch.bfloat16, lens, [0, 1, 0, 0, 1, 0], seed=12)
+    torch.manual_seed(13)
+    qs = [torch.randn(L, B, Hq, D).bfloat16().cuda() for _ in range(steps)]
+    ks = [torch.randn(L, B, Hkv, D).bfloat16().cuda() for _ in range(steps)]
+    vs = [torch.randn(L, B, Hkv, D).bfloat16().cuda() for _ in range(steps)]
+    ref = [torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda") for _ in range(steps)]
+    got = [torch.full((L, B, Hq, D), float("nan"), dtype=torch.float32, device="cuda") for _ in range(steps)]
+    for t in range(steps):
+        lt.decode_step(whole.shape, qs[t], ks[t], vs[t], whole.tables, whole.mask, whole.seq_lens, ref[t], whole.ws)
+    torch.cuda.synchronize()
+    for t in range(steps):
+        for l in range(L):
+            lt.decode_step(chain.shape, qs[t], ks[t], vs[t], chain.tables, chain.mask, chain.seq_lens, got[t], chain.ws,
+                           layer_begin=l, layer_count=1, advance_seq_lens=(l == L - 1))
+    torch.cuda.synchronize()
+    for t in range(steps):
+        assert torch.equal(got[t], ref[t]), t
+    assert torch.equal(chain.seq_lens, whole.seq_lens) and chain.seq_lens.cpu().tolist() == [n + steps for n in lens]
+    for l in range(L):
+        assert torch.equal(chain.k_full[l], whole.k_full[l]) and torch.equal(chain.v_full[l], whole.v_full[l])
+        assert torch.equal(chain.k_stream[l], whole.k_stream[l]) and torch.equal(chain.v_stream[l], whole.v_stream[l])
+    assert lt.check(chain.ws) == 0
+    # the attention half alone, layer by layer (no append): same chain, same bits
+    out_whole = whole.attend(qs[0], torch.float32)
+    out_chain = torch.full_like(out_whole, float("nan"))
+    for l in range(L):
+        lt.hybrid_decode_attn(chain.shape, qs[0], chain.tables, chain.mask, chain.seq_lens, out_chain, chain.ws,
+                              layer_begin=l, layer_count=1)
+    assert torch.equal(out_chain, out_whole)
+
+
 def test_position_beyond_capacity_is_flagged_and_not_stored():
     st = Stack(2, 1, 4, 1, 128, 4, 12, 32)
     st.k_full[0].normal_(); st.v_full[0].normal_(); st.k_full[1].normal_(); st.v_full[1].normal_()
