@@ -74,6 +74,13 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], u
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// m16n8k32, E4M3 x E4M3 -> fp32: A holds 16 rows x 32 bytes, B 32 bytes x 8 columns
+__device__ __forceinline__ void mma_e4m3(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
@@ -106,6 +113,31 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
 __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
   const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two_bytes, __NV_E4M3);
   return (uint32_t)h.x | ((uint32_t)h.y << 16);
+}
+// two floats -> two E4M3 bytes (low byte first), round to nearest even, saturating
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
+  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+}
+// Four floats x[0..3] (already divided by the head's scale) as a sum of kQTerms E4M3 values each: term t of
+// element i goes to byte i of out[t].  Every residual x - (terms so far) is exact in fp32, so after three
+// terms what is left of an element is below 2^-12 of it (or below E4M3's smallest step, 2^-9).
+constexpr int kQTerms = 3;
+__device__ __forceinline__ void split_e4m3x4(const float (&x)[4], uint32_t (&out)[kQTerms]) {
+  float r[4] = {x[0], x[1], x[2], x[3]};
+#pragma unroll
+  for (int t = 0; t < kQTerms; ++t) {
+    const uint32_t lo = f32x2_to_e4m3x2(r[0], r[1]), hi = f32x2_to_e4m3x2(r[2], r[3]);
+    out[t] = lo | (hi << 16);
+    if (t + 1 < kQTerms) {
+      const uint32_t h01 = e4m3x2_to_f16x2(lo), h23 = e4m3x2_to_f16x2(hi);
+      const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+      const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+      r[0] -= f01.x;
+      r[1] -= f01.y;
+      r[2] -= f23.x;
+      r[3] -= f23.y;
+    }
+  }
 }
 template <uint32_t SEL>
 __device__ __forceinline__ uint32_t e4m3_pair_to_f16x2_div256(uint32_t w) {
@@ -348,31 +380,65 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     }
 
     // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
-    uint32_t qf[8][2];
+    uint32_t qf[FP8 ? 1 : 8][2];
+    // 8-bit caches: the stored K bytes are the A operand of E4M3 MMAs as they are, and q is their B operand as
+    // a sum of kQTerms E4M3 terms at one power-of-two scale per head (block blk covers d = 32 blk .. 32 blk + 31:
+    // bytes 4c .. 4c+3 in b0, 16 + 4c .. in b1).
+    uint32_t q8[FP8 ? kQTerms : 1][4][2];
+    float q_scale0 = 1.f, q_scale1 = 1.f;  // scale of heads 2c and 2c + 1 (this thread's S columns)
     {
       const __nv_bfloat16* qp =
           (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + gp) * kD;
+      if constexpr (FP8) {
+        float x[4][2][4];
+        float amax = 0.f;
 #pragma unroll
-      for (int ks8 = 0; ks8 < 8; ++ks8) {
-        if (gp < G) {
-          if constexpr (FP8) {
-            // k-block ks8 covers d = 16 ks8 .. 16 ks8 + 15 in the order of the byte fragments:
-            // slots (2c, 2c+1) <-> d + 4c, 4c+1 and slots (2c+8, 2c+9) <-> d + 4c+2, 4c+3.
-            // f16 operands: bf16 -> f16 is exact inside f16's range.
-            const uint2 q4 = *reinterpret_cast<const uint2*>(qp + 16 * ks8 + 4 * c);
-            qf[ks8][0] = pack_f16(bf16_lo(q4.x), bf16_hi(q4.x));
-            qf[ks8][1] = pack_f16(bf16_lo(q4.y), bf16_hi(q4.y));
-          } else {
+        for (int blk = 0; blk < 4; ++blk)
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            uint2 q4 = make_uint2(0u, 0u);
+            if (gp < G) q4 = *reinterpret_cast<const uint2*>(qp + 32 * blk + 16 * hf + 4 * c);
+            x[blk][hf][0] = bf16_lo(q4.x);
+            x[blk][hf][1] = bf16_hi(q4.x);
+            x[blk][hf][2] = bf16_lo(q4.y);
+            x[blk][hf][3] = bf16_hi(q4.y);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fabsf(x[blk][hf][e]));
+          }
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));  // the four lanes of a head hold its 128 values
+        // power-of-two scale that puts the head's largest |q| into [128, 256): inside E4M3's range (448)
+        const int e2 = (amax > 0.f && amax < INFINITY) ? ilogbf(amax) - 7 : 0;
+        const float inv = exp2f((float)-e2), scale = exp2f((float)e2);
+#pragma unroll
+        for (int blk = 0; blk < 4; ++blk)
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            float y[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) y[e] = x[blk][hf][e] * inv;
+            uint32_t terms[kQTerms];
+            split_e4m3x4(y, terms);
+#pragma unroll
+            for (int t = 0; t < kQTerms; ++t) q8[t][blk][hf] = terms[t];
+          }
+        q_scale0 = __shfl_sync(0xffffffffu, scale, (2 * c) * 4);
+        q_scale1 = __shfl_sync(0xffffffffu, scale, (2 * c + 1) * 4);
+      } else {
+#pragma unroll
+        for (int ks8 = 0; ks8 < 8; ++ks8) {
+          if (gp < G) {
             qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
             qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
+          } else {
+            qf[ks8][0] = 0u;
+            qf[ks8][1] = 0u;
           }
-        } else {
-          qf[ks8][0] = 0u;
-          qf[ks8][1] = 0u;
         }
       }
     }
 
+    const float cs0 = cs_l * q_scale0, cs1 = cs_l * q_scale1;  // per S column (head 2c, 2c + 1)
     float o[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
@@ -402,13 +468,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
             uint32_t m[4];
             const int chunk = 2 * blk + k_chk;
             ldmatrix_x4(m, st + row * kD + ((chunk ^ (row & 7)) << 4));
+            // the bytes are the A fragment as they are: rows g | g + 8, bytes 4c .. | 16 + 4c ..
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              // adjacent byte pairs: one conversion instruction each
-              const uint32_t af[4] = {e4m3x2_to_f16x2(m[2 * hf] & 0xffffu), e4m3x2_to_f16x2(m[2 * hf + 1] & 0xffffu),
-                                      e4m3x2_to_f16x2(m[2 * hf] >> 16), e4m3x2_to_f16x2(m[2 * hf + 1] >> 16)};
-              mma_f16(sc[mt], af, qf[2 * blk + hf][0], qf[2 * blk + hf][1]);
-            }
+            for (int t = 0; t < kQTerms; ++t) mma_e4m3(sc[mt], m, q8[t][blk][0], q8[t][blk][1]);
           }
         } else {
           // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
@@ -431,10 +493,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       for (int mt = 0; mt < MT; ++mt) {
         const int key_lo = key_base + mt * 16 + gp;
         const bool v_lo = key_lo < j1, v_hi = key_lo + 8 < j1;
-        sc[mt][0] = v_lo ? sc[mt][0] * cs_l : -INFINITY;
-        sc[mt][1] = v_lo ? sc[mt][1] * cs_l : -INFINITY;
-        sc[mt][2] = v_hi ? sc[mt][2] * cs_l : -INFINITY;
-        sc[mt][3] = v_hi ? sc[mt][3] * cs_l : -INFINITY;
+        sc[mt][0] = v_lo ? sc[mt][0] * cs0 : -INFINITY;
+        sc[mt][1] = v_lo ? sc[mt][1] * cs1 : -INFINITY;
+        sc[mt][2] = v_hi ? sc[mt][2] * cs0 : -INFINITY;
+        sc[mt][3] = v_hi ? sc[mt][3] * cs1 : -INFINITY;
         mx0 = fmaxf(mx0, fmaxf(sc[mt][0], sc[mt][2]));
         mx1 = fmaxf(mx1, fmaxf(sc[mt][1], sc[mt][3]));
       }

@@ -59,6 +59,31 @@ def test_scores_match_oracle(dtype, D, Hq, Hkv, S, R, n_ctx, T, scale):
     assert torch.equal(_run_scores(st, q_tail, n_ctx, T), torch.from_numpy(got).float().cuda())   # deterministic
 
 
+@pytest.mark.parametrize("dtype,D", [(torch.float32, 64), (torch.bfloat16, 128)])
+def test_scoring_a_layer_range_equals_the_whole_stack_call(dtype, D):
+    """Layer by layer, in ranges and all at once: the same bits, only the scored layers' slices are written, and
+    table entries outside the range may be missing (both kernels: CUDA-core and tensor-core path)."""
+    torch.manual_seed(8)
+    L, B, Hq, Hkv, S, R, n_ctx, T = 5, 2, 4, 2, 4, 60, 700, 16
+    st = Stack(L, B, Hq, Hkv, D, S, R, n_ctx + 1, dtype, n_ctx_max=n_ctx, w_last_max=T)
+    for l in range(L):
+        st.k_full[l][:, :, :n_ctx] = torch.randn(B, Hkv, n_ctx, D).to(dtype).cuda()
+    q_tail = (1.3 * torch.randn(L, B, Hq, T, D)).to(dtype).cuda()
+    whole = _run_scores(st, q_tail, n_ctx, T)
+    assert np.max(np.abs(f64(whole) - _oracle_scores(st, q_tail, n_ctx))) <= SCORE_ABS
+    for ranges in ([(l, 1) for l in range(L)], [(0, 2), (2, 3)], [(3, 2), (0, 3)]):
+        got = torch.full_like(whole, float("nan"))
+        for begin, count in ranges:
+            before = got.clone()
+            only = [st.k_full[l] if begin <= l < begin + count else None for l in range(L)]     # the rest is "freed"
+            tabs = lt.LayerTables(st.shape, only, None, None, None)
+            lt.lazy_scores(st.shape, q_tail, tabs, n_ctx, T, got, st.ws, layer_begin=begin, layer_count=count)
+            untouched = [l for l in range(L) if not begin <= l < begin + count]
+            assert torch.equal(torch.nan_to_num(got[untouched], nan=-7.0), torch.nan_to_num(before[untouched], nan=-7.0))
+        assert torch.equal(got, whole), ranges
+    assert lt.check(st.ws) == 0
+
+
 def test_select_fed_oracle_scores_is_bit_exact():
     g = np.random.default_rng(6)
     for L, B, Hq in [(2, 1, 4), (32, 8, 32), (64, 4, 40), (7, 3, 5), (128, 1, 1)]:
