@@ -61,7 +61,8 @@ def test_scores_match_oracle(dtype, D, Hq, Hkv, S, R, n_ctx, T, scale):
 
 @pytest.mark.parametrize("dtype,D", [(torch.float32, 64), (torch.bfloat16, 128)])
 def test_scoring_a_layer_range_equals_the_whole_stack_call(dtype, D):
-    """Layer by layer, in ranges and all at once: the same bits, only the scored layers' slices are written, and
+    """Layer by layer, in ranges and all at once: the same scores up to the rounding of another split of the keys
+    (the split depends on how many layers share the launch), only the scored layers' slices are written, and
     table entries outside the range may be missing (both kernels: CUDA-core and tensor-core path)."""
     torch.manual_seed(8)
     L, B, Hq, Hkv, S, R, n_ctx, T = 5, 2, 4, 2, 4, 60, 700, 16
@@ -80,7 +81,8 @@ def test_scoring_a_layer_range_equals_the_whole_stack_call(dtype, D):
             lt.lazy_scores(st.shape, q_tail, tabs, n_ctx, T, got, st.ws, layer_begin=begin, layer_count=count)
             untouched = [l for l in range(L) if not begin <= l < begin + count]
             assert torch.equal(torch.nan_to_num(got[untouched], nan=-7.0), torch.nan_to_num(before[untouched], nan=-7.0))
-        assert torch.equal(got, whole), ranges
+        assert float((got - whole).abs().max()) <= 2e-6, ranges
+        assert np.max(np.abs(f64(got) - _oracle_scores(st, q_tail, n_ctx))) <= SCORE_ABS
     assert lt.check(st.ws) == 0
 
 
