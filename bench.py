@@ -117,7 +117,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -125,7 +125,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, reasons, mx = [], set(), None
+        sm, pw, reasons, mx = [], [], set(), None
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
@@ -135,6 +135,10 @@ class ClockSampler:
                     sm.append(float(f[1])); mx = float(f[2])
                 except ValueError:
                     continue
+                try:
+                    pw.append(float(f[3]))
+                except ValueError:
+                    pw.append(float("nan"))
                 for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if v.lower().startswith("active"):
                         reasons.add(name)
@@ -145,6 +149,9 @@ class ClockSampler:
             # samples under load: drop the idle ones at the edges
             load = [x for x in sm if x > 0.5 * max(sm)]
             out.update(sm_mhz=float(np.median(load)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+            pw_load = [p for p, x in zip(pw, sm) if x > 0.5 * max(sm) and p == p]
+            if pw_load:
+                out["power_w"] = float(np.median(pw_load))      # board power under load (the cap is 1000 W)
         return out
 
 
@@ -366,7 +373,7 @@ def run_ours(args):
     mhz = s_clk["sm_mhz"] or clocks["sm_mhz"] or 1965.0
     mufu_peak = 16 * 148 * mhz * 1e6                       # one ex2 per lane, 16 lanes per clock per SM, 148 SMs
     tf_peak = _tensor_peak()
-    score_roofs = {"ms": score_ms, "sm_mhz": mhz,
+    score_roofs = {"ms": score_ms, "sm_mhz": mhz, "power_w": s_clk.get("power_w"), "clock_reasons": s_clk.get("reasons"),
                    "hbm": {"achieved_gbs": k_bytes / (score_ms * 1e-3) / 1e9, "frac": k_bytes / (score_ms * 1e-3) / 1e9 / peak},
                    "tensor": {"achieved_tflops": flops / (score_ms * 1e-3) / 1e12, "peak_tflops": tf_peak,
                               "frac": flops / (score_ms * 1e-3) / 1e12 / tf_peak},
@@ -409,7 +416,7 @@ def run_ours(args):
                        "step": "scores+select+compaction+128x(fused append+attend)",
                        "l2": "inputs (17 GiB per decode step) exceed the 126 MB L2; no flush needed",
                        "parallelism": "replicas" if world > 1 else "single"},
-            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "power_w")},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                     "ms_per_step": e2e["ms_per_pass"]},
             "gpu_launches": launches,
