@@ -508,7 +508,32 @@ def run_variants(wl, mask_hybrid):
     ms = time_steps(shape8, tables8, ws8, cfg.n_ctx)
     kv8 = algorithmic_bytes_decode(cfg, n_mean, cfg.n_lazy) / 2          # one byte per cached element
     res["fp8_caches"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs_of_8bit_bytes": kv8 / (ms * 1e-3) / 1e9}
-    del k8, v8, ks8, vs8, ws8
+    del k8, v8, ks8, vs8, ws8, tables8
+    # (c) the same stack with head_dim 64 (bf16): half the bytes per token, 32-key tiles of 128-byte rows
+    shape64 = lt.Shape(L, B, Hq, Hkv, 64, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16)
+    mk64 = lambda n: [torch.randn((B, Hkv, n, 64), device=dev).bfloat16() for _ in range(L)]  # noqa: E731
+    k64, v64, ks64, vs64 = mk64(cap), mk64(cap), mk64(C), mk64(C)
+    tables64 = lt.LayerTables(shape64, k64, v64, ks64, vs64)
+    ws64 = torch.empty(lt.workspace_bytes(shape64), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws64)
+    q64, kn64 = (torch.randn((L, B, h, 64), device=dev).bfloat16() for h in (Hq, Hkv))
+    out64 = torch.zeros((L, B, Hq, 64), dtype=torch.bfloat16, device=dev)
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        lt.decode_step(shape64, q64, kn64, kn64, tables64, mask_hybrid, seq, out64, ws64)
+    torch.cuda.synchronize()
+    seq.fill_(cfg.n_ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(16):
+        lt.decode_step(shape64, q64, kn64, kn64, tables64, mask_hybrid, seq, out64, ws64)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws64) == 0
+    ms = e0.elapsed_time(e1) / 16
+    b64 = algorithmic_bytes_decode(cfg.scaled(head_dim=64), n_mean, cfg.n_lazy)
+    res["head_dim_64"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b64 / (ms * 1e-3) / 1e9}
+    del k64, v64, ks64, vs64, ws64, tables64
     return res
 
 

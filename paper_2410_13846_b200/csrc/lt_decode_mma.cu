@@ -1,5 +1,5 @@
-// Decode step, bandwidth path: bf16 activations, head_dim 128, GQA group <= 8;
-// caches in bf16 or (template branch FP8) in E4M3 bytes.
+// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 8;
+// caches in bf16 or (template branch FP8, head_dim 128) in E4M3 bytes.
 //
 // A persistent launch (two CTAs per SM) walks the flattened work list of
 // (layer, batch row, kv head, KV chunk) items; items are handed out through a
@@ -148,8 +148,6 @@ __device__ __forceinline__ void st_shared_u32x4(uint32_t addr, uint32_t x, uint3
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
 
-constexpr int kD = 128;
-constexpr int kSrcRowBytes = kD * 2;  // one row of q, k_new, v_new (bf16)
 
 }  // namespace
 
@@ -186,13 +184,19 @@ struct TileSrc {
 // Q and P are f16 as well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
 // is folded into the softmax scale and the V scale (x 256) into the final
 // normalisation.  32-key tiles give every warp two independent MMA chains.
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
+  static_assert(DH == 128 || (DH == 64 && !FP8), "head_dim 128, or 64 with 16-bit caches");
+  constexpr int kD = DH;                       // head_dim
+  constexpr int kSrcRowBytes = kD * 2;         // one row of q, k_new, v_new (bf16)
+  constexpr int NK = kD / 16;                  // 16-wide k-steps of S = K Q^T = 16-row tiles of O^T
+  constexpr int HALVES = kD / 64;              // 128-byte halves of a 16-bit row
+  constexpr int VPR = kD / 8;                  // 16-byte vectors of a 16-bit row
   constexpr int MT = TILE / 16;                // 16-key MMA tiles per pipeline tile
   constexpr int HALF_BYTES = TILE * 128;       // one half-tile
-  constexpr int STAGE_BYTES = 4 * HALF_BYTES;  // K halves + V halves (16-bit layout)
+  constexpr int STAGE_BYTES = 2 * HALVES * HALF_BYTES;  // K halves + V halves (16-bit layout)
   constexpr int kRowBytes = FP8 ? kD : 2 * kD;             // one cached K or V row
   constexpr int RAW_BYTES = 2 * TILE * kD;                 // FP8: K rows + V rows of a tile as stored
   constexpr int RING_STAGE = FP8 ? RAW_BYTES : STAGE_BYTES;  // what one ring stage holds
@@ -204,7 +208,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads;
-  float* sm_buf = reinterpret_cast<float*>(smem + RING_BYTES);  // [2][8][128]
+  float* sm_buf = reinterpret_cast<float*>(smem + RING_BYTES);  // [2][8][head_dim]
   float* sm_m = sm_buf + 2 * 8 * kD;                            // [WARPS][8]
   float* sm_l = sm_m + WARPS * 8;                               // [WARPS][8]
   pdl_wait_prior_grid();   // the previous launch of the stream is complete: lengths, counters and partial slots are ours
@@ -302,16 +306,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < TILE / 2; ++i) {
-        const int r = 2 * i + (lane >> 4);
-        const int p = lane & 15;
+      for (int i = 0; i < TILE * VPR / 32; ++i) {
+        const int r = (32 / VPR) * i + lane / VPR;
+        const int p = lane % VPR;
         const int row = key_base + r;
         const bool valid = row < t.j1;
         const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
         const uint32_t soff = (p >> 3) * HALF_BYTES + r * 128 + (((p & 7) ^ (r & 7)) << 4);
         const bool fresh = row == t.new_row;
         cp_async16(st + soff, fresh ? t.k_new_row + p * 16 : t.Kb + goff, valid ? 16 : 0);
-        cp_async16(st + 2 * HALF_BYTES + soff, fresh ? t.v_new_row + p * 16 : t.Vb + goff, valid ? 16 : 0);
+        cp_async16(st + HALVES * HALF_BYTES + soff, fresh ? t.v_new_row + p * 16 : t.Vb + goff, valid ? 16 : 0);
       }
     }
   };
@@ -372,15 +376,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           *reinterpret_cast<uint4*>(dp) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
         }
       } else {
-        const uint8_t* sp = (lane < 16 ? src_cur.k_new_row : src_cur.v_new_row) + (lane & 15) * 16;
-        uint8_t* dp = const_cast<uint8_t*>(lane < 16 ? src_cur.Kb : src_cur.Vb) +
-                      cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane & 15) * 16;
-        *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
+        if (lane < 2 * VPR) {
+          const uint8_t* sp = (lane < VPR ? src_cur.k_new_row : src_cur.v_new_row) + (lane % VPR) * 16;
+          uint8_t* dp = const_cast<uint8_t*>(lane < VPR ? src_cur.Kb : src_cur.Vb) +
+                        cache_row(src_cur, src_cur.new_row) * kRowBytes + (lane % VPR) * 16;
+          *reinterpret_cast<uint4*>(dp) = *reinterpret_cast<const uint4*>(sp);
+        }
       }
     }
 
     // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
-    uint32_t qf[FP8 ? 1 : 8][2];
+    uint32_t qf[FP8 ? 1 : NK][2];
     // 8-bit caches: the stored K bytes are the A operand of E4M3 MMAs as they are, and q is their B operand as
     // a sum of kQTerms E4M3 terms at one power-of-two scale per head (block blk covers d = 32 blk .. 32 blk + 31:
     // bytes 4c .. 4c+3 in b0, 16 + 4c .. in b1).
@@ -426,7 +432,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         q_scale1 = __shfl_sync(0xffffffffu, scale, (2 * c + 1) * 4);
       } else {
 #pragma unroll
-        for (int ks8 = 0; ks8 < 8; ++ks8) {
+        for (int ks8 = 0; ks8 < NK; ++ks8) {
           if (gp < G) {
             qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
             qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
@@ -439,9 +445,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     }
 
     const float cs0 = cs_l * q_scale0, cs1 = cs_l * q_scale1;  // per S column (head 2c, 2c + 1)
-    float o[8][4];
+    float o[NK][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < NK; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
     float M0 = -INFINITY, M1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2c and 2c+1
@@ -476,7 +482,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
           float sc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int ks8 = 0; ks8 < 8; ++ks8) {
+          for (int ks8 = 0; ks8 < NK; ++ks8) {
             uint32_t af[4];
             const int chunk = 2 * (ks8 & 3) + k_chk;
             ldmatrix_x4(af, st + (ks8 >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
@@ -512,7 +518,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       l0 *= corr0;
       l1 *= corr1;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < NK; ++i) {
         o[i][0] *= corr0;
         o[i][1] *= corr1;
         o[i][2] *= corr0;
@@ -555,11 +561,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         } else {
           const int row = mt * 16 + v_row;
 #pragma unroll
-          for (int dt = 0; dt < 8; ++dt) {
+          for (int dt = 0; dt < NK; ++dt) {
             uint32_t af[4];
             const int chunk = 2 * (dt & 3) + v_chk;
-            ldmatrix_x4_trans(af,
-                              st + 2 * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4));
+            ldmatrix_x4_trans(af, st + HALVES * HALF_BYTES + (dt >> 2) * HALF_BYTES + row * 128 +
+                                      ((chunk ^ (row & 7)) << 4));
             mma_bf16(o[dt], af, bh0, bh1);
             mma_bf16(o[dt], af, bl0, bl1);
           }
@@ -603,7 +609,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       const float f0 = Mx0 > -INFINITY ? exp2f(M0 - Mx0) : 0.f;
       const float f1 = Mx1 > -INFINITY ? exp2f(M1 - Mx1) : 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < NK; ++i) {
         o[i][0] *= f0;
         o[i][1] *= f1;
         o[i][2] *= f0;
@@ -614,7 +620,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     auto buf_at = [&](int which, int) { return sm_buf + which * (8 * kD) + (2 * c) * kD; };
     if (warp >= 2) {
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
+      for (int dt = 0; dt < NK; ++dt) {
         float* p = buf_at(warp - 2, dt);
         p[dmap(dt, 0)] = o[dt][0];
         p[kD + dmap(dt, 0)] = o[dt][1];
@@ -625,7 +631,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     __syncthreads();
     if (warp < 2) {
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
+      for (int dt = 0; dt < NK; ++dt) {
         const float* p = buf_at(warp, dt);
         o[dt][0] += p[dmap(dt, 0)];
         o[dt][1] += p[kD + dmap(dt, 0)];
@@ -636,7 +642,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     __syncthreads();  // buffer 0 has been read by warp 0 before warp 1 overwrites it
     if (warp == 1) {
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
+      for (int dt = 0; dt < NK; ++dt) {
         float* p = buf_at(0, dt);
         p[dmap(dt, 0)] = o[dt][0];
         p[kD + dmap(dt, 0)] = o[dt][1];
@@ -648,7 +654,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     const bool single = w.nc <= 1;  // the whole (layer, b, kv head) is this one chunk
     if (warp == 0) {
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
+      for (int dt = 0; dt < NK; ++dt) {
         const float* p = buf_at(0, dt);
         o[dt][0] += p[dmap(dt, 0)];
         o[dt][1] += p[kD + dmap(dt, 0)];
@@ -664,7 +670,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           if (g < G) {
             const float den = e ? ls1 : ls0;
 #pragma unroll
-            for (int dt = 0; dt < 8; ++dt) {
+            for (int dt = 0; dt < NK; ++dt) {
 #pragma unroll
               for (int half = 0; half < 2; ++half) {
                 const float num = o[dt][e + 2 * half];
@@ -684,7 +690,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
           if (g < G) {
             float* po = a.part_o + (unit * G + g) * kD;
 #pragma unroll
-            for (int dt = 0; dt < 8; ++dt) {
+            for (int dt = 0; dt < NK; ++dt) {
               po[dmap(dt, 0)] = o[dt][e];
               po[dmap(dt, 1)] = o[dt][e + 2];
             }
@@ -717,17 +723,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   finish_launch(a);
 }
 bool decode_mma_supported(const lt_shape& s) {
-  return s.dtype == LT_BF16 && s.head_dim == 128 && (s.n_q_heads / s.n_kv_heads) <= 8;
+  return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) && (s.n_q_heads / s.n_kv_heads) <= 8;
 }
 
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8>
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int ring = FP8 ? WARPS * NSTAGE * TILE * 256 : WARPS * NSTAGE * TILE * 512;
-  constexpr int merge = 2 * 8 * 128 * 4 + 2 * WARPS * 8 * 4;
-  static_assert(2 * 8 * 128 * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
+  constexpr int ring = FP8 ? WARPS * NSTAGE * TILE * 256 : WARPS * NSTAGE * TILE * 4 * DH;
+  constexpr int merge = 2 * 8 * DH * 4 + 2 * WARPS * 8 * 4;
+  static_assert(2 * 8 * DH * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
-  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8>;
+  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8, DH>;
   // Per device, behind a lock (host threads may issue their first calls concurrently): the dynamic
   // shared-memory limit is raised once to the largest size any launch of this variant can ask for, and
   // the occupancy of each shared-memory size met so far is remembered (host time matters for per-layer callers).
@@ -768,8 +774,10 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
   // 8-bit caches: three raw stages of 32 keys (8 KB) = the 24 KB per warp of the 16-bit ring
-  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true>(a, kf, vf, ks, vs, st);
-  return launch_variant<16, 3, 4, 2, false>(a, kf, vf, ks, vs, st);
+  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true, 128>(a, kf, vf, ks, vs, st);
+  // head_dim 64: rows are half as long, so 32-key tiles keep the bytes in flight per warp (24 KB) the same
+  if (a.s.head_dim == 64) return launch_variant<32, 3, 4, 2, false, 64>(a, kf, vf, ks, vs, st);
+  return launch_variant<16, 3, 4, 2, false, 128>(a, kf, vf, ks, vs, st);
 }
 
 }  // namespace lt
