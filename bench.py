@@ -534,6 +534,31 @@ def run_variants(wl, mask_hybrid):
     b64 = algorithmic_bytes_decode(cfg.scaled(head_dim=64), n_mean, cfg.n_lazy)
     res["head_dim_64"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b64 / (ms * 1e-3) / 1e9}
     del k64, v64, ks64, vs64, ws64, tables64
+    # (d) a query group of 16 (32 q / 2 kv heads): the kernel serves it as two sub-groups of 8 heads, i.e. two work
+    # items per chunk; algorithmic bytes count every cached byte once
+    cfg16 = cfg.scaled(n_kv_heads=2)
+    shape16 = lt.Shape(L, B, Hq, 2, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16)
+    mk16 = lambda n: [torch.randn((B, 2, n, D), device=dev).bfloat16() for _ in range(L)]  # noqa: E731
+    k16, v16, ks16, vs16 = mk16(cap), mk16(cap), mk16(C), mk16(C)
+    tables16 = lt.LayerTables(shape16, k16, v16, ks16, vs16)
+    ws16 = torch.empty(lt.workspace_bytes(shape16), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws16)
+    kn16 = torch.randn((L, B, 2, D), device=dev).bfloat16()
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        lt.decode_step(shape16, q, kn16, kn16, tables16, mask_hybrid, seq, out, ws16)
+    torch.cuda.synchronize()
+    seq.fill_(cfg.n_ctx)
+    e0.record()
+    for _ in range(16):
+        lt.decode_step(shape16, q, kn16, kn16, tables16, mask_hybrid, seq, out, ws16)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws16) == 0
+    ms = e0.elapsed_time(e1) / 16
+    b16 = algorithmic_bytes_decode(cfg16, n_mean, cfg.n_lazy)
+    res["group_16"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b16 / (ms * 1e-3) / 1e9}
+    del k16, v16, ks16, vs16, ws16, tables16
     return res
 
 

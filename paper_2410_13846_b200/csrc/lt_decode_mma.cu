@@ -1,4 +1,5 @@
-// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 8;
+// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 16 (groups above 8 as
+// two sub-groups of at most 8 heads, each its own work item);
 // caches in bf16 or (template branch FP8, head_dim 128) in E4M3 bytes.
 //
 // A persistent launch (two CTAs per SM) walks the flattened work list of
@@ -214,7 +215,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   pdl_wait_prior_grid();   // the previous launch of the stream is complete: lengths, counters and partial slots are ours
   pdl_allow_next_grid();   // the next launch may take SMs as this one's CTAs retire (it waits the same way)
   WorkList wl;
-  wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
+  wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch, a.hsub);
   wl.build(a, kf, vf, ks, vs);
   const int n_items = wl.total(a);
 
@@ -352,6 +353,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   while (cur < n_items) {
     const int l = w.l, b = w.b, h = w.h;
+    const int Gn = w.gn;  // query heads served by this item (the group, or one sub-group of at most 8)
     const int j1 = src_cur.j1;
     int fetched_next = 0;
     if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
@@ -394,7 +396,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     float q_scale0 = 1.f, q_scale1 = 1.f;  // scale of heads 2c and 2c + 1 (this thread's S columns)
     {
       const __nv_bfloat16* qp =
-          (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + gp) * kD;
+          (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + w.g0 + gp) * kD;
       if constexpr (FP8) {
         float x[4][2][4];
         float amax = 0.f;
@@ -403,7 +405,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             uint2 q4 = make_uint2(0u, 0u);
-            if (gp < G) q4 = *reinterpret_cast<const uint2*>(qp + 32 * blk + 16 * hf + 4 * c);
+            if (gp < Gn) q4 = *reinterpret_cast<const uint2*>(qp + 32 * blk + 16 * hf + 4 * c);
             x[blk][hf][0] = bf16_lo(q4.x);
             x[blk][hf][1] = bf16_hi(q4.x);
             x[blk][hf][2] = bf16_lo(q4.y);
@@ -433,7 +435,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       } else {
 #pragma unroll
         for (int ks8 = 0; ks8 < NK; ++ks8) {
-          if (gp < G) {
+          if (gp < Gn) {
             qf[ks8][0] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 2 * c);
             qf[ks8][1] = *reinterpret_cast<const uint32_t*>(qp + 16 * ks8 + 8 + 2 * c);
           } else {
@@ -663,11 +665,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       }
       if (single) {
         // no partials: normalise and write the output of heads 2c, 2c + 1 directly
-        const long long ob = (((long long)l * s.batch + b) * s.n_q_heads + h * G) * kD;
+        const long long ob = (((long long)l * s.batch + b) * s.n_q_heads + h * G + w.g0) * kD;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
-          if (g < G) {
+          if (g < Gn) {
             const float den = e ? ls1 : ls0;
 #pragma unroll
             for (int dt = 0; dt < NK; ++dt) {
@@ -687,16 +689,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
-          if (g < G) {
-            float* po = a.part_o + (unit * G + g) * kD;
+          if (g < Gn) {
+            float* po = a.part_o + (unit * a.gp_stride + g) * kD;
 #pragma unroll
             for (int dt = 0; dt < NK; ++dt) {
               po[dmap(dt, 0)] = o[dt][e];
               po[dmap(dt, 1)] = o[dt][e + 2];
             }
             if (gp == 0) {
-              a.part_ml[(unit * G + g) * 2] = e ? Mx1 : Mx0;
-              a.part_ml[(unit * G + g) * 2 + 1] = e ? ls1 : ls0;
+              a.part_ml[(unit * a.gp_stride + g) * 2] = e ? Mx1 : Mx0;
+              a.part_ml[(unit * a.gp_stride + g) * 2 + 1] = e ? ls1 : ls0;
             }
           }
         }
@@ -723,7 +725,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   finish_launch(a);
 }
 bool decode_mma_supported(const lt_shape& s) {
-  return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) && (s.n_q_heads / s.n_kv_heads) <= 8;
+  // groups of 9..16 are served as two sub-groups of at most 8 heads (the chunk is read twice, the second time from L2)
+  return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
+         (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 8 : 16);
 }
 
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
