@@ -16,7 +16,7 @@
 // ranges, one per CTA, so every SM gets the same number of tiles whatever the
 // unit count; a unit that straddles a cut gets its own statistics slots per piece.
 // With the denominator given (lt_lazy_scores_lse) the work items are the host's
-// key splits of the kept ranges, dealt round-robin.
+// key splits of the kept ranges, a contiguous run of them per CTA.
 //
 // Roles (18 warps):
 //   warp 0      producer: one lane streams the unit's query block (64 KB, at a change
@@ -326,10 +326,14 @@ __device__ __forceinline__ bool next_piece(const ScoreArgs& a, long long& cursor
     slot = (int)blockIdx.x - score_tile_owner(a.total_tiles, gridDim.x, (long long)unit * TU);
     cursor += n_tiles;
   } else {
+    // host splits of the kept key ranges: every CTA takes a contiguous run of (unit, split) items, so that the
+    // query block in shared memory is replaced only when the run moves on to the next unit
     const int host_splits = a.n_splits / 2;
     const long long n_items = (long long)a.n_units * host_splits;
-    const long long item = (long long)blockIdx.x + cursor * gridDim.x;
-    if (item >= n_items) return false;
+    long long i_begin, i_end;
+    score_cta_tiles(n_items, gridDim.x, blockIdx.x, &i_begin, &i_end);
+    const long long item = i_begin + cursor;
+    if (item >= i_end) return false;
     unit = (int)(item / host_splits);
     slot = (int)(item - (long long)unit * host_splits);
     score_split_range(a, slot, &k0, &k1);
