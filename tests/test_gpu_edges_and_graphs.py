@@ -113,3 +113,56 @@ def test_captured_decode_step_replays():
     assert torch.equal(graph.seq_lens, eager.seq_lens) and lt.check(graph.ws) == 0
     for l in range(L):
         assert torch.equal(graph.k_full[l], eager.k_full[l]) and torch.equal(graph.k_stream[l], eager.k_stream[l])
+
+
+def test_captured_per_layer_step_replays():
+    """A step issued layer by layer (launches that carry the programmatic-serialization attribute) captured
+    as one CUDA graph: every replay equals an eager whole-stack step, bit for bit."""
+    torch.manual_seed(6)
+    L, B, Hq, Hkv, D, S, R, n0, steps = 5, 2, 8, 2, 128, 4, 28, 700, 12
+    cap = n0 + steps + 2
+    eager = Stack(L, B, Hq, Hkv, D, S, R, cap)
+    graph = Stack(L, B, Hq, Hkv, D, S, R, cap)
+    for st in (eager, graph):
+        st.set_mask([0, 1, 0, 1, 0]); st.set_seq_lens([n0, n0 - 300])
+    for l in range(L):
+        k0 = torch.randn(B, Hkv, cap, D).bfloat16().cuda(); v0 = torch.randn(B, Hkv, cap, D).bfloat16().cuda()
+        for st in (eager, graph):
+            st.k_full[l].copy_(k0); st.v_full[l].copy_(v0)
+    for st in (eager, graph):
+        lt.stream_init(st.shape, st.mask, st.tables, st.seq_lens, ws=st.ws)
+    sq = torch.zeros(L, B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    sk = torch.zeros(L, B, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    sv = torch.zeros_like(sk)
+    so = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+
+    def per_layer_step(st):
+        for l in range(L):
+            lt.decode_step(st.shape, sq, sk, sv, st.tables, st.mask, st.seq_lens, so, st.ws, layer_begin=l,
+                           layer_count=1, advance_seq_lens=(l == L - 1))
+
+    warm = Stack(L, B, Hq, Hkv, D, S, R, cap)                    # per-device lookups happen outside the capture
+    warm.set_seq_lens([1, 1])
+    per_layer_step(warm)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            per_layer_step(graph)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    ref = torch.zeros_like(so)
+    for step in range(steps):
+        q = torch.randn(L, B, Hq, D).bfloat16().cuda()
+        k = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        v = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        lt.decode_step(eager.shape, q, k, v, eager.tables, eager.mask, eager.seq_lens, ref, eager.ws)
+        sq.copy_(q); sk.copy_(k); sv.copy_(v)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(so, ref), step
+    assert torch.equal(graph.seq_lens, eager.seq_lens) and lt.check(graph.ws) == 0
+    for l in range(L):
+        assert torch.equal(graph.k_full[l], eager.k_full[l]) and torch.equal(graph.k_stream[l], eager.k_stream[l])
