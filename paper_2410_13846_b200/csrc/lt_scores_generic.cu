@@ -92,31 +92,32 @@ cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cuda
   return cudaGetLastError();
 }
 
-// One thread per (layer, b, hq): merge the statistics slots of every tail row, take the
-// row's mass W/A, average over the w_last rows in row order.  The statistics are indexed by the
-// layer's position in the scored range.
+// One warp per (layer, b, hq): lane t, t + 32, ... merges the statistics slots of its tail rows and takes the
+// row's mass W/A; the lanes' sums are added in a fixed tree and divided by w_last.  The statistics are indexed by
+// the layer's position in the scored range.
 __global__ void scores_finish_kernel(ScoreArgs a) {
   const lt_shape& s = a.s;
   const long long per_layer = (long long)s.batch * s.n_q_heads;
-  const long long rel = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (rel >= a.layer_count * per_layer) return;
+  const int lane = threadIdx.x & 31;
+  const long long rel = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (rel >= a.layer_count * per_layer) return;  // whole warps leave together
   const long long idx = a.layer_begin * per_layer + rel;
   const int T = a.w_last;
+  int n_slots = a.n_splits;
+  long long unit_row0 = 0;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  const int hq = (int)(rel % s.n_q_heads);
+  if (a.streamk) unit_row0 = ((rel / s.n_q_heads) * s.n_kv_heads + hq / G) * a.row_blocks;  // first unit of this kv head
   float sum = 0.f;
-  for (int t = 0; t < T; ++t) {
+  for (int t = lane; t < T; t += 32) {
     const float* st = a.stats + ((rel * T + t) * a.n_splits) * 3;
-    int n_slots = a.n_splits;
     if (a.streamk) {
-      // the persistent kernel wrote one slot per piece of this row's unit: the CTAs from the owner of the
-      // unit's first tile to the owner of its last one
-      const int G = s.n_q_heads / s.n_kv_heads;
-      const int hq = (int)(rel % s.n_q_heads);
-      const long long lb = rel / s.n_q_heads;  // (layer in range) * B + b
-      const int r = (hq % G) * T + t;          // row among the kv head's G * T query rows
-      const long long unit = (lb * s.n_kv_heads + hq / G) * a.row_blocks + r / kScoreBlockM;
-      const long long g0 = unit * a.tiles_per_unit;
+      // the persistent kernel wrote two slots per piece of this row's unit: the CTAs from the owner of the
+      // unit's first tile to the owner of its last one (two slots each: halves of a tile's keys)
+      const int r = (hq % G) * T + t;  // row among the kv head's G * T query rows
+      const long long g0 = (unit_row0 + r / kScoreBlockM) * a.tiles_per_unit;
       n_slots = 2 * (score_tile_owner(a.total_tiles, a.grid, g0 + a.tiles_per_unit - 1) -
-                     score_tile_owner(a.total_tiles, a.grid, g0) + 1);  // two slots per piece (halves of a tile's keys)
+                     score_tile_owner(a.total_tiles, a.grid, g0) + 1);
     }
     float Mx = -INFINITY;
     for (int sp = 0; sp < n_slots; ++sp) Mx = fmaxf(Mx, st[sp * 3]);
@@ -136,12 +137,14 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
       sum += W / A;
     }
   }
-  a.scores[idx] = sum / (float)T;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+  if (lane == 0) a.scores[idx] = sum / (float)T;
 }
 
 cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st) {
-  const long long total = (long long)a.layer_count * a.s.batch * a.s.n_q_heads;
-  scores_finish_kernel<<<(unsigned)((total + 127) / 128), 128, 0, st>>>(a);
+  const long long warps = (long long)a.layer_count * a.s.batch * a.s.n_q_heads;
+  scores_finish_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(a);
   return cudaGetLastError();
 }
 
