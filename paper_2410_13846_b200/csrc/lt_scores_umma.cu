@@ -36,8 +36,8 @@
 //               chunk is in registers.
 //
 // Exponentials.  One ex2 per score on the special-function unit (16 per clock per
-// SM) is the floor of this kernel (the unit is ~80 % busy with nothing but the
-// statistics running), so a fixed share of the columns takes 2^x on the FMA pipe
+// SM) makes that unit the busiest of the SM (~80 %), so a fixed share of the columns
+// takes 2^x on the FMA pipe
 // instead: the reference of a row is an INTEGER M >= max (log2 domain), so x = t - M
 // splits exactly into round(x) and a remainder f in [-1/2, 1/2]; 2^f is a cubic
 // (relative error 7.5e-5, far inside the 1e-3 absolute tolerance of a ratio of sums)
@@ -45,6 +45,10 @@
 // uses the packed two-lane fp32 instructions (fma / add .f32x2).  The share is small
 // (an eighth): measured, an ex2 costs the scheduler about five issue slots and the
 // polynomial about twelve, so a larger share only trades one bound for another.
+//
+// On B200 the pass as a whole runs at the board's power limit (about 1 kW with the
+// key stream, the MMAs and the statistics all active): its time follows its energy,
+// and changes to the instruction stream mostly change the clock the governor leaves.
 //
 // Every wait on an mbarrier is bounded in time; on expiry the kernel raises
 // LT_DEVERR_TIMEOUT in the workspace header, all roles leave their loops, TMEM
