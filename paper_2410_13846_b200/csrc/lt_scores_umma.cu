@@ -605,6 +605,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         ok = mbar_wait(bar_sfull + 8 * mb, uses & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        if (mb * 128 + quad * 32 >= rows_here) {
+          // none of this warp's 32 rows exists (a ragged query block): nothing to read, hand the accumulator back
+          tc_fence_before();
+          mbar_arrive(bar_sempty + 8 * mb);
+          continue;
+        }
         // Four chunks of 32 columns through one register buffer: the load of a chunk is not overlapped
         // by this warp's own arithmetic but by the three other statistics warps of its scheduler (two
         // buffers would not fit the 96 registers a thread gets).
