@@ -10,6 +10,7 @@ all 32 layers + seq_lens advance).
 `value` = decode tokens of all ranks / time of the timed passes.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --workload {llama2_7b_4k,llama31_8b_128k,qwq32b_longgen}   # one of the other workloads alone
 
 N > 1 (under torch.distributed.run) runs one independent replica per GPU: the
 path has no exchange step, so there is no data-path collective.
@@ -612,7 +613,7 @@ def run_per_layer_calls(wl, mask_hybrid, peak):
             "frac_of_peak": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
 
 
-def run_other_configs(device, peak, gpu_index):
+def run_other_configs(device, peak, gpu_index, only=None):
     """Throughput of the other paper-shaped workloads (detail only; the headline stays the 32K stack):
     the Llama-2-7B-shaped MHA 4K stack (hybrid against all-full), the Llama-3.1-8B-shaped 128K stack with
     the lazy fraction swept over 0 / 25 / 50 / 75 %, and the QwQ-32B-shaped long generation as a
@@ -642,7 +643,7 @@ def run_other_configs(device, peak, gpu_index):
         return e0.elapsed_time(e1) / iters
 
     # ---- Llama-2-7B-shaped MHA stack, 4K context ------------------------------------------------------
-    try:
+    def mha_4k():
         cfg = CONFIGS["llama2_7b_4k"]
         wl = Workload(cfg, device)
         lt = wl.lt
@@ -657,17 +658,12 @@ def run_other_configs(device, peak, gpu_index):
         full = _time_decode_steps(lt, wl.shape, wl.tables, full_mask, wl.seq, cfg.n_ctx, wl.step_inputs, wl.out, wl.ws, steps)
         assert lt.check(wl.ws) == 0
         h, f = step_metrics(cfg, hyb, cfg.n_lazy, n_mean), step_metrics(cfg, full, 0, n_mean)
-        res["llama2_7b_4k"] = {"shape": "32 layers, 32 q / 32 kv heads (MHA), batch 32, context 4096, 16 lazy",
-                               "lazy_score_ms": s_ms, "hybrid": h, "all_full": f,
-                               "hybrid_over_all_full": full / hyb,
-                               "byte_ratio_ceiling": f["algorithmic_bytes"] / h["algorithmic_bytes"]}
-        del wl
-    except torch.cuda.OutOfMemoryError as e:  # a smaller device: say so instead of failing the headline
-        res["llama2_7b_4k"] = {"skipped": f"out of device memory: {e}"[:200]}
-    gc.collect(); torch.cuda.empty_cache()
+        return {"shape": "32 layers, 32 q / 32 kv heads (MHA), batch 32, context 4096, 16 lazy",
+                "lazy_score_ms": s_ms, "hybrid": h, "all_full": f, "hybrid_over_all_full": full / hyb,
+                "byte_ratio_ceiling": f["algorithmic_bytes"] / h["algorithmic_bytes"]}
 
     # ---- Llama-3.1-8B-shaped stack, 128K context, lazy fraction sweep ---------------------------------------
-    try:
+    def ctx_128k():
         cfg = CONFIGS["llama31_8b_128k"]
         wl = Workload(cfg, device)
         lt = wl.lt
@@ -688,15 +684,11 @@ def run_other_configs(device, peak, gpu_index):
             m["byte_ratio_ceiling"] = base_bytes / m["algorithmic_bytes"]
             sweep[f"{100 * n_lazy // L}%_lazy"] = m
         assert lt.check(wl.ws) == 0
-        res["llama31_8b_128k"] = {"shape": "32 layers, 32 q / 8 kv heads, batch 2, context 131072, window 4 + 4092",
-                                  "lazy_score_ms": s_ms, "lazy_fraction_sweep": sweep}
-        del wl
-    except torch.cuda.OutOfMemoryError as e:
-        res["llama31_8b_128k"] = {"skipped": f"out of device memory: {e}"[:200]}
-    gc.collect(); torch.cuda.empty_cache()
+        return {"shape": "32 layers, 32 q / 8 kv heads, batch 2, context 131072, window 4 + 4092",
+                "lazy_score_ms": s_ms, "lazy_fraction_sweep": sweep}
 
     # ---- QwQ-32B-shaped long generation: eager loop against a graph-replayed loop -------------------------
-    try:
+    def long_generation():
         cfg = CONFIGS["qwq32b_longgen"]
         wl = Workload(cfg, device)
         lt = wl.lt
@@ -747,7 +739,7 @@ def run_other_configs(device, peak, gpu_index):
         graph_ms = e0.elapsed_time(e1)
         assert lt.check(wl.ws) == 0 and wl.seq.cpu().tolist() == [cfg.n_ctx + n_steps] * B
         nbytes = float(np.mean([algorithmic_bytes_decode(cfg, cfg.n_ctx + i + 1, cfg.n_lazy) for i in range(n_steps)]))
-        res["qwq32b_longgen"] = {
+        return {
             "shape": "64 layers, 40 q / 8 kv heads (group of 5), batch 4, prompt 1024, 32 lazy, window 4 + 4092",
             "decode_steps": n_steps, "context_from_to": [cfg.n_ctx, cfg.n_ctx + n_steps],
             "mean_algorithmic_bytes_per_step": nbytes,
@@ -757,10 +749,15 @@ def run_other_configs(device, peak, gpu_index):
                              "decode_tokens_per_s": B * n_steps / (graph_ms * 1e-3),
                              "gbs": nbytes / (graph_ms / n_steps * 1e-3) / 1e9,
                              "frac_of_peak": nbytes / (graph_ms / n_steps * 1e-3) / 1e9 / peak}}
-        del wl, graph
-    except torch.cuda.OutOfMemoryError as e:
-        res["qwq32b_longgen"] = {"skipped": f"out of device memory: {e}"[:200]}
-    gc.collect(); torch.cuda.empty_cache()
+
+    for name, fn in (("llama2_7b_4k", mha_4k), ("llama31_8b_128k", ctx_128k), ("qwq32b_longgen", long_generation)):
+        if only is not None and only != name:
+            continue
+        try:
+            res[name] = fn()                   # the stack lives in fn's frame: gone when it returns
+        except torch.cuda.OutOfMemoryError as e:  # a smaller device: say so instead of failing the headline
+            res[name] = {"skipped": f"out of device memory: {e}"[:200]}
+        gc.collect(); torch.cuda.empty_cache()
     return res
 
 
@@ -847,6 +844,18 @@ def cpu_baseline(cfg, wl):
         return wl.q_tail[0, 0].double().cpu().numpy(), wl.k_full[0][0, :, :cfg.n_ctx].double().cpu().numpy()
 
     return _oracle_sample(cfg, get_unit, get_tail)
+
+
+def run_one_other_workload(args):
+    """`--workload NAME`: one of the other paper-shaped workloads alone (what the default run reports under
+    `detail.other_configs`), as one JSON line.  The headline line is the default run's."""
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(0)
+    from paper_2410_13846_b200 import build
+    build.build_library()
+    peak, peak_kind = _peaks()
+    res = run_other_configs(torch.device("cuda", 0), peak, 0, only=args.workload)
+    print(json.dumps({"workload": args.workload, "peak_gbs": peak, "peak_kind": f"of {peak_kind}", **res}))
 
 
 def run_reference(args):
@@ -945,6 +954,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default=None, choices=["llama2_7b_4k", "llama31_8b_128k", "qwq32b_longgen"],
+                    help="run one of the other workloads alone and print its detail (not the headline line)")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the MHA 4K, long-generation and 128K workloads that are reported in `detail`")
     ap.add_argument("--profile-case", type=int, default=0, metavar="DECODE_STEPS",
@@ -958,6 +969,8 @@ def main():
         run_profile_case(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.workload:
+        run_one_other_workload(args)
     else:
         run_ours(args)
 
