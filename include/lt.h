@@ -131,9 +131,11 @@ int32_t lt_version(void);
 int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent);
 
 /*
- * Bytes of workspace that lt_lazy_scores (prompt length up to n_ctx_max, up to
- * w_last_max tail queries) and lt_hybrid_decode_attn (any seq_len up to
- * max(full_capacity, n_sink + n_recent)) need for this shape.  Host only.
+ * Bytes of workspace that lt_lazy_scores / lt_lazy_scores_lse (prompt length up
+ * to n_ctx_max, up to w_last_max tail queries, any layer range) and
+ * lt_hybrid_decode_attn / lt_decode_step (any seq_len up to
+ * max(full_capacity, n_sink + n_recent), any layer range) need for this shape.
+ * Host only; pass 0, 0 when the workspace will not be used for scoring.
  * The workspace is device memory, 256-byte aligned, owned by the caller; it
  * starts with the device error word and the counters of the decode step, which
  * must be zeroed once with lt_workspace_init (every call leaves them zero).
