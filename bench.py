@@ -534,7 +534,25 @@ def run_variants(wl, mask_hybrid):
     ms = e0.elapsed_time(e1) / 16
     b64 = algorithmic_bytes_decode(cfg.scaled(head_dim=64), n_mean, cfg.n_lazy)
     res["head_dim_64"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b64 / (ms * 1e-3) / 1e9}
-    del k64, v64, ks64, vs64, ws64, tables64
+    # ... and its lazy scores over the whole prompt (Eq. 1): the tensor-core kernel with four 16-wide k-steps per tile
+    T = cfg.w_last
+    wsS = torch.empty(lt.workspace_bytes(shape64, cfg.n_ctx, T), dtype=torch.uint8, device=dev)
+    lt.workspace_init(wsS)
+    qt64 = torch.randn((L, B, Hq, T, 64), device=dev).bfloat16()
+    sc64 = torch.zeros((L, B, Hq), dtype=torch.float32, device=dev)
+    for _ in range(2):
+        lt.lazy_scores(shape64, qt64, tables64, cfg.n_ctx, T, sc64, wsS)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        lt.lazy_scores(shape64, qt64, tables64, cfg.n_ctx, T, sc64, wsS)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(wsS) == 0
+    ms = e0.elapsed_time(e1) / 3
+    res["head_dim_64"]["lazy_scores_ms"] = ms
+    res["head_dim_64"]["lazy_scores_tflops"] = 2.0 * L * B * Hq * T * cfg.n_ctx * 64 / (ms * 1e-3) / 1e12
+    del k64, v64, ks64, vs64, ws64, wsS, qt64, tables64
     # (d) a query group of 16 (32 q / 2 kv heads): the kernel serves it as two sub-groups of 8 heads, i.e. two work
     # items per chunk; algorithmic bytes count every cached byte once
     cfg16 = cfg.scaled(n_kv_heads=2)

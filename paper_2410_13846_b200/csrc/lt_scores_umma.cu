@@ -1,4 +1,4 @@
-// Lazy ratio (Eq. 1), Blackwell tensor-core path: bf16, head_dim 128.
+// Lazy ratio (Eq. 1), Blackwell tensor-core path: bf16, head_dim 128 or 64.
 //
 // S = Q K^T is a real dense contraction here (G * w_last query rows against
 // every prompt key), so it runs on the 5th-generation tensor cores:
@@ -66,17 +66,22 @@ namespace lt {
 
 namespace {
 
-constexpr int kD = 128;  // head_dim
-constexpr int kRowBytes = 256;
 constexpr int kBlockM = kScoreBlockM;  // query rows per unit (2 UMMA row blocks)
 constexpr int kBlockN = kScoreBlockN;  // keys per tile (one UMMA instruction wide)
-constexpr int kStages = 2;
-constexpr int kQHalfBytes = kBlockM * 128;        // one d-half of the query block: [256 rows][128 B]
-constexpr int kQBytes = 2 * kQHalfBytes;          // 64 KB
-constexpr int kKHalfBytes = kBlockN * 128;        // one d-half of a K tile: [256 rows][128 B]
-constexpr int kStageBytes = 2 * kKHalfBytes;      // 64 KB
+constexpr int kQHalfBytes = kBlockM * 128;        // 64 d (one 128-byte half of a row) of the query block: [256 rows][128 B]
+constexpr int kKHalfBytes = kBlockN * 128;        // 64 d of a K tile: [256 rows][128 B]
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+// Geometry that depends on the head dimension DH (128 or 64): a row has DH / 64 halves of 128 bytes; the K ring
+// holds 128 KB either way (2 stages of 64 KB, or 4 of 32 KB).
+template <int DH>
+struct Geo {
+  static constexpr int kHalves = DH / 64;
+  static constexpr int kQBytes = kHalves * kQHalfBytes;      // 64 KB or 32 KB
+  static constexpr int kStageBytes = kHalves * kKHalfBytes;  // 64 KB or 32 KB
+  static constexpr int kStages = 4 / kHalves;
+  static constexpr int kKSteps = DH / 16;                    // 16-wide k-steps of the contraction
+  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+};
 constexpr int kStatWarps = 16;
 constexpr int kThreads = 64 + kStatWarps * 32;    // 576 (registers are granted as for 640: 96 per thread)
 constexpr int kTmemCols = 512;   // two accumulators of 256 columns, one per row block
@@ -362,8 +367,11 @@ __device__ __forceinline__ bool next_piece(const ScoreArgs& a, long long& cursor
   return true;
 }
 
+template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
     scores_umma_kernel(ScoreArgs a, const __grid_constant__ KeyMaps maps) {
+  constexpr int kHalves = Geo<DH>::kHalves, kQBytes = Geo<DH>::kQBytes, kStageBytes = Geo<DH>::kStageBytes;
+  constexpr int kStages = Geo<DH>::kStages, kKSteps = Geo<DH>::kKSteps;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern of the MMA is a function of address bits 4..9
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -439,8 +447,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!ok) break;
             mbar_expect_tx(bar_qfull, kQBytes);
             const int yq = ((p.l * s.batch + p.b) * s.n_q_heads + p.h * G) * T + p.rb * kBlockM;
-            tma_load_2d(sQ, &maps.q, 0, yq, bar_qfull);
-            tma_load_2d(sQ + kQHalfBytes, &maps.q, 64, yq, bar_qfull);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) tma_load_2d(sQ + hf * kQHalfBytes, &maps.q, 64 * hf, yq, bar_qfull);
             ++q_loads;
             prev_unit = p.unit;
           }
@@ -464,8 +472,9 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int page = s.block_table[(long long)p.b * s.pages_per_seq + pg];
                 y = (page * s.n_kv_heads + p.h) * s.page_size + j % s.page_size;
               }
-              tma_load_2d(dst + rh * (128 * 128), map, 0, y, bar);
-              tma_load_2d(dst + kKHalfBytes + rh * (128 * 128), map, 64, y, bar);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf)
+                tma_load_2d(dst + hf * kKHalfBytes + rh * (128 * 128), map, 64 * hf, y, bar);
             }
           }
         }
@@ -511,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               tc_fence_after();
               const uint32_t d_tmem = tmem_base + mb * 256;
 #pragma unroll
-              for (int ks = 0; ks < 8; ++ks) {
+              for (int ks = 0; ks < kKSteps; ++ks) {
                 const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + mb * (128 * 128) + (ks & 3) * 32;
                 const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
                 umma_bf16_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
@@ -647,7 +656,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 bool scores_umma_supported(const lt_shape& s, int /*w_last*/) {
-  return s.dtype == LT_BF16 && s.head_dim == 128 &&
+  return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
          (long long)s.batch * s.n_kv_heads * s.full_capacity < (1ll << 31);  // tensor-map rows fit an int32 coordinate
 }
 
@@ -670,20 +679,21 @@ EncodeTiledFn encode_tiled_fn() {
 }
 }  // namespace
 
-// grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 640.
-cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
+// grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 576.
+template <int DH>
+static cudaError_t launch_scores_umma_dh(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return cudaErrorNotSupported;
   const cuuint64_t rows_total = a.s.page_size > 0 ? (cuuint64_t)a.s.n_pages * a.s.n_kv_heads * a.s.page_size
                                                   : (cuuint64_t)a.s.batch * a.s.n_kv_heads * a.s.full_capacity;
-  const cuuint64_t gdim[2] = {(cuuint64_t)kD, rows_total};
-  const cuuint64_t gstride[1] = {(cuuint64_t)kRowBytes};
+  const cuuint64_t gdim[2] = {(cuuint64_t)DH, rows_total};
+  const cuuint64_t gstride[1] = {(cuuint64_t)(2 * DH)};
   const cuuint32_t box[2] = {64u, 128u};
   const cuuint32_t estride[2] = {1u, 1u};
   KeyMaps local;
   {
-    // the tail queries of the whole stack as one matrix of 128-element rows; a box is one d-half of a unit's 256 rows
-    const cuuint64_t qdim[2] = {(cuuint64_t)kD,
+    // the tail queries of the whole stack as one matrix of head_dim-element rows; a box is 64 d of a unit's 256 rows
+    const cuuint64_t qdim[2] = {(cuuint64_t)DH,
                                 (cuuint64_t)a.s.n_layers * a.s.batch * a.s.n_q_heads * (cuuint64_t)a.w_last};
     const cuuint32_t qbox[2] = {64u, (cuuint32_t)kBlockM};
     const CUresult r = encode(&local.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.q_tail), qdim, gstride,
@@ -700,10 +710,15 @@ cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStr
   }
   for (int l = 0; l < LT_MAX_LAYERS; ++l)
     if (l < a.layer_begin || l >= l_end) local.m[l] = local.m[a.layer_begin];
-  cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  constexpr int smem = Geo<DH>::kSmemBytes;
+  cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  scores_umma_kernel<<<a.grid, kThreads, kSmemBytes, st>>>(a, local);
+  scores_umma_kernel<DH><<<a.grid, kThreads, smem, st>>>(a, local);
   return cudaGetLastError();
+}
+
+cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
+  return a.s.head_dim == 64 ? launch_scores_umma_dh<64>(a, kf, st) : launch_scores_umma_dh<128>(a, kf, st);
 }
 
 }  // namespace lt

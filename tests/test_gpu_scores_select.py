@@ -36,6 +36,8 @@ CASES = [
     (torch.bfloat16, 128, 4, 1, 4, 2044, 2500, 64, 0.0),   # paper defaults
     (torch.bfloat16, 128, 4, 1, 4, 60, 40, 40, 0.0),       # window covers everything -> 1.0
     (torch.bfloat16, 64, 4, 2, 2, 9, 300, 5, 0.0),         # D=64
+    (torch.bfloat16, 64, 16, 2, 4, 60, 1500, 64, 0.0),     # D=64, GQA 8: two 256-row blocks per (b, h)
+    (torch.bfloat16, 64, 8, 2, 6, 252, 4100, 32, 0.3),     # D=64, several key splits, custom scale
     (torch.bfloat16, 128, 8, 2, 6, 252, 4100, 32, 0.0),    # several key splits
 ]
 
@@ -59,7 +61,7 @@ def test_scores_match_oracle(dtype, D, Hq, Hkv, S, R, n_ctx, T, scale):
     assert torch.equal(_run_scores(st, q_tail, n_ctx, T), torch.from_numpy(got).float().cuda())   # deterministic
 
 
-@pytest.mark.parametrize("dtype,D", [(torch.float32, 64), (torch.bfloat16, 128)])
+@pytest.mark.parametrize("dtype,D", [(torch.float32, 64), (torch.bfloat16, 128), (torch.bfloat16, 64)])
 def test_scoring_a_layer_range_equals_the_whole_stack_call(dtype, D):
     """Layer by layer, in ranges and all at once: the same scores up to the rounding of another split of the keys
     (the split depends on how many layers share the launch), only the scored layers' slices are written, and

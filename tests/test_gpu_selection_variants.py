@@ -154,6 +154,7 @@ PER_ROW_CASES = [
     (torch.bfloat16, 128, 2, 2, 0, 16, 130, 64),          # T > R, no sink
     (torch.bfloat16, 128, 4, 1, 4, 252, 2500, 64),
     (torch.bfloat16, 128, 4, 1, 4, 60, 40, 40),           # covers everything
+    (torch.bfloat16, 64, 8, 2, 4, 60, 777, 64),           # head_dim 64 on the tensor-core route
 ]
 
 
