@@ -291,8 +291,8 @@ __device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem
         }
       }
     }
-    // 8-bit caches: V's scale comes in here (x 256: the kernels accumulate value / 256)
-    const float vsc = s.kv_fp8 ? s.kv_scales[2 * w.l + 1] * 256.f : 1.f;
+    // 8-bit caches: V's scale comes in here
+    const float vsc = s.kv_fp8 ? s.kv_scales[2 * w.l + 1] : 1.f;
     const float r0 = den > 0.f ? (num.x / den) * vsc : 0.f, r1 = den > 0.f ? (num.y / den) * vsc : 0.f;
     const float r2 = den > 0.f ? (num.z / den) * vsc : 0.f, r3 = den > 0.f ? (num.w / den) * vsc : 0.f;
     const long long oi = (((long long)w.l * s.batch + w.b) * s.n_q_heads + w.h * G + w.g0 + g) * D + d;

@@ -69,18 +69,32 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// Two 16 x 16 byte matrices, transposed: lane i gives the address of the 16 bytes of matrix row i (rows 0-15:
+// first matrix, 16-31: second).  Thread (g = lane / 4, c = lane % 4) receives, four bytes per register,
+// r0 = rows 4c .. 4c+3 of byte column g, r1 = the same rows of column g + 8, r2 / r3 = rows 16 + 4c .. of
+// columns g / g + 8.  With rows = keys and columns = d, a register is V^T[d][four keys]: its two halves
+// convert to the f16 pairs of an m16n8k16 A fragment (r0, r1: first 16 keys; r2, r3: second 16).
+__device__ __forceinline__ void ldmatrix_b8_x2_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
 __device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// m16n8k32, E4M3 x E4M3 -> fp32: A holds 16 rows x 32 bytes, B 32 bytes x 8 columns
-__device__ __forceinline__ void mma_e4m3(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+// The two low / two high E4M3 bytes of a word -> two f16 (exact: every E4M3 value is an f16 value).
+__device__ __forceinline__ uint32_t e4m3_lo2_to_f16x2(uint32_t w) {
+  uint32_t d;
+  asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %1;\ncvt.rn.f16x2.e4m3x2 %0, lo;\n}\n" : "=r"(d) : "r"(w));
+  return d;
+}
+__device__ __forceinline__ uint32_t e4m3_hi2_to_f16x2(uint32_t w) {
+  uint32_t d;
+  asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %1;\ncvt.rn.f16x2.e4m3x2 %0, hi;\n}\n" : "=r"(d) : "r"(w));
+  return d;
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
@@ -104,46 +118,6 @@ __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x 
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
-}
-// Two E4M3 bytes of a 32-bit word -> two f16 whose value is the E4M3 value / 256, by moving bits only:
-// an E4M3 byte s.eeee.mmm placed at bits 15..8 and shifted so that eeee.mmm lands in f16's exponent /
-// mantissa field reads as 2^(e-15) (1 + m/8) instead of 2^(e-7) (1 + m/8), subnormals included
-// (m/8 * 2^-14 instead of m/8 * 2^-6).  The factor 256 is folded into the per-layer scales.
-// SEL picks the two bytes: 0x2404 bytes (0, 2), 0x3414 bytes (1, 3).
-// two E4M3 bytes (low byte first) -> two f16 with the hardware conversion (exact: every E4M3 value is an f16 value)
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
-  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two_bytes, __NV_E4M3);
-  return (uint32_t)h.x | ((uint32_t)h.y << 16);
-}
-// two floats -> two E4M3 bytes (low byte first), round to nearest even, saturating
-__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
-  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
-}
-// Four floats x[0..3] (already divided by the head's scale) as a sum of kQTerms E4M3 values each: term t of
-// element i goes to byte i of out[t].  Every residual x - (terms so far) is exact in fp32, so after three
-// terms what is left of an element is below 2^-12 of it (or below E4M3's smallest step, 2^-9).
-constexpr int kQTerms = 3;
-__device__ __forceinline__ void split_e4m3x4(const float (&x)[4], uint32_t (&out)[kQTerms]) {
-  float r[4] = {x[0], x[1], x[2], x[3]};
-#pragma unroll
-  for (int t = 0; t < kQTerms; ++t) {
-    const uint32_t lo = f32x2_to_e4m3x2(r[0], r[1]), hi = f32x2_to_e4m3x2(r[2], r[3]);
-    out[t] = lo | (hi << 16);
-    if (t + 1 < kQTerms) {
-      const uint32_t h01 = e4m3x2_to_f16x2(lo), h23 = e4m3x2_to_f16x2(hi);
-      const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&h01));
-      const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&h23));
-      r[0] -= f01.x;
-      r[1] -= f01.y;
-      r[2] -= f23.x;
-      r[3] -= f23.y;
-    }
-  }
-}
-template <uint32_t SEL>
-__device__ __forceinline__ uint32_t e4m3_pair_to_f16x2_div256(uint32_t w) {
-  const uint32_t t = __byte_perm(w, 0u, SEL);  // first byte -> bits 15..8, second byte -> bits 31..24
-  return (t & 0x80008000u) | ((t >> 1) & 0x3f803f80u);
 }
 __device__ __forceinline__ void st_shared_u32x4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
@@ -171,20 +145,22 @@ struct TileSrc {
 // 16-byte column c of row r sits at column c ^ (r & 7).
 //
 // FP8 = true: the caches hold E4M3 bytes (rows of 128 B) with one scale per layer
-// for K and one for V.  A ring stage then holds the raw bytes of a tile (K rows,
-// then V rows, the 16-byte column c of row r at column c ^ (r & 7)) and the MMA
-// fragments are made from the bytes in registers, as f16:
+// for K and one for V.  A ring stage then holds the raw bytes of a 32-key tile (K rows,
+// then V rows); the MMA fragments are made from the bytes in registers, as f16, with one
+// conversion instruction per byte pair (this GPU's warp-level MMAs take no 8-bit floats:
+// the compiler expands them into the same conversions plus f16 MMAs, less well):
 //   K: ldmatrix on the bytes hands thread (g, c) the four bytes d = 4c .. 4c+3 of
-//      row g - an A fragment for a d order that Q's fragments simply follow;
-//   V: ldmatrix.trans on byte pairs hands it V[2c][2g], V[2c][2g+1], V[2c+1][2g],
-//      V[2c+1][2g+1]: bytes (0, 2) feed an MMA over the even d, bytes (1, 3) one
-//      over the odd d, so an accumulator tile owns d = 32 blk + 16 half + 2 g + parity.
-// K bytes become f16 with the conversion instruction (one per byte pair), V
-// bytes - whose pairs are not adjacent - with integer bit moves that yield
-// value / 256; both run on the integer pipe, which is what bounds this path.
-// Q and P are f16 as well (P as one f16 term: its 11 bits are far finer than E4M3's 4); the K scale
-// is folded into the softmax scale and the V scale (x 256) into the final
-// normalisation.  32-key tiles give every warp two independent MMA chains.
+//      row g - the halves of that register are the f16 pairs of an A fragment for a d
+//      order that Q's fragments simply follow;
+//   V: the byte-transposing ldmatrix (16 x 16 bytes, two per instruction) hands it
+//      V^T[d][four keys], again two f16 pairs of an A fragment (16 d x 16 keys); lane i
+//      addresses the key that byte i stands for, chosen as the order in which movmatrix
+//      delivers P.
+// Q and P are f16 as well (P = 256 * 2^(t - M) as one f16 term: its 11 bits are far finer
+// than E4M3's 4; O and the row sums both carry the factor 256, their ratio none).  The K
+// scale is folded into the softmax scale and the V scale into the final normalisation.
+// 16-byte column c of K row r sits at column c ^ (r & 7), of V row r at
+// c ^ (r & 7) ^ (4 * ((r >> 3) & 1)): the eight rows of either ldmatrix phase fall into eight different bank groups.
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
@@ -227,10 +203,14 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   const int k_chk = lane >> 4;
   const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8;  // V (A operand, transposed)
   const int v_chk = (lane >> 3) & 1;
+  // 8-bit V: lane i addresses the key that byte i of the transposed 16-key block stands for (bytes 4c, 4c + 1
+  // are keys 2c, 2c + 1 and bytes 4c + 2, 4c + 3 keys 2c + 8, 2c + 9: the order in which movmatrix delivers P)
+  const int v8_key = 16 * (lane >> 4) + 2 * ((lane & 15) >> 2) + (lane & 1) + 8 * ((lane >> 1) & 1);
+  const int v8_swz = (v8_key & 7) ^ ((v8_key >> 1) & 4);
 
   // d index of accumulator element (tile idx, row half) of this thread
   auto dmap = [&](int idx, int half) {
-    return FP8 ? 32 * (idx >> 1) + 16 * half + 2 * gp + (idx & 1) : idx * 16 + gp + 8 * half;
+    return idx * 16 + gp + 8 * half;
   };
   auto make_src = [&](const WorkItem& w) {
     TileSrc t;
@@ -293,16 +273,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         const bool valid = row < t.j1;
         const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
         const uint32_t soff = r * kD + ((p ^ (r & 7)) << 4);
+        const uint32_t soff_v = TILE * kD + r * kD + ((p ^ (r & 7) ^ ((r >> 1) & 4)) << 4);
         if (row == t.new_row) {
           // the new token's row is quantised on the fly from k_new / v_new
           uint32_t q4[4];
           quantize16(t.k_new_row + p * 32, a.s.kv_scales[2 * t.layer], q4);
           st_shared_u32x4(st + soff, q4[0], q4[1], q4[2], q4[3]);
           quantize16(t.v_new_row + p * 32, a.s.kv_scales[2 * t.layer + 1], q4);
-          st_shared_u32x4(st + TILE * kD + soff, q4[0], q4[1], q4[2], q4[3]);
+          st_shared_u32x4(st + soff_v, q4[0], q4[1], q4[2], q4[3]);
         } else {
           cp_async16(st + soff, t.Kb + goff, valid ? 16 : 0);
-          cp_async16(st + TILE * kD + soff, t.Vb + goff, valid ? 16 : 0);
+          cp_async16(st + soff_v, t.Vb + goff, valid ? 16 : 0);
         }
       }
     } else {
@@ -361,8 +342,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     // per-layer scales of 8-bit caches: K's goes into the softmax scale, V's into the normalisation
     float cs_l = a.cs, v_scale = 1.f;
     if constexpr (FP8) {
-      cs_l = a.cs * a.s.kv_scales[2 * l];  // K fragments hold the true values  // 256: the expanded tile holds value / 256
-      v_scale = a.s.kv_scales[2 * l + 1] * 256.f;
+      cs_l = a.cs * a.s.kv_scales[2 * l];
+      v_scale = a.s.kv_scales[2 * l + 1];
     }
 
     // fused append: store the new token's row into the cache
@@ -387,49 +368,40 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       }
     }
 
-    // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8)
-    uint32_t qf[FP8 ? 1 : NK][2];
-    // 8-bit caches: the stored K bytes are the A operand of E4M3 MMAs as they are, and q is their B operand as
-    // a sum of kQTerms E4M3 terms at one power-of-two scale per head (block blk covers d = 32 blk .. 32 blk + 31:
-    // bytes 4c .. 4c+3 in b0, 16 + 4c .. in b1).
-    uint32_t q8[FP8 ? kQTerms : 1][4][2];
+    // Q fragments (B operand of S^T = K Q^T): head gp, d = 16*ks + 2c (+8).
+    // 8-bit caches: K's bytes reach the MMA as f16 in the d order the byte ldmatrix delivers (k-step ks covers
+    // d = 16 ks .. 16 ks + 15, this thread's four are 16 ks + 4c .. 4c+3), and q follows as f16 at one
+    // power-of-two scale per head (bf16 -> f16 is exact inside f16's range, which the scale centres).
+    uint32_t qf[NK][2];
     float q_scale0 = 1.f, q_scale1 = 1.f;  // scale of heads 2c and 2c + 1 (this thread's S columns)
     {
       const __nv_bfloat16* qp =
           (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + w.g0 + gp) * kD;
       if constexpr (FP8) {
-        float x[4][2][4];
+        float x[NK][4];
         float amax = 0.f;
 #pragma unroll
-        for (int blk = 0; blk < 4; ++blk)
+        for (int ks = 0; ks < NK; ++ks) {
+          uint2 q4 = make_uint2(0u, 0u);
+          if (gp < Gn) q4 = *reinterpret_cast<const uint2*>(qp + 16 * ks + 4 * c);
+          x[ks][0] = bf16_lo(q4.x);
+          x[ks][1] = bf16_hi(q4.x);
+          x[ks][2] = bf16_lo(q4.y);
+          x[ks][3] = bf16_hi(q4.y);
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            uint2 q4 = make_uint2(0u, 0u);
-            if (gp < Gn) q4 = *reinterpret_cast<const uint2*>(qp + 32 * blk + 16 * hf + 4 * c);
-            x[blk][hf][0] = bf16_lo(q4.x);
-            x[blk][hf][1] = bf16_hi(q4.x);
-            x[blk][hf][2] = bf16_lo(q4.y);
-            x[blk][hf][3] = bf16_hi(q4.y);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fabsf(x[blk][hf][e]));
-          }
+          for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fabsf(x[ks][e]));
+        }
         amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
         amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));  // the four lanes of a head hold its 128 values
-        // power-of-two scale that puts the head's largest |q| into [128, 256): inside E4M3's range (448)
-        const int e2 = (amax > 0.f && amax < INFINITY) ? ilogbf(amax) - 7 : 0;
+        // power-of-two scale that puts the head's largest |q| into [1, 2): products with |K| <= 448 stay far
+        // inside f16's range and values down to 2^-14 of the largest keep all their bits
+        const int e2 = (amax > 0.f && amax < INFINITY) ? ilogbf(amax) : 0;
         const float inv = exp2f((float)-e2), scale = exp2f((float)e2);
 #pragma unroll
-        for (int blk = 0; blk < 4; ++blk)
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            float y[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) y[e] = x[blk][hf][e] * inv;
-            uint32_t terms[kQTerms];
-            split_e4m3x4(y, terms);
-#pragma unroll
-            for (int t = 0; t < kQTerms; ++t) q8[t][blk][hf] = terms[t];
-          }
+        for (int ks = 0; ks < NK; ++ks) {
+          qf[ks][0] = pack_f16(x[ks][0] * inv, x[ks][1] * inv);
+          qf[ks][1] = pack_f16(x[ks][2] * inv, x[ks][3] * inv);
+        }
         q_scale0 = __shfl_sync(0xffffffffu, scale, (2 * c) * 4);
         q_scale1 = __shfl_sync(0xffffffffu, scale, (2 * c + 1) * 4);
       } else {
@@ -471,15 +443,23 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         sc[mt][0] = sc[mt][1] = sc[mt][2] = sc[mt][3] = 0.f;
         const int row = mt * 16 + k_row;
         if constexpr (FP8) {
+          float sc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int blk = 0; blk < 4; ++blk) {  // 32 d per ldmatrix: matrices (rows 0-7 | 8-15) x (chunk 2 blk | 2 blk + 1)
             uint32_t m[4];
             const int chunk = 2 * blk + k_chk;
             ldmatrix_x4(m, st + row * kD + ((chunk ^ (row & 7)) << 4));
-            // the bytes are the A fragment as they are: rows g | g + 8, bytes 4c .. | 16 + 4c ..
-#pragma unroll
-            for (int t = 0; t < kQTerms; ++t) mma_e4m3(sc[mt], m, q8[t][blk][0], q8[t][blk][1]);
+            // a register holds bytes d = 4c .. 4c+3 of row g (m0, m2) or g + 8 (m1, m3): its halves are the
+            // f16 pairs of the A fragment, contraction index 2c + j <-> d 4c + j, 2c + 8 + j <-> d 4c + 2 + j
+            const uint32_t a0[4] = {e4m3_lo2_to_f16x2(m[0]), e4m3_lo2_to_f16x2(m[1]), e4m3_hi2_to_f16x2(m[0]),
+                                    e4m3_hi2_to_f16x2(m[1])};
+            const uint32_t a1[4] = {e4m3_lo2_to_f16x2(m[2]), e4m3_lo2_to_f16x2(m[3]), e4m3_hi2_to_f16x2(m[2]),
+                                    e4m3_hi2_to_f16x2(m[3])};
+            mma_f16(sc[mt], a0, qf[2 * blk][0], qf[2 * blk][1]);
+            mma_f16(sc2, a1, qf[2 * blk + 1][0], qf[2 * blk + 1][1]);
           }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) sc[mt][i] += sc2[i];
         } else {
           // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
           float sc2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -527,40 +507,44 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         o[i][3] *= corr1;
       }
       // ---- P = 2^(t - M), O^T += V^T P ---------------------------------------
+      if constexpr (FP8) {
+        static_assert(!FP8 || MT == 2, "one byte-transposing ldmatrix spans the 32 keys of a tile");
+        const float Ms0 = Mn0 - 8.f, Ms1 = Mn1 - 8.f;  // P (and with it O and the row sums) carries the factor 256:
+        uint32_t bh[MT][2];                            // small probabilities stay normal numbers in f16
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        const float p0 = ex2(sc[mt][0] - Mn0), p1 = ex2(sc[mt][1] - Mn1);
-        const float p2 = ex2(sc[mt][2] - Mn0), p3 = ex2(sc[mt][3] - Mn1);
-        l0 += p0 + p2;
-        l1 += p1 + p3;
-        // P for the B operand: one f16 term with 8-bit caches, a bf16 head and a bf16 residual otherwise
-        const uint32_t hi01 = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
-        const uint32_t hi23 = FP8 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
-        const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
-        uint32_t bl0 = 0u, bl1 = 0u;
-        if constexpr (!FP8) {
-          bl0 = movmatrix_trans(pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01)));
-          bl1 = movmatrix_trans(pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23)));
+        for (int mt = 0; mt < MT; ++mt) {
+          const float p0 = ex2(sc[mt][0] - Ms0), p1 = ex2(sc[mt][1] - Ms1);
+          const float p2 = ex2(sc[mt][2] - Ms0), p3 = ex2(sc[mt][3] - Ms1);
+          l0 += p0 + p2;
+          l1 += p1 + p3;
+          // thread (g, c) gets head g, keys 2c, 2c + 1 (bh[.][0]) and 2c + 8, 2c + 9 (bh[.][1]) of this 16-key block
+          bh[mt][0] = movmatrix_trans(pack_f16(p0, p1));
+          bh[mt][1] = movmatrix_trans(pack_f16(p2, p3));
         }
-        if constexpr (FP8) {
-          const int row = mt * 16 + k_row;  // same matrix order as K: (keys 0-7 | 8-15) x (chunk 2 blk | 2 blk + 1)
 #pragma unroll
-          for (int blk = 0; blk < 4; ++blk) {
-            uint32_t m[4];
-            const int chunk = 2 * blk + k_chk;
-            ldmatrix_x4_trans(m, st + TILE * kD + row * kD + ((chunk ^ (row & 7)) << 4));
-            {  // even d: rows g <-> d = 32 blk + 2g (m0, m1), rows g + 8 <-> d = 32 blk + 16 + 2g (m2, m3)
-              const uint32_t af[4] = {e4m3_pair_to_f16x2_div256<0x2404>(m[0]), e4m3_pair_to_f16x2_div256<0x2404>(m[2]),
-                                      e4m3_pair_to_f16x2_div256<0x2404>(m[1]), e4m3_pair_to_f16x2_div256<0x2404>(m[3])};
-              mma_f16(o[2 * blk], af, bh0, bh1);
-            }
-            {  // odd d
-              const uint32_t af[4] = {e4m3_pair_to_f16x2_div256<0x3414>(m[0]), e4m3_pair_to_f16x2_div256<0x3414>(m[2]),
-                                      e4m3_pair_to_f16x2_div256<0x3414>(m[1]), e4m3_pair_to_f16x2_div256<0x3414>(m[3])};
-              mma_f16(o[2 * blk + 1], af, bh0, bh1);
-            }
-          }
-        } else {
+        for (int db = 0; db < NK; ++db) {  // 16 d per instruction = one 16-byte column of the V rows
+          uint32_t r[4];
+          ldmatrix_b8_x2_trans(r, st + TILE * kD + v8_key * kD + ((db ^ v8_swz) << 4));
+          const uint32_t a0[4] = {e4m3_lo2_to_f16x2(r[0]), e4m3_lo2_to_f16x2(r[1]), e4m3_hi2_to_f16x2(r[0]),
+                                  e4m3_hi2_to_f16x2(r[1])};
+          const uint32_t a1[4] = {e4m3_lo2_to_f16x2(r[2]), e4m3_lo2_to_f16x2(r[3]), e4m3_hi2_to_f16x2(r[2]),
+                                  e4m3_hi2_to_f16x2(r[3])};
+          mma_f16(o[db], a0, bh[0][0], bh[0][1]);
+          mma_f16(o[db], a1, bh[1][0], bh[1][1]);
+        }
+      } else {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const float p0 = ex2(sc[mt][0] - Mn0), p1 = ex2(sc[mt][1] - Mn1);
+          const float p2 = ex2(sc[mt][2] - Mn0), p3 = ex2(sc[mt][3] - Mn1);
+          l0 += p0 + p2;
+          l1 += p1 + p3;
+          // P for the B operand: a bf16 head and a bf16 residual
+          const uint32_t hi01 = pack_bf16(p0, p1);
+          const uint32_t hi23 = pack_bf16(p2, p3);
+          const uint32_t bh0 = movmatrix_trans(hi01), bh1 = movmatrix_trans(hi23);
+          const uint32_t bl0 = movmatrix_trans(pack_bf16(p0 - bf16_lo(hi01), p1 - bf16_hi(hi01)));
+          const uint32_t bl1 = movmatrix_trans(pack_bf16(p2 - bf16_lo(hi23), p3 - bf16_hi(hi23)));
           const int row = mt * 16 + v_row;
 #pragma unroll
           for (int dt = 0; dt < NK; ++dt) {
