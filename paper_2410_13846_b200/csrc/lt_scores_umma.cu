@@ -88,6 +88,7 @@ constexpr int kTmemCols = 512;   // two accumulators of 256 columns, one per row
 constexpr int kChunk = 32;       // columns per tcgen05.ld
 constexpr int kPolyOf8 = LT_SCORES_POLY_OF8;
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 1.9 GHz
+constexpr uint32_t kSuspendHintNs = 1000000u;    // a waiting thread may stay suspended this long before try_wait returns
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
@@ -103,10 +104,10 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok;
 }
@@ -125,12 +126,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (true) {
+  for (uint32_t polls = 1;; ++polls) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      *abort_flag = 1;
-      return false;
+    if ((polls & 15u) == 0u) {  // the flag and the clock are looked at every 16th poll: a poll stays four instructions
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
     }
   }
 }
@@ -576,18 +579,22 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int lim = min(vis, k1 - 1);     // last key of this piece that the row may see
       float Mr = -INFINITY, sA = 0.f, sWn = 0.f;  // reference exponent (an integer), sum, windowed sum
 
+      // statistics of one chunk whose 32 keys all count, inside the window (in_win) or all outside it
+      auto plain_stats = [&](uint32_t (&v)[kChunk], bool in_win) {
+        const float Mn = fmaxf(Mr, ceilf(max32(v) * cs));
+        const float corr = ex2(Mr - Mn);
+        const float ps = sum_ex2_32_mixed(v, cs, Mn);
+        sA = fmaf(sA, corr, ps);
+        sWn = fmaf(sWn, corr, in_win ? ps : 0.f);
+        Mr = Mn;
+      };
       // statistics of one chunk (32 keys from jb) already in registers
       auto chunk_stats = [&](uint32_t (&v)[kChunk], int jb) {
         const int jend = jb + kChunk;
         const bool all_win = (jend <= S) || (jb >= win_lo);
         const bool no_win = (jb >= S) && (jend <= win_lo);
         if ((jb >= k0) && (jend - 1 <= lim) && (all_win || no_win)) {
-          const float Mn = fmaxf(Mr, ceilf(max32(v) * cs));
-          const float corr = ex2(Mr - Mn);
-          const float ps = sum_ex2_32_mixed(v, cs, Mn);
-          sA = fmaf(sA, corr, ps);
-          sWn = fmaf(sWn, corr, all_win ? ps : 0.f);
-          Mr = Mn;
+          plain_stats(v, all_win);
         } else if (max(jb, k0) <= min(jend - 1, lim)) {
           // boundary chunk (piece start, causal tail, piece end or window edge): mask in place.
           // 2^(-inf) = 0, and at least one key is visible, so the maximum is finite.
@@ -623,16 +630,35 @@ __global__ void __launch_bounds__(kThreads, 1)
         // Four chunks of 32 columns through one register buffer: the load of a chunk is not overlapped
         // by this warp's own arithmetic but by the three other statistics warps of its scheduler (two
         // buffers would not fit the 96 registers a thread gets).
+        // Most tiles lie inside the piece, before every row's last visible key and on one side of the window's
+        // edges for all 32 rows of the warp: their chunks need no per-chunk tests.
+        const int kend = kb + 128;
+        const bool span_in = (kend <= S) || (kb >= win_lo);
+        const bool span_out = (kb >= S) && (kend <= win_lo);
+        const bool plain = __all_sync(0xffffffffu, (kb >= k0) && (kend - 1 <= lim) && (span_in || span_out));
+        if (plain) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          tmem_ld32(lane_addr + c * kChunk, va);
-          tmem_ld_wait();
-          if (c == 3) {
-            // the row's last chunk is in registers: the accumulator may be overwritten
-            tc_fence_before();
-            mbar_arrive(bar_sempty + 8 * mb);
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(lane_addr + c * kChunk, va);
+            tmem_ld_wait();
+            if (c == 3) {
+              tc_fence_before();
+              mbar_arrive(bar_sempty + 8 * mb);
+            }
+            plain_stats(va, span_in);
           }
-          chunk_stats(va, kb + c * kChunk);
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(lane_addr + c * kChunk, va);
+            tmem_ld_wait();
+            if (c == 3) {
+              // the row's last chunk is in registers: the accumulator may be overwritten
+              tc_fence_before();
+              mbar_arrive(bar_sempty + 8 * mb);
+            }
+            chunk_stats(va, kb + c * kChunk);
+          }
         }
       }
       if (!ok) break;
