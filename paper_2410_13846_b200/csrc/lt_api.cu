@@ -58,7 +58,7 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   if (cap > (int64_t)0x7fffffff) cap = 0x7fffffff;
   p.items_cap = (int)cap;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const int gp = decode_mma_supported(s) && G > 8 ? 8 : G;  // heads per partial slot
+  const int gp = G;  // heads per partial slot
   p.ml_floats = (size_t)cap * gp * 2;
   p.o_floats = (size_t)cap * gp * s.head_dim;
   return p;
@@ -475,9 +475,7 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.layer_count = layer_count;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
   a.hsub = decode_head_subgroups(*shape);
-  a.gp_stride = (decode_mma_supported(*shape) && shape->n_q_heads / shape->n_kv_heads > 8)
-                    ? 8
-                    : shape->n_q_heads / shape->n_kv_heads;
+  a.gp_stride = shape->n_q_heads / shape->n_kv_heads;
   a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads * a.hsub;
   a.work_counter = a.done_counter + 1;
   a.part_ml = reinterpret_cast<float*>((char*)ws + prefix);

@@ -134,7 +134,7 @@ struct TileSrc {
   const uint8_t* v_new_row;
   int j0, j1;                // key rows of the chunk
   int new_row;               // -1 when the chunk does not hold the new token
-  int my_tiles;              // tiles of this warp (tiles warp, warp + WARPS, ... of the chunk)
+  int my_tiles;              // tiles of this warp's stream (tiles stream, stream + STREAMS, ... of the chunk)
   int tbl_off;               // paged full cache: offset of this batch row's block-table row, else -1
   int layer;                 // for the per-layer scales of 8-bit caches
 };
@@ -161,11 +161,19 @@ struct TileSrc {
 // scale is folded into the softmax scale and the V scale into the final normalisation.
 // 16-byte column c of K row r sits at column c ^ (r & 7), of V row r at
 // c ^ (r & 7) ^ (4 * ((r >> 3) & 1)): the eight rows of either ldmatrix phase fall into eight different bank groups.
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
+//
+// PAIR = true (query groups of 9..16 heads): the four warps work as two pairs.  The warps of a pair walk the same
+// tiles through one shared ring (each copies half of every tile, a 64-thread named barrier per tile makes the
+// copies visible and frees the stage that is refilled), warp 0 of the pair serves heads 0-7 of the group and warp
+// 1 heads 8-15, so the chunk still crosses HBM, L2 and shared memory once.
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, bool PAIR>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
   static_assert(DH == 128 || (DH == 64 && !FP8), "head_dim 128, or 64 with 16-bit caches");
+  static_assert(!(PAIR && FP8), "warp pairs are written for the 16-bit caches");
+  constexpr int STREAMS = PAIR ? WARPS / 2 : WARPS;   // independent tile streams of the CTA
+  constexpr int RSTAGES = NSTAGE;                     // ring stages of a stream
   constexpr int kD = DH;                       // head_dim
   constexpr int kSrcRowBytes = kD * 2;         // one row of q, k_new, v_new (bf16)
   constexpr int NK = kD / 16;                  // 16-wide k-steps of S = K Q^T = 16-row tiles of O^T
@@ -177,8 +185,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   constexpr int kRowBytes = FP8 ? kD : 2 * kD;             // one cached K or V row
   constexpr int RAW_BYTES = 2 * TILE * kD;                 // FP8: K rows + V rows of a tile as stored
   constexpr int RING_STAGE = FP8 ? RAW_BYTES : STAGE_BYTES;  // what one ring stage holds
-  constexpr int WARP_BYTES = NSTAGE * RING_STAGE;
-  constexpr int RING_BYTES = WARPS * WARP_BYTES;
+  constexpr int STREAM_BYTES = RSTAGES * RING_STAGE;
+  constexpr int RING_BYTES = STREAMS * STREAM_BYTES;
   constexpr int MERGE_BYTES = 2 * 8 * kD * 4 + 2 * WARPS * 8 * 4;
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ int s_flag, s_next;
@@ -197,7 +205,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
-  const uint32_t wsm = smem_u32(smem) + warp * WARP_BYTES;
+  const int stream = PAIR ? warp >> 1 : warp;  // tile stream of this warp
+  const int role = PAIR ? warp & 1 : 0;        // pair: which eight heads of the group this warp serves
+  const uint32_t wsm = smem_u32(smem) + stream * STREAM_BYTES;
+  auto stream_sync = [&]() {  // the threads that share a ring: the warp, or the 64 threads of a pair
+    if constexpr (PAIR) {
+      if (stream == 0) asm volatile("bar.sync 1, 64;\n" ::: "memory");
+      else asm volatile("bar.sync 2, 64;\n" ::: "memory");
+    } else {
+      __syncwarp();
+    }
+  };
   // lane-constant parts of the ldmatrix addresses
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8;  // K (A operand, not transposed)
   const int k_chk = lane >> 4;
@@ -233,7 +251,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       t.v_new_row = (const uint8_t*)a.v_new + src;
     }
     const int n_tiles = (w.j1 - w.j0 + TILE - 1) / TILE;
-    t.my_tiles = (n_tiles > warp) ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
+    t.my_tiles = (n_tiles > stream) ? (n_tiles - stream + STREAMS - 1) / STREAMS : 0;
     return t;
   };
   // copy this warp's idx-th tile of `t` into ring stage `stage` (no commit)
@@ -259,11 +277,37 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       out[i] = packed;
     }
   };
+  // Lane-constant parts of a tile copy.  One pass of the warp covers RPI rows; this lane's first row is f_row,
+  // its later rows f_row + dr with dr a multiple of RPI, so that (row & 7) = (f_row & 7) ^ (dr & 7): the swizzled
+  // offset of every pass is the first one xor a constant.
+  constexpr int VPRX = FP8 ? 8 : VPR;             // 16-byte vectors of a cached row
+  constexpr int RPI = 32 / VPRX;
+  constexpr int FROWS = PAIR ? TILE / 2 : TILE;   // rows of a tile this warp copies (a pair's warps: half each)
+  const int f_row = role * FROWS + lane / VPRX;
+  const int f_p = lane % VPRX;
+  const uint32_t f_goff = f_row * kRowBytes + f_p * 16;
+  const uint32_t f_soff = FP8 ? f_row * kD + ((f_p ^ (f_row & 7)) << 4)
+                              : (f_p >> 3) * HALF_BYTES + f_row * 128 + (((f_p & 7) ^ (f_row & 7)) << 4);
+  const uint32_t f_soff_v = FP8 ? TILE * kD + f_row * kD + ((f_p ^ (f_row & 7) ^ ((f_row >> 1) & 4)) << 4)
+                                : HALVES * HALF_BYTES + f_soff;
   auto fetch_tile = [&](const TileSrc& t, int idx, int stage) {
-    const int key_base = t.j0 + (warp + idx * WARPS) * TILE;
+    const int key_base = t.j0 + (stream + idx * STREAMS) * TILE;
     const long long tile_row = cache_row(t, key_base);
     const uint32_t st = wsm + stage * RING_STAGE;
-    if constexpr (FP8) {
+    if (key_base + TILE <= t.j1 && (t.new_row < key_base || t.new_row >= key_base + TILE)) {
+      // every row of the tile is a cached row (the usual case): addresses are a base plus constants
+      const uint8_t* kp = t.Kb + tile_row * kRowBytes + f_goff;
+      const uint8_t* vp = t.Vb + tile_row * kRowBytes + f_goff;
+#pragma unroll
+      for (int i = 0; i < FROWS / RPI; ++i) {
+        constexpr int kSRow = FP8 ? kD : 128;  // bytes between rows in a stage
+        const int dr = RPI * i;
+        const uint32_t x = (uint32_t)(dr & 7) << 4;
+        const uint32_t xv = FP8 ? (uint32_t)((dr & 7) ^ ((dr >> 1) & 4)) << 4 : x;
+        cp_async16(st + ((f_soff ^ x) + dr * kSRow), kp + (long long)dr * kRowBytes, 16);
+        cp_async16(st + ((f_soff_v ^ xv) + dr * kSRow), vp + (long long)dr * kRowBytes, 16);
+      }
+    } else if constexpr (FP8) {
       // raw rows: 8 chunks of 16 bytes per row, K rows then V rows
 #pragma unroll
       for (int i = 0; i < TILE / 4; ++i) {
@@ -287,9 +331,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         }
       }
     } else {
+      constexpr int ROWS = PAIR ? TILE / 2 : TILE;  // a pair's warps copy half a tile each
 #pragma unroll
-      for (int i = 0; i < TILE * VPR / 32; ++i) {
-        const int r = (32 / VPR) * i + lane / VPR;
+      for (int i = 0; i < ROWS * VPR / 32; ++i) {
+        const int r = role * ROWS + (32 / VPR) * i + lane / VPR;
         const int p = lane % VPR;
         const int row = key_base + r;
         const bool valid = row < t.j1;
@@ -324,7 +369,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       la_in_next = 1;
       la_idx = 0;
     }
-    const int stage = issued % NSTAGE;
+    const int stage = issued % RSTAGES;
     if (la_in_next == 0) fetch_tile(src_cur, la_idx, stage);
     else if (la_idx < src_nxt.my_tiles) fetch_tile(src_nxt, la_idx, stage);
     ++la_idx;
@@ -334,7 +379,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   while (cur < n_items) {
     const int l = w.l, b = w.b, h = w.h;
-    const int Gn = w.gn;  // query heads served by this item (the group, or one sub-group of at most 8)
+    // query heads served by this warp: the item's (the group, or one sub-group of at most 8), or this warp's
+    // eight of a pair's sixteen
+    const int g0 = PAIR ? role * 8 : w.g0;
+    const int Gn = PAIR ? min(8, G - role * 8) : w.gn;
     const int j1 = src_cur.j1;
     int fetched_next = 0;
     if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
@@ -376,7 +424,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     float q_scale0 = 1.f, q_scale1 = 1.f;  // scale of heads 2c and 2c + 1 (this thread's S columns)
     {
       const __nv_bfloat16* qp =
-          (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + w.g0 + gp) * kD;
+          (const __nv_bfloat16*)a.q + (((long long)l * s.batch + b) * s.n_q_heads + h * G + g0 + gp) * kD;
       if constexpr (FP8) {
         float x[NK][4];
         float amax = 0.f;
@@ -426,15 +474,23 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
     float M0 = -INFINITY, M1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2c and 2c+1
 
-    while (issued - consumed < NSTAGE - 1) issue_slot();
+    while (issued - consumed < RSTAGES - 1) issue_slot();
     for (int it = 0; it < src_cur.my_tiles; ++it) {
-      __syncwarp();              // every lane is done reading the stage that is refilled next
-      issue_slot();
-      cp_async_wait<NSTAGE - 1>();
-      __syncwarp();              // all lanes' copies of this tile have landed
-      const uint32_t st = wsm + (consumed % NSTAGE) * RING_STAGE;
+      if constexpr (PAIR) {
+        // one barrier per tile: behind it both warps' copies of this tile have landed and both are done with the
+        // previous tile, whose stage the next slot refills
+        cp_async_wait<RSTAGES - 2>();
+        stream_sync();
+        issue_slot();
+      } else {
+        __syncwarp();              // every lane is done reading the stage that is refilled next
+        issue_slot();
+        cp_async_wait<NSTAGE - 1>();
+        __syncwarp();              // all lanes' copies of this tile have landed
+      }
+      const uint32_t st = wsm + (consumed % RSTAGES) * RING_STAGE;
       ++consumed;
-      const int key_base = src_cur.j0 + (warp + it * WARPS) * TILE;
+      const int key_base = src_cur.j0 + (stream + it * STREAMS) * TILE;
 
       // ---- S^T = K Q^T ------------------------------------------------------
       float sc[MT][4];
@@ -497,14 +553,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       const float corr0 = ex2(M0 - Mn0), corr1 = ex2(M1 - Mn1);
       M0 = Mn0;
       M1 = Mn1;
-      l0 *= corr0;
-      l1 *= corr1;
+      // once the running maxima have settled the factors are exactly 1 for every lane: skip the rescale then
+      if (__any_sync(0xffffffffu, (corr0 != 1.f) | (corr1 != 1.f))) {
+        l0 *= corr0;
+        l1 *= corr1;
 #pragma unroll
-      for (int i = 0; i < NK; ++i) {
-        o[i][0] *= corr0;
-        o[i][1] *= corr1;
-        o[i][2] *= corr0;
-        o[i][3] *= corr1;
+        for (int i = 0; i < NK; ++i) {
+          o[i][0] *= corr0;
+          o[i][1] *= corr1;
+          o[i][2] *= corr0;
+          o[i][3] *= corr1;
+        }
       }
       // ---- P = 2^(t - M), O^T += V^T P ---------------------------------------
       if constexpr (FP8) {
@@ -578,19 +637,23 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     if (threadIdx.x == 0) s_next = fetched_next;
     __syncthreads();  // (max, sum) of every warp and the next item index are visible
     const int after_next = s_next;
+    // the warps whose results belong to the same heads: all four, or (pairs) the two of this warp's role
+    constexpr int W0_STEP = PAIR ? 2 : 1;
+    const int w_first = PAIR ? role : 0;
     float Mx0 = -INFINITY, Mx1 = -INFINITY;
 #pragma unroll
-    for (int ww = 0; ww < WARPS; ++ww) {
+    for (int ww = w_first; ww < WARPS; ww += W0_STEP) {
       Mx0 = fmaxf(Mx0, sm_m[ww * 8 + 2 * c]);
       Mx1 = fmaxf(Mx1, sm_m[ww * 8 + 2 * c + 1]);
     }
     float ls0 = 0.f, ls1 = 0.f;
     if (Mx0 > -INFINITY)
 #pragma unroll
-      for (int ww = 0; ww < WARPS; ++ww) ls0 += exp2f(sm_m[ww * 8 + 2 * c] - Mx0) * sm_l[ww * 8 + 2 * c];
+      for (int ww = w_first; ww < WARPS; ww += W0_STEP) ls0 += exp2f(sm_m[ww * 8 + 2 * c] - Mx0) * sm_l[ww * 8 + 2 * c];
     if (Mx1 > -INFINITY)
 #pragma unroll
-      for (int ww = 0; ww < WARPS; ++ww) ls1 += exp2f(sm_m[ww * 8 + 2 * c + 1] - Mx1) * sm_l[ww * 8 + 2 * c + 1];
+      for (int ww = w_first; ww < WARPS; ww += W0_STEP)
+        ls1 += exp2f(sm_m[ww * 8 + 2 * c + 1] - Mx1) * sm_l[ww * 8 + 2 * c + 1];
     {
       const float f0 = Mx0 > -INFINITY ? exp2f(M0 - Mx0) : 0.f;
       const float f1 = Mx1 > -INFINITY ? exp2f(M1 - Mx1) : 0.f;
@@ -625,31 +688,36 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         o[dt][3] += p[kD + dmap(dt, 1)];
       }
     }
-    __syncthreads();  // buffer 0 has been read by warp 0 before warp 1 overwrites it
-    if (warp == 1) {
+    if constexpr (!PAIR) {
+      __syncthreads();  // buffer 0 has been read by warp 0 before warp 1 overwrites it
+      if (warp == 1) {
 #pragma unroll
-      for (int dt = 0; dt < NK; ++dt) {
-        float* p = buf_at(0, dt);
-        p[dmap(dt, 0)] = o[dt][0];
-        p[kD + dmap(dt, 0)] = o[dt][1];
-        p[dmap(dt, 1)] = o[dt][2];
-        p[kD + dmap(dt, 1)] = o[dt][3];
+        for (int dt = 0; dt < NK; ++dt) {
+          float* p = buf_at(0, dt);
+          p[dmap(dt, 0)] = o[dt][0];
+          p[kD + dmap(dt, 0)] = o[dt][1];
+          p[dmap(dt, 1)] = o[dt][2];
+          p[kD + dmap(dt, 1)] = o[dt][3];
+        }
       }
+      __syncthreads();
     }
-    __syncthreads();
     const bool single = w.nc <= 1;  // the whole (layer, b, kv head) is this one chunk
-    if (warp == 0) {
+    // the warp that holds the item's sum: warp 0, or (pairs) warps 0 and 1 with eight heads each
+    if (PAIR ? warp < 2 : warp == 0) {
+      if constexpr (!PAIR) {
 #pragma unroll
-      for (int dt = 0; dt < NK; ++dt) {
-        const float* p = buf_at(0, dt);
-        o[dt][0] += p[dmap(dt, 0)];
-        o[dt][1] += p[kD + dmap(dt, 0)];
-        o[dt][2] += p[dmap(dt, 1)];
-        o[dt][3] += p[kD + dmap(dt, 1)];
+        for (int dt = 0; dt < NK; ++dt) {
+          const float* p = buf_at(0, dt);
+          o[dt][0] += p[dmap(dt, 0)];
+          o[dt][1] += p[kD + dmap(dt, 0)];
+          o[dt][2] += p[dmap(dt, 1)];
+          o[dt][3] += p[kD + dmap(dt, 1)];
+        }
       }
       if (single) {
         // no partials: normalise and write the output of heads 2c, 2c + 1 directly
-        const long long ob = (((long long)l * s.batch + b) * s.n_q_heads + h * G + w.g0) * kD;
+        const long long ob = (((long long)l * s.batch + b) * s.n_q_heads + h * G + g0) * kD;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
@@ -674,15 +742,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
           if (g < Gn) {
-            float* po = a.part_o + (unit * a.gp_stride + g) * kD;
+            const long long pslot = unit * a.gp_stride + (PAIR ? g0 : 0) + g;  // the slot's heads in group order
+            float* po = a.part_o + pslot * kD;
 #pragma unroll
             for (int dt = 0; dt < NK; ++dt) {
               po[dmap(dt, 0)] = o[dt][e];
               po[dmap(dt, 1)] = o[dt][e + 2];
             }
             if (gp == 0) {
-              a.part_ml[(unit * a.gp_stride + g) * 2] = e ? Mx1 : Mx0;
-              a.part_ml[(unit * a.gp_stride + g) * 2 + 1] = e ? ls1 : ls0;
+              a.part_ml[pslot * 2] = e ? Mx1 : Mx0;
+              a.part_ml[pslot * 2 + 1] = e ? ls1 : ls0;
             }
           }
         }
@@ -714,14 +783,15 @@ bool decode_mma_supported(const lt_shape& s) {
          (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 8 : 16);
 }
 
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH>
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, bool PAIR>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int ring = FP8 ? WARPS * NSTAGE * TILE * 256 : WARPS * NSTAGE * TILE * 4 * DH;
+  constexpr int streams = PAIR ? WARPS / 2 : WARPS;
+  constexpr int ring = FP8 ? streams * NSTAGE * TILE * 256 : streams * NSTAGE * TILE * 4 * DH;
   constexpr int merge = 2 * 8 * DH * 4 + 2 * WARPS * 8 * 4;
   static_assert(2 * 8 * DH * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
-  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8, DH>;
+  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8, DH, PAIR>;
   // Per device, behind a lock (host threads may issue their first calls concurrently): the dynamic
   // shared-memory limit is raised once to the largest size any launch of this variant can ask for, and
   // the occupancy of each shared-memory size met so far is remembered (host time matters for per-layer callers).
@@ -762,10 +832,14 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
   // 8-bit caches: three raw stages of 32 keys (8 KB) = the 24 KB per warp of the 16-bit ring
-  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true, 128>(a, kf, vf, ks, vs, st);
+  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true, 128, false>(a, kf, vf, ks, vs, st);
+  const bool pair = a.s.n_q_heads / a.s.n_kv_heads > 8;  // groups of 9..16: two warps per tile, eight heads each
   // head_dim 64: rows are half as long, so 32-key tiles keep the bytes in flight per warp (24 KB) the same
-  if (a.s.head_dim == 64) return launch_variant<32, 3, 4, 2, false, 64>(a, kf, vf, ks, vs, st);
-  return launch_variant<16, 3, 4, 2, false, 128>(a, kf, vf, ks, vs, st);
+  if (a.s.head_dim == 64)
+    return pair ? launch_variant<32, 6, 4, 2, false, 64, true>(a, kf, vf, ks, vs, st)
+                : launch_variant<32, 3, 4, 2, false, 64, false>(a, kf, vf, ks, vs, st);
+  return pair ? launch_variant<32, 3, 4, 2, false, 128, true>(a, kf, vf, ks, vs, st)
+              : launch_variant<16, 3, 4, 2, false, 128, false>(a, kf, vf, ks, vs, st);
 }
 
 }  // namespace lt

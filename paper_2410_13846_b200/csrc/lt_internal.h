@@ -149,8 +149,8 @@ cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, con
 bool decode_mma_supported(const lt_shape& s);
 // Sub-groups of at most 8 query heads that a kv head's group is served in (1 unless the tensor-core path has a group above 8).
 inline int decode_head_subgroups(const lt_shape& s) {
-  const int G = s.n_q_heads / s.n_kv_heads;
-  return (decode_mma_supported(s) && G > 8) ? (G + 7) / 8 : 1;
+  (void)s;
+  return 1;
 }
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                               const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
