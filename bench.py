@@ -553,8 +553,7 @@ def run_variants(wl, mask_hybrid):
     res["head_dim_64"]["lazy_scores_ms"] = ms
     res["head_dim_64"]["lazy_scores_tflops"] = 2.0 * L * B * Hq * T * cfg.n_ctx * 64 / (ms * 1e-3) / 1e12
     del k64, v64, ks64, vs64, ws64, wsS, qt64, tables64
-    # (d) a query group of 16 (32 q / 2 kv heads): the kernel serves it as two sub-groups of 8 heads, i.e. two work
-    # items per chunk; algorithmic bytes count every cached byte once
+    # (d) a query group of 16 (32 q / 2 kv heads): two warps share every tile and serve eight heads each
     cfg16 = cfg.scaled(n_kv_heads=2)
     shape16 = lt.Shape(L, B, Hq, 2, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16)
     mk16 = lambda n: [torch.randn((B, 2, n, D), device=dev).bfloat16() for _ in range(L)]  # noqa: E731

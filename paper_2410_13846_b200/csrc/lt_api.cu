@@ -43,8 +43,7 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   DecodePlan p;
   const int64_t n_max = (int64_t)((s.full_capacity > s.n_sink + s.n_recent) ? s.full_capacity
                                                                             : s.n_sink + s.n_recent);
-  const int hsub = decode_head_subgroups(s);
-  const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads * hsub;
+  const int64_t units = (int64_t)s.n_layers * s.batch * s.n_kv_heads;
   // Measured on B200 (32K context, whole stack and one layer per call): long chunks win, per-item
   // hand-off costs more than an uneven last round; shorter chunks only pay when a launch has very few keys.
   p.min_chunk = 512;
@@ -124,7 +123,7 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
 }
 
 size_t ws_prefix_bytes(const lt_shape& s) {
-  const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads * decode_head_subgroups(s) + 2) * sizeof(int);
+  const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads + 2) * sizeof(int);
   return kWsHeaderBytes + round_up(counters, kWsAlign);
 }
 
@@ -474,9 +473,7 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.layer_begin = layer_begin;
   a.layer_count = layer_count;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
-  a.hsub = decode_head_subgroups(*shape);
-  a.gp_stride = shape->n_q_heads / shape->n_kv_heads;
-  a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads * a.hsub;
+  a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;
   a.work_counter = a.done_counter + 1;
   a.part_ml = reinterpret_cast<float*>((char*)ws + prefix);
   a.part_o = reinterpret_cast<float*>((char*)ws + prefix + ml_bytes);

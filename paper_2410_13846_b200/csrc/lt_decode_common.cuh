@@ -10,9 +10,6 @@
 // the same work list:
 //   entry e = (layer, batch row)      n_e = visible keys, nc_e = chunks
 //   items of e = n_kv_heads * nc_e    item -> (kv head, chunk)
-//                (x 2 on the tensor-core path when the query group has 9..16 heads: an item then serves one
-//                 sub-group of at most 8 heads, and the two items of a chunk are neighbours in the list so that
-//                 the second read of the chunk finds it in L2)
 // The prefix sum over entries lives in shared memory; an item index is turned
 // into (entry, kv head, chunk) by binary search.  The chunk length is chosen on
 // the device from the total number of keys of the launch, so that a whole stack
@@ -39,15 +36,12 @@ __device__ __forceinline__ void pdl_allow_next_grid() { asm volatile("griddepcon
 
 struct WorkItem {
   int l, b, h, c;  // layer, batch row, kv head, chunk
-  int hs;          // sub-group of the kv head's query heads served by this item (0 unless the group exceeds 8)
-  int g0, gn;      // first query head of the sub-group within the group, and how many it has
   int nc;          // chunks of this (layer, batch row)
   int n;           // visible keys of this (layer, batch row), clamped to the cache
   int j0, j1;      // key rows [j0, j1) of this chunk
   int rows;        // rows per (b, kv head) of the cache that is read
   int new_row;     // fused append: row taken from k_new / v_new (and stored) by this item, else -1
-  int slot0;       // partial slot of chunk 0 of this (layer, b, kv head, sub-group); chunk c uses slot0 + c * hsub
-  int hsub;        // sub-groups per kv head in this launch (= distance between the slots of consecutive chunks)
+  int slot0;       // partial slot of chunk 0 of this (layer, b, kv head); chunk c uses slot0 + c
   bool lazy;
 };
 
@@ -64,11 +58,9 @@ struct WorkList {
   uint8_t* kind;  // [entries]  bit 0 lazy, bit 1 table entry missing
   int entries;
   int chunk;      // keys per chunk of this launch (before balancing)
-  int hsub;       // sub-groups of query heads per kv head (1, or 2 for groups of 9..16 on the tensor-core path)
 
-  __device__ __forceinline__ void carve(uint8_t* mem, int layer_count, int batch, int head_subgroups) {
+  __device__ __forceinline__ void carve(uint8_t* mem, int layer_count, int batch) {
     entries = layer_count * batch;
-    hsub = head_subgroups;
     prefix = reinterpret_cast<int*>(mem);
     seq = prefix + entries + 1;
     kind = reinterpret_cast<uint8_t*>(seq + batch);
@@ -113,7 +105,7 @@ struct WorkList {
     {
       unsigned long long mine = 0ull;
       for (int e = e0; e < e1; ++e)
-        if (!(kind[e] & 2)) mine += (unsigned long long)visible(a, e, e % B, blockIdx.x == 0) * s.n_kv_heads * hsub;
+        if (!(kind[e] & 2)) mine += (unsigned long long)visible(a, e, e % B, blockIdx.x == 0) * s.n_kv_heads;
       if (mine) atomicAdd(&total_keys, mine);
     }
     __syncthreads();
@@ -131,7 +123,7 @@ struct WorkList {
       if (!(kind[e] & 2)) {
         const int n = visible(a, e, b, false);
         const int nc = max(1, (n + chunk - 1) / chunk);
-        items = s.n_kv_heads * hsub * nc;
+        items = s.n_kv_heads * nc;
       }
       prefix[e + 1] = items;  // turned into the prefix below
       run += items;
@@ -186,15 +178,9 @@ struct WorkList {
     w.n = visible(a, lo, w.b, false);
     w.nc = max(1, (w.n + chunk - 1) / chunk);
     const int rem = idx - prefix[lo];
-    const int per_head = w.nc * hsub;
-    w.h = rem / per_head;
-    const int r2 = rem - w.h * per_head;
-    w.c = r2 / hsub;
-    w.hs = r2 - w.c * hsub;
-    w.hsub = hsub;
-    w.g0 = w.hs * 8;
-    w.gn = hsub > 1 ? min(8, s.n_q_heads / s.n_kv_heads - w.g0) : s.n_q_heads / s.n_kv_heads;
-    w.slot0 = idx - w.c * hsub;
+    w.h = rem / w.nc;
+    w.c = rem - w.h * w.nc;
+    w.slot0 = idx - w.c;
     int len = (w.n + w.nc - 1) / w.nc;  // balanced chunks: no tiny last chunk
     if (s.page_size > 0) len = (len + 31) & ~31;  // paged caches: a 16- or 32-key tile never straddles two pages
     w.j0 = min(w.n, w.c * len);
@@ -209,8 +195,8 @@ struct WorkList {
   }
 };
 
-// Slot of the partials of (layer, b, kv head, sub-group, chunk): the item's own index.
-__device__ __forceinline__ long long partial_unit(const DecodeArgs&, const WorkItem& w) { return w.slot0 + w.c * w.hsub; }
+// Slot of the partials of (layer, b, kv head, chunk): the item's own index.
+__device__ __forceinline__ long long partial_unit(const DecodeArgs&, const WorkItem& w) { return w.slot0 + w.c; }
 
 // Staging buffer (shared memory) for the (max, sum) pairs of a unit's chunks
 // while they are merged; units with more pairs read them from global memory.
@@ -225,7 +211,7 @@ __device__ __forceinline__ bool count_item_in(const DecodeArgs& a, const WorkIte
     __syncthreads();
     return true;
   }
-  const long long unit = (((long long)w.l * a.s.batch + w.b) * a.s.n_kv_heads + w.h) * w.hsub + w.hs;
+  const long long unit = ((long long)w.l * a.s.batch + w.b) * a.s.n_kv_heads + w.h;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();  // cumulative: the partials written before the barrier are visible device-wide
@@ -248,10 +234,10 @@ __device__ __forceinline__ bool count_item_in(const DecodeArgs& a, const WorkIte
 __device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem& w, float2* s_ml) {
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads, D = s.head_dim;
-  const int GP = a.gp_stride;   // heads per partial slot
-  const int Gn = w.gn;          // heads of this sub-group
+  const int GP = G;             // heads per partial slot
+  const int Gn = G;
   const long long unit0 = w.slot0;
-  const long long cs_ml = (long long)w.hsub * GP;  // float2s between the slots of consecutive chunks
+  const long long cs_ml = GP;   // float2s between the slots of consecutive chunks
   const int pairs = w.nc * Gn;
   const bool staged = pairs <= kCombineStagePairs;
   const float2* ml_g = reinterpret_cast<const float2*>(a.part_ml) + unit0 * GP;  // chunk c, head g at c * cs_ml + g
@@ -295,7 +281,7 @@ __device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem
     const float vsc = s.kv_fp8 ? s.kv_scales[2 * w.l + 1] : 1.f;
     const float r0 = den > 0.f ? (num.x / den) * vsc : 0.f, r1 = den > 0.f ? (num.y / den) * vsc : 0.f;
     const float r2 = den > 0.f ? (num.z / den) * vsc : 0.f, r3 = den > 0.f ? (num.w / den) * vsc : 0.f;
-    const long long oi = (((long long)w.l * s.batch + w.b) * s.n_q_heads + w.h * G + w.g0 + g) * D + d;
+    const long long oi = (((long long)w.l * s.batch + w.b) * s.n_q_heads + w.h * G + g) * D + d;
     if (a.out_dtype == LT_F32) {
       *reinterpret_cast<float4*>((float*)a.out + oi) = make_float4(r0, r1, r2, r3);
     } else {

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a, Layer
   pdl_wait_prior_grid();
   pdl_allow_next_grid();
   WorkList wl;
-  wl.carve(smem, a.layer_count, s.batch, 1);
+  wl.carve(smem, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
   const int n_items = wl.total(a);
   const float cs = a.cs;

@@ -1,5 +1,5 @@
-// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 16 (groups above 8 as
-// two sub-groups of at most 8 heads, each its own work item);
+// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 16 (groups above 8 by
+// warp pairs: template branch PAIR);
 // caches in bf16 or (template branch FP8, head_dim 128) in E4M3 bytes.
 //
 // A persistent launch (two CTAs per SM) walks the flattened work list of
@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   pdl_wait_prior_grid();   // the previous launch of the stream is complete: lengths, counters and partial slots are ours
   pdl_allow_next_grid();   // the next launch may take SMs as this one's CTAs retire (it waits the same way)
   WorkList wl;
-  wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch, a.hsub);
+  wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
   const int n_items = wl.total(a);
 
@@ -379,10 +379,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   while (cur < n_items) {
     const int l = w.l, b = w.b, h = w.h;
-    // query heads served by this warp: the item's (the group, or one sub-group of at most 8), or this warp's
-    // eight of a pair's sixteen
-    const int g0 = PAIR ? role * 8 : w.g0;
-    const int Gn = PAIR ? min(8, G - role * 8) : w.gn;
+    // query heads served by this warp: the group, or this warp's eight of a pair's sixteen
+    const int g0 = role * 8;
+    const int Gn = PAIR ? min(8, G - role * 8) : G;
     const int j1 = src_cur.j1;
     int fetched_next = 0;
     if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
@@ -742,7 +741,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         for (int e = 0; e < 2; ++e) {
           const int g = 2 * c + e;
           if (g < Gn) {
-            const long long pslot = unit * a.gp_stride + (PAIR ? g0 : 0) + g;  // the slot's heads in group order
+            const long long pslot = unit * G + g0 + g;  // a slot holds the group's heads in order
             float* po = a.part_o + pslot * kD;
 #pragma unroll
             for (int dt = 0; dt < NK; ++dt) {
@@ -778,7 +777,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   finish_launch(a);
 }
 bool decode_mma_supported(const lt_shape& s) {
-  // groups of 9..16 are served as two sub-groups of at most 8 heads (the chunk is read twice, the second time from L2)
+  // groups of 9..16: two warps per tile, eight heads each
   return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
          (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 8 : 16);
 }

@@ -108,8 +108,6 @@ struct DecodeArgs {
   int min_chunk, max_chunk, target_items, items_cap;
   int fused, advance;
   int pdl;   // launch with the programmatic-serialization attribute (the step comes as several launches)
-  int hsub;       // sub-groups of query heads per kv head: 1, or 2 on the tensor-core path for groups of 9..16
-  int gp_stride;  // heads per partial slot: min(group, 8) on the tensor-core path, the group otherwise
   float cs;  // softmax scale * log2(e)
   float* part_ml;
   float* part_o;
@@ -147,11 +145,6 @@ cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, con
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 // bf16, head_dim 128 or 64, group size <= 16 (<= 8 with 8-bit caches): tensor-core path.
 bool decode_mma_supported(const lt_shape& s);
-// Sub-groups of at most 8 query heads that a kv head's group is served in (1 unless the tensor-core path has a group above 8).
-inline int decode_head_subgroups(const lt_shape& s) {
-  (void)s;
-  return 1;
-}
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                               const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
 

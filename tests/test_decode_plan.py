@@ -26,8 +26,7 @@ def _round_up(x, a):
 def items_of_launch(n_visible, hkv, grid, max_chunk):
     """Items (= partial slots) of one launch over (layer, batch row) pairs with the
     given visible lengths, as the kernels derive them.  `hkv` counts the units of a
-    (layer, batch row): kv heads x sub-groups of at most 8 query heads (the tensor-core
-    path serves a group of 9..16 heads as two sub-groups)."""
+    (layer, batch row): its kv heads."""
     total_keys = sum(n_visible) * hkv
     target = min(grid * 8, TARGET_ITEMS)
     c = -(-total_keys // target) if total_keys else 0
@@ -40,11 +39,9 @@ def slots_in_workspace(shape):
     """Partial slots that the workspace reported by the library has room for."""
     G = shape.n_q_heads // shape.n_kv_heads
     nbytes = lt.workspace_bytes(shape, 0, 0)
-    hsub = 2 if 8 < G <= 16 else 1                    # bf16, head_dim 128: the tensor-core path
-    units = shape.n_layers * shape.batch * shape.n_kv_heads * hsub
+    units = shape.n_layers * shape.batch * shape.n_kv_heads
     prefix = HEADER + _round_up((units + 2) * 4, ALIGN)
-    gp = min(G, 8) if hsub > 1 else G                 # heads per partial slot
-    per_slot = gp * 2 * 4 + gp * shape.head_dim * 4
+    per_slot = G * 2 * 4 + G * shape.head_dim * 4      # a slot holds (max, sum) and O of every head of the group
     # two regions, each rounded up to the alignment: at least (bytes - prefix - 2 * ALIGN) / per_slot slots
     return (nbytes - prefix - 2 * ALIGN) // per_slot, (nbytes - prefix) // per_slot
 
@@ -59,7 +56,6 @@ def test_workspace_covers_every_launch(fp8):
         B = int(g.choice([1, 2, 3, 8, 32, 100]))
         Hkv = int(g.choice([1, 2, 8]))
         G = int(g.choice([1, 4, 5, 8] if fp8 else [1, 4, 5, 8, 12, 16]))
-        hsub = 2 if G > 8 else 1
         S = int(g.choice([0, 4, 64]))
         R = int(g.choice([1, 60, 2044, 4092, 20000]))
         cap = int(g.choice([1, 17, 511, 512, 513, 2047, 2048, 2049, 4097, 32768 + 128, 70000, 131072 + 4]))
@@ -93,7 +89,7 @@ def test_workspace_covers_every_launch(fp8):
                 for done in range(0, count, layers_per_launch):
                     layers = range(begin + done, begin + min(count, done + layers_per_launch))
                     n_vis = [min(int(n), C if mask[l] else cap) for l in layers for n in lens]
-                    items, chunk = items_of_launch(n_vis, Hkv * hsub, grid, max_chunk)
+                    items, chunk = items_of_launch(n_vis, Hkv, grid, max_chunk)
                     assert items <= lo_slots, (trial, L, B, Hkv, G, cap, C, chunk, items, lo_slots)
                     worst = max(worst, items / max(lo_slots, 1))
     assert worst > 0.5          # the sweep does get near the bound: the bound is not vacuous

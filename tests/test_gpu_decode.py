@@ -46,12 +46,12 @@ CASES = [
     (torch.bfloat16, 128, 5, 1, 4, 28, [2049, 2048, 2047, 33], 0.0),        # G=5, chunk boundaries
     (torch.bfloat16, 128, 2, 2, 0, 16, [100, 16, 3], 0.11),                 # G=1, no sink, custom scale
     (torch.bfloat16, 128, 16, 2, 2, 6, [700, 5], 0.0),                      # G=8
-    (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40], 0.0),                    # G=16: two sub-groups of 8 heads per kv head
-    (torch.bfloat16, 128, 12, 1, 4, 28, [4200, 2049, 65], 0.0),             # G=12: sub-groups of 8 and 4, several chunks
+    (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40], 0.0),                    # G=16: warp pairs, eight heads per warp
+    (torch.bfloat16, 128, 12, 1, 4, 28, [4200, 2049, 65], 0.0),             # G=12: warps of a pair serve 8 and 4 heads, several chunks
     (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40], 0.0),                    # G=20 -> CUDA-core path
     (torch.bfloat16, 64, 4, 2, 4, 60, [257, 90], 0.0),                      # D=64: 32-key tiles of 128-byte rows
     (torch.bfloat16, 64, 8, 1, 4, 28, [2049, 2048, 2047, 33, 4500], 0.0),   # D=64, G=8, chunk boundaries
-    (torch.bfloat16, 64, 16, 1, 4, 28, [300, 2100], 0.0),                   # D=64, G=16: sub-groups
+    (torch.bfloat16, 64, 16, 1, 4, 28, [300, 2100], 0.0),                   # D=64, G=16: warp pairs
     (torch.float32, 128, 4, 4, 4, 20, [129, 77], 0.0),                      # fp32
     (torch.float32, 64, 4, 2, 4, 60, [513], 0.0),                           # toy shape
 ]

@@ -31,7 +31,7 @@ CASES = [
     # dtype, D, Hq, Hkv, S, R, lens, steps
     (torch.bfloat16, 128, 8, 2, 4, 28, [300, 1, 0, 31, 32, 2047], 40),      # tensor-core path; wraps; n = 0 start
     (torch.bfloat16, 128, 5, 1, 0, 16, [2040, 15], 20),                    # G=5, no sink, chunk boundary crossed
-    (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40, 2040], 20),              # G=16: two sub-groups per kv head, both store the new row
+    (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40, 2040], 20),              # G=16: warp pairs; the fused append stores the new row once
     (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40], 20),                    # G=20 -> CUDA-core path
     (torch.bfloat16, 64, 8, 2, 4, 28, [300, 1, 0, 31, 32, 2047], 40),      # head_dim 64 on the tensor-core path; wraps
     (torch.bfloat16, 64, 5, 1, 0, 16, [2040, 15], 20),                     # head_dim 64, G=5, chunk boundary crossed
