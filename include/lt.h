@@ -107,7 +107,7 @@ typedef struct lt_shape {
      v_new and out stay in `dtype`.  A stored byte c of layer l means E4M3(c) * kv_scales[l][0] for K and
      * kv_scales[l][1] for V; lt_kv_append / lt_decode_step store code(x) = E4M3 nearest to
      float32(x) / scale (float32 division, round to nearest even, saturating at +-448).  Needs
-     dtype = LT_BF16, head_dim = 128 and a query group of at most 8.  The kernels turn the stored bytes into
+     dtype = LT_BF16, head_dim = 128 and a query group of at most 16.  The kernels turn the stored bytes into
      f16 in registers (exact) and multiply on the tensor cores with fp32 accumulation, q as f16 at one
      power-of-two scale per head (exact for bf16 inputs), the probabilities as one f16 term.  lt_lazy_scores and
      lt_lazy_scores_lse do not read 8-bit keys: score from the prefill's 16-bit keys with a shape whose kv_fp8 is 0. */

@@ -171,7 +171,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
   static_assert(DH == 128 || (DH == 64 && !FP8), "head_dim 128, or 64 with 16-bit caches");
-  static_assert(!(PAIR && FP8), "warp pairs are written for the 16-bit caches");
   constexpr int STREAMS = PAIR ? WARPS / 2 : WARPS;   // independent tile streams of the CTA
   constexpr int RSTAGES = NSTAGE;                     // ring stages of a stream
   constexpr int kD = DH;                       // head_dim
@@ -310,9 +309,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     } else if constexpr (FP8) {
       // raw rows: 8 chunks of 16 bytes per row, K rows then V rows
 #pragma unroll
-      for (int i = 0; i < TILE / 4; ++i) {
-        const int ci = i * 32 + lane;
-        const int r = ci >> 3, p = ci & 7;
+      for (int i = 0; i < FROWS / 4; ++i) {
+        const int r = role * FROWS + 4 * i + (lane >> 3), p = lane & 7;
         const int row = key_base + r;
         const bool valid = row < t.j1;
         const long long goff = (tile_row + (valid ? r : 0)) * kRowBytes + p * 16;
@@ -779,7 +777,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 bool decode_mma_supported(const lt_shape& s) {
   // groups of 9..16: two warps per tile, eight heads each
   return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
-         (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 8 : 16);
+         (s.n_q_heads / s.n_kv_heads) <= 16;
 }
 
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, bool PAIR>
@@ -830,9 +828,11 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
-  // 8-bit caches: three raw stages of 32 keys (8 KB) = the 24 KB per warp of the 16-bit ring
-  if (a.s.kv_fp8) return launch_variant<32, 3, 4, 2, true, 128, false>(a, kf, vf, ks, vs, st);
   const bool pair = a.s.n_q_heads / a.s.n_kv_heads > 8;  // groups of 9..16: two warps per tile, eight heads each
+  // 8-bit caches: raw stages of 32 keys (8 KB); a warp's three stages or a pair's six hold what the 16-bit ring holds
+  if (a.s.kv_fp8)
+    return pair ? launch_variant<32, 6, 4, 2, true, 128, true>(a, kf, vf, ks, vs, st)
+                : launch_variant<32, 3, 4, 2, true, 128, false>(a, kf, vf, ks, vs, st);
   // head_dim 64: rows are half as long, so 32-key tiles keep the bytes in flight per warp (24 KB) the same
   if (a.s.head_dim == 64)
     return pair ? launch_variant<32, 6, 4, 2, false, 64, true>(a, kf, vf, ks, vs, st)

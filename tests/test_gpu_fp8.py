@@ -30,6 +30,8 @@ class Fp8Stack:
     (8, 2, 4, 28, [300, 1, 31, 2047], 36),         # G = 4; the ring wraps; a chunk boundary is crossed
     (5, 1, 0, 16, [70, 15], 20),                   # G = 5, no sink
     (16, 2, 3, 9, [5, 0], 14),                     # G = 8, starts (almost) empty
+    (32, 2, 4, 28, [300, 2047, 33], 36),           # G = 16: warp pairs on the byte path, ring wraps, chunk boundary
+    (12, 1, 2, 12, [4200, 64], 6),                 # G = 12: the second warp of a pair serves four heads; several chunks
 ])
 def test_fp8_caches_append_codes_and_attention(Hq, Hkv, S, R, lens, steps):
     torch.manual_seed(33)
@@ -95,7 +97,7 @@ def test_fp8_shape_is_validated_and_scoring_refuses_8bit_keys():
     sc = torch.full((2, 2), 0.02, dtype=torch.float32, device="cuda")
     ok = lt.Shape(2, 1, 8, 2, 128, 4, 12, 64, lt.LT_BF16, 0.0, kv_fp8=1, kv_scales=sc)
     assert lt.workspace_bytes(ok) > 0
-    for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=32)):
+    for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=34)):
         d = dict(ok.__dict__); d.update(kw)
         with pytest.raises(lt.LtError):
             lt.workspace_bytes(lt.Shape(**d))

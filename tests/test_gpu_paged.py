@@ -58,6 +58,8 @@ CASES = [
     (torch.bfloat16, 128, 5, 1, 0, 16, 256, 9, [2040, 255], 8),                # G=5, several chunks over several pages
     (torch.float32, 64, 4, 2, 4, 28, 128, 3, [200, 40], 16),                   # CUDA-core paths
     (torch.bfloat16, 64, 8, 2, 4, 60, 128, 20, [2300, 129, 2048], 16),         # head_dim 64: 32-key tiles over page boundaries
+    (torch.bfloat16, 128, 32, 2, 4, 60, 128, 20, [2300, 129, 2048], 8),        # G=16: warp pairs, 32-key tiles over page boundaries
+    (torch.bfloat16, 64, 12, 1, 4, 28, 128, 5, [300, 511], 8),                 # head_dim 64, G=12: warp pairs
 ]
 
 
