@@ -34,6 +34,12 @@
 //               exp - no shuffles, no shared memory, nothing written until the end of the
 //               piece.  The accumulator goes back to the MMA warp as soon as the row's last
 //               chunk is in registers.
+// Warps 2-9 read accumulator 0 and warps 10-17 accumulator 1.  A unit with more than 128
+// query rows fills both with every tile (one row block each).  A unit with at most 128
+// rows (multi-head attention, short tails) alternates instead: tile i goes to
+// accumulator i & 1, so the MMAs of a tile run under the statistics of the tile before
+// it, and the second group hands its sums to the first through shared memory at the
+// end of the piece (two mbarriers, waits bounded like all others).
 //
 // Exponentials.  One ex2 per score on the special-function unit (16 per clock per
 // SM) makes that unit the busiest of the SM (~80 %), so a fixed share of the columns
@@ -71,6 +77,7 @@ constexpr int kBlockN = kScoreBlockN;  // keys per tile (one UMMA instruction wi
 constexpr int kQHalfBytes = kBlockM * 128;        // 64 d (one 128-byte half of a row) of the query block: [256 rows][128 B]
 constexpr int kKHalfBytes = kBlockN * 128;        // 64 d of a K tile: [256 rows][128 B]
 constexpr int kBarBytes = 256;
+constexpr int kMergeBytes = 2 * 128 * 3 * 4;      // (reference, sum, windowed sum) of 128 rows x two key halves
 // Geometry that depends on the head dimension DH (128 or 64): a row has DH / 64 halves of 128 bytes; the K ring
 // holds 128 KB either way (2 stages of 64 KB, or 4 of 32 KB).
 template <int DH>
@@ -80,7 +87,7 @@ struct Geo {
   static constexpr int kStageBytes = kHalves * kKHalfBytes;  // 64 KB or 32 KB
   static constexpr int kStages = 4 / kHalves;
   static constexpr int kKSteps = DH / 16;                    // 16-wide k-steps of the contraction
-  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kMergeBytes + 1024;  // + alignment slack
 };
 constexpr int kStatWarps = 16;
 constexpr int kThreads = 64 + kStatWarps * 32;    // 576 (registers are granted as for 640: 96 per thread)
@@ -390,7 +397,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t bar_qfree = bar_qfull + 8;            //            every MMA that reads the query block has completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 16 * kStages + 56);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * kStages + 64);
-  static_assert(16 * kStages + 72 <= kBarBytes, "barrier area too small");
+  const uint32_t bar_mgfull = bar0 + 16 * kStages + 72;  // second statistics group has published its partial sums
+  const uint32_t bar_mgfree = bar_mgfull + 8;            // first group has read them
+  float* merge_buf = reinterpret_cast<float*>(bar_mem + kBarBytes);
+  static_assert(16 * kStages + 88 <= kBarBytes, "barrier area too small");
 
   const lt_shape& s = a.s;
   const int G = s.n_q_heads / s.n_kv_heads;
@@ -411,6 +421,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     mbar_init(bar_qfull, 1);
     mbar_init(bar_qfree, 1);
+    mbar_init(bar_mgfull, kStatWarps * 32 / 2);
+    mbar_init(bar_mgfree, kStatWarps * 32 / 2);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -513,22 +525,26 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int st = kt % kStages;
             ok = mbar_wait(bar_full + 8 * st, (kt / kStages) & 1, abort_flag);
             if (!ok) break;
-            for (int mb = 0; mb < n_mb; ++mb) {
-              int& uses = mb ? uses1 : uses0;
+            // A unit with two row blocks fills both accumulators with every tile.  A unit with one (at most 128
+            // query rows) alternates: tile `it` goes to accumulator it & 1, so that the MMAs of one tile run
+            // while the statistics of the tile before it are taken, by the other group of statistics warps.
+            for (int j = 0; j < n_mb; ++j) {
+              const int acc = n_mb == 1 ? (it & 1) : j;  // accumulator (and statistics group)
+              int& uses = acc ? uses1 : uses0;
               if (uses > 0) {
-                ok = mbar_wait(bar_sempty + 8 * mb, (uses - 1) & 1, abort_flag);
+                ok = mbar_wait(bar_sempty + 8 * acc, (uses - 1) & 1, abort_flag);
                 if (!ok) break;
               }
               ++uses;
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + mb * 256;
+              const uint32_t d_tmem = tmem_base + acc * 256;
 #pragma unroll
               for (int ks = 0; ks < kKSteps; ++ks) {
-                const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + mb * (128 * 128) + (ks & 3) * 32;
+                const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + j * (128 * 128) + (ks & 3) * 32;
                 const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
                 umma_bf16_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
               }
-              umma_commit(bar_sfull + 8 * mb);
+              umma_commit(bar_sfull + 8 * acc);
             }
             if (!ok) break;
             umma_commit(bar_empty + 8 * st);
@@ -542,7 +558,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // Four consecutive warps cover the four TMEM lane quadrants (a warp may access lanes 32 * (warp % 4) ...).
     const int sw = warp - 2;
     const int quad = warp & 3;       // TMEM lane quadrant this warp may access
-    const int mb = (sw >> 2) & 1;    // row block of this warp
+    const int mb = (sw >> 2) & 1;    // statistics group = accumulator of this warp
     const int ch = sw >> 3;          // half of the tile's 256 keys that this warp reads
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + mb * 256 + ch * 128;
     const float cs = a.cs;
@@ -550,14 +566,19 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     bool ok = true;
     long long cursor = 0;
-    int uses = 0;  // score blocks of this row block consumed so far
+    int uses = 0;    // score blocks of this accumulator consumed so far
+    int merges = 0;  // pieces whose partial sums went from the second group to the first
     Piece p;
     uint32_t va[kChunk];
     while (ok && next_piece(a, cursor, p)) {
       const int rows_here = rows_of(p.rb);
       const int n_mb = (rows_here + 127) / 128;
-      const bool active = mb < n_mb;
-      const int r_local = mb * 128 + quad * 32 + lane;
+      // one row block: both groups serve it, tile `it` belongs to group it & 1, and the second group hands
+      // its sums to the first at the end of the piece
+      const bool alt = n_mb == 1;
+      const bool active = alt || mb < n_mb;
+      const int rblk = alt ? 0 : mb;  // row block of the unit that this warp's rows are in
+      const int r_local = rblk * 128 + quad * 32 + lane;
       const int r = p.rb * kBlockM + r_local;   // row of the kv head's G * T query rows
       const bool row_valid = r_local < rows_here;
       const int g = r / T, tq = r - g * T;
@@ -566,7 +587,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       float* stp = a.stats + (rowid * a.n_splits + 2 * p.slot + ch) * 3;
       if (!active || p.n_tiles == 0) {
         // nothing to read: an idle row block, or an empty key range (its slots still get neutral statistics)
-        if (active && row_valid) {
+        if (active && row_valid && (!alt || mb == 0)) {
           stp[0] = -INFINITY;
           stp[1] = 0.f;
           stp[2] = 0.f;
@@ -616,12 +637,14 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       };
 
-      for (int it = 0; it < p.n_tiles; ++it, ++uses) {
+      for (int it = 0; it < p.n_tiles; ++it) {
+        if (alt && (it & 1) != mb) continue;  // the other group's tile
         const int kb = p.ts0 + it * kBlockN + ch * 128;  // first key of this thread's 128 columns
         ok = mbar_wait(bar_sfull + 8 * mb, uses & 1, abort_flag);
         if (!ok) break;
+        ++uses;
         tc_fence_after();
-        if (mb * 128 + quad * 32 >= rows_here) {
+        if (rblk * 128 + quad * 32 >= rows_here) {
           // none of this warp's 32 rows exists (a ragged query block): nothing to read, hand the accumulator back
           tc_fence_before();
           mbar_arrive(bar_sempty + 8 * mb);
@@ -662,6 +685,32 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
       if (!ok) break;
+      if (alt) {
+        // every thread of both groups takes part (also those whose rows do not exist): the barriers count threads
+        float* mg = merge_buf + ((ch * 128 + quad * 32 + lane) * 3);
+        if (mb == 1) {
+          if (merges > 0) ok = mbar_wait(bar_mgfree, (merges - 1) & 1, abort_flag);  // the last piece's values were read
+          if (!ok) break;
+          mg[0] = Mr;
+          mg[1] = sA;
+          mg[2] = sWn;
+          mbar_arrive(bar_mgfull);
+          ++merges;
+          continue;  // the first group writes the piece's statistics
+        }
+        ok = mbar_wait(bar_mgfull, merges & 1, abort_flag);
+        if (!ok) break;
+        const float M1 = mg[0], sA1 = mg[1], sW1 = mg[2];
+        mbar_arrive(bar_mgfree);
+        ++merges;
+        const float Mn = fmaxf(Mr, M1);
+        if (Mn > -INFINITY) {
+          const float c0 = ex2(Mr - Mn), c1 = ex2(M1 - Mn);  // 2^(-inf) = 0 for a side that saw no key
+          sA = sA * c0 + sA1 * c1;
+          sWn = sWn * c0 + sW1 * c1;
+          Mr = Mn;
+        }
+      }
       if (row_valid) {
         stp[0] = Mr;
         stp[1] = sA;
