@@ -47,13 +47,24 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   // Measured on B200 (32K context, whole stack and one layer per call): long chunks win, per-item
   // hand-off costs more than an uneven last round; shorter chunks only pay when a launch has very few keys.
   p.min_chunk = 512;
-  // 8-bit caches: that path is bound by SM-side work, where the hand-off between items (four CTA barriers) is
-  // pure loss: 8192-key chunks measured 9 % faster than 2048-key ones; the 16-bit path is flat from 2048 to 4096.
-  p.max_chunk = s.kv_fp8 ? 8192 : 2048;
+  // 8-bit caches: 8192-key chunks measured 9 % faster than 2048-key ones (the hand-off between items, four CTA
+  // barriers, weighs more the less time an item's bytes take).
+  // The 16-bit path: 4096-key chunks when the launch still has a few of them per CTA (at least 2 * target_items *
+  // 4096 keys, a whole stack at long context: fewer hand-offs, and contexts up to 4096 need no split at all),
+  // 2048 otherwise (one layer per call, where long chunks leave the last round of the grid half empty).
+  p.max_chunk = s.kv_fp8 ? 8192 : 4096;
+  p.mid_chunk = s.kv_fp8 ? 8192 : 2048;
   p.target_items = 592;
-  // chunk = clamp(ceil(keys / target), min, max) gives at most target + units items
-  // when it is not clamped at max, and units * ceil(n_max / max) when it is
-  int64_t cap = units * ((n_max + p.max_chunk - 1) / p.max_chunk) + p.target_items + units;
+  // chunk = clamp(ceil(keys / target), min, max or mid) gives at most target + units items when it is not clamped
+  // from above, units * ceil(n_max / max) when it is clamped at max, fewer than 2 * target * max / mid + units when
+  // it is clamped at mid (such a launch has fewer than 2 * target * max keys), and never more than with every
+  // chunk at its shortest
+  int64_t cap = units * ((n_max + p.max_chunk - 1) / p.max_chunk);
+  const int64_t few = 2 * (int64_t)p.target_items * p.max_chunk / p.mid_chunk;
+  if (cap < few) cap = few;
+  cap += p.target_items + units;
+  const int64_t shortest = units * ((n_max + p.min_chunk - 1) / p.min_chunk);
+  if (cap > shortest) cap = shortest;
   if (cap > (int64_t)0x7fffffff) cap = 0x7fffffff;
   p.items_cap = (int)cap;
   const int G = s.n_q_heads / s.n_kv_heads;
@@ -463,6 +474,7 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.out_dtype = out_dtype;
   a.min_chunk = dp.min_chunk;
   a.max_chunk = dp.max_chunk;
+  a.mid_chunk = dp.mid_chunk;
   a.target_items = dp.target_items;
   a.items_cap = dp.items_cap;
   a.fused = fused;

@@ -113,7 +113,10 @@ struct WorkList {
       const long long target = min((long long)gridDim.x * 8, (long long)a.target_items);
       long long c = (long long)((total_keys + target - 1) / target);
       c = (c + 63) / 64 * 64;
-      chunk = (int)max((long long)a.min_chunk, min((long long)a.max_chunk, c));
+      // the longest chunks only for launches that keep a few of them per CTA
+      const long long hi =
+          total_keys >= 2ull * (unsigned long long)a.target_items * (unsigned long long)a.max_chunk ? a.max_chunk : a.mid_chunk;
+      chunk = (int)max((long long)a.min_chunk, min(hi, c));
     }
     // items per entry, then an exclusive scan
     int run = 0;

@@ -27,6 +27,7 @@ size_t ws_prefix_bytes(const lt_shape& s);
 // workspace query and every later call agree.
 struct DecodePlan {
   int min_chunk, max_chunk;  // the kernels pick the chunk length of a launch in this range (multiples of 64)
+  int mid_chunk;             // upper end of the range for launches with few keys (see make_decode_plan)
   int target_items;          // items a launch aims for when its keys allow (a few per CTA)
   int items_cap;             // most items (= partial slots) any launch over this shape can have
   size_t ml_floats;          // [items_cap][G][2]
@@ -105,7 +106,7 @@ struct DecodeArgs {
   void* out;
   int out_dtype;
   int layer_begin, layer_count;
-  int min_chunk, max_chunk, target_items, items_cap;
+  int min_chunk, mid_chunk, max_chunk, target_items, items_cap;
   int fused, advance;
   int pdl;   // launch with the programmatic-serialization attribute (the step comes as several launches)
   float cs;  // softmax scale * log2(e)

@@ -5,10 +5,12 @@ The kernels choose the chunk length of a launch on the device, from the total
 number of visible keys of that launch; the host sizes the workspace from the
 shape alone.  The item count of a launch is restated here from its definition
 (chunk = total keys spread over the launch's target item count, rounded up to
-64 and clamped to [512, max chunk]; a (layer, batch row) has ceil(n / chunk)
-chunks, at least one, per kv head) and swept over lengths, batch sizes, layer
-ranges, masks and both maximum chunk lengths (2048 for 16-bit caches, 8192 for
-8-bit ones); the real library's workspace size must cover it every time.
+64 and clamped to [512, max chunk], the maximum being the larger one only for
+launches of at least 2 x target x max keys; a (layer, batch row) has
+ceil(n / chunk) chunks, at least one, per kv head) and swept over lengths, batch
+sizes, layer ranges, masks and both pairs of maximum chunk lengths (2048 / 4096
+for 16-bit caches, 8192 / 8192 for 8-bit ones); the real library's workspace size
+must cover it every time.
 """
 import numpy as np
 import pytest
@@ -23,7 +25,7 @@ def _round_up(x, a):
     return (x + a - 1) // a * a
 
 
-def items_of_launch(n_visible, hkv, grid, max_chunk):
+def items_of_launch(n_visible, hkv, grid, max_chunk, mid_chunk):
     """Items (= partial slots) of one launch over (layer, batch row) pairs with the
     given visible lengths, as the kernels derive them.  `hkv` counts the units of a
     (layer, batch row): its kv heads."""
@@ -31,7 +33,8 @@ def items_of_launch(n_visible, hkv, grid, max_chunk):
     target = min(grid * 8, TARGET_ITEMS)
     c = -(-total_keys // target) if total_keys else 0
     c = _round_up(c, 64)
-    chunk = max(MIN_CHUNK, min(max_chunk, c))
+    hi = max_chunk if total_keys >= 2 * TARGET_ITEMS * max_chunk else mid_chunk   # the longest chunks only for large launches
+    chunk = max(MIN_CHUNK, min(hi, c))
     return sum(hkv * max(1, -(-n // chunk)) for n in n_visible), chunk
 
 
@@ -42,14 +45,15 @@ def slots_in_workspace(shape):
     units = shape.n_layers * shape.batch * shape.n_kv_heads
     prefix = HEADER + _round_up((units + 2) * 4, ALIGN)
     per_slot = G * 2 * 4 + G * shape.head_dim * 4      # a slot holds (max, sum) and O of every head of the group
-    # two regions, each rounded up to the alignment: at least (bytes - prefix - 2 * ALIGN) / per_slot slots
-    return (nbytes - prefix - 2 * ALIGN) // per_slot, (nbytes - prefix) // per_slot
+    # two regions of 4-byte words, each rounded up to the alignment (at most ALIGN - 4 bytes of padding each):
+    # slots * per_slot >= bytes - prefix - 2 * (ALIGN - 4)
+    return -(-(nbytes - prefix - 2 * (ALIGN - 4)) // per_slot), (nbytes - prefix) // per_slot
 
 
 @pytest.mark.parametrize("fp8", [0, 1])
 def test_workspace_covers_every_launch(fp8):
     g = np.random.default_rng(5 + fp8)
-    max_chunk = 8192 if fp8 else 2048
+    max_chunk, mid_chunk = (8192, 8192) if fp8 else (4096, 2048)
     worst = 0.0
     for trial in range(400):
         L = int(g.choice([1, 2, 3, 8, 32, 64, 128]))
@@ -89,19 +93,21 @@ def test_workspace_covers_every_launch(fp8):
                 for done in range(0, count, layers_per_launch):
                     layers = range(begin + done, begin + min(count, done + layers_per_launch))
                     n_vis = [min(int(n), C if mask[l] else cap) for l in layers for n in lens]
-                    items, chunk = items_of_launch(n_vis, Hkv, grid, max_chunk)
+                    items, chunk = items_of_launch(n_vis, Hkv, grid, max_chunk, mid_chunk)
                     assert items <= lo_slots, (trial, L, B, Hkv, G, cap, C, chunk, items, lo_slots)
                     worst = max(worst, items / max(lo_slots, 1))
     assert worst > 0.5          # the sweep does get near the bound: the bound is not vacuous
 
 
 def test_restated_item_count_on_the_benchmark_stack():
-    """The 32K benchmark stack: 16 full layers x 8 rows x 8 kv heads x 17 chunks of
-    <= 2048 keys + 16 lazy layers with one chunk per (row, kv head)."""
+    """The 32K benchmark stack: 16 full layers x 8 rows x 8 kv heads x 9 chunks of
+    <= 4096 keys + 16 lazy layers with one chunk per (row, kv head); one of its layers alone: 2048-key chunks."""
     n = 32768 + 64
     n_vis = [n] * (16 * 8) + [2048] * (16 * 8)
-    items, chunk = items_of_launch(n_vis, 8, 296, 2048)
-    assert chunk == 2048 and items == 16 * 8 * 8 * 17 + 16 * 8 * 8
+    items, chunk = items_of_launch(n_vis, 8, 296, 4096, 2048)
+    assert chunk == 4096 and items == 16 * 8 * 8 * 9 + 16 * 8 * 8
+    items, chunk = items_of_launch([n] * 8, 8, 296, 4096, 2048)
+    assert chunk == 2048 and items == 8 * 8 * 17
     # a one-layer call over 3000 keys picks the shortest chunks
-    items, chunk = items_of_launch([3000], 2, 296, 2048)
+    items, chunk = items_of_launch([3000], 2, 296, 4096, 2048)
     assert chunk == 512 and items == 2 * 6
