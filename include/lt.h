@@ -144,6 +144,14 @@ int32_t lt_ring_slot(int32_t pos, int32_t n_sink, int32_t n_recent);
 lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max,
                              size_t* bytes_out /* host */);
 
+/*
+ * lt_workspace_bytes for a workspace that lt_decode_step_layers can use as well
+ * (Appendix A's per-layer call): never less than lt_workspace_bytes, and room
+ * for every layer's own partial slots.  Host only.
+ */
+lt_status lt_workspace_bytes_layers(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max,
+                                    size_t* bytes_out /* host */);
+
 /* Zero the workspace (async on `stream`); once, before its first use. */
 lt_status lt_workspace_init(void* ws /* dev */, size_t ws_bytes, void* stream);
 
@@ -355,6 +363,40 @@ lt_status lt_decode_step(const lt_shape* shape, const void* q /* dev */, const v
                          const uint8_t* layer_mask /* dev */, int32_t* seq_lens /* dev [B] */, void* out /* dev */,
                          int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int32_t advance_seq_lens,
                          void* ws /* dev */, size_t ws_bytes, void* stream);
+
+/*
+ * lt_decode_step for a caller that issues one step as several launches over
+ * disjoint layer ranges (Appendix A runs the cache-updating attention call once
+ * per layer) and can tell the library which of them do not depend on the launch
+ * before them.  Same operation, arguments and results as lt_decode_step, plus:
+ *   independent_of_previous  0: plain stream order, as lt_decode_step.
+ *       1: the caller vouches that the work enqueued on `stream` since the last
+ *       call of this function with independent_of_previous = 0 consists only of
+ *       calls of this function for the same step (same shape, tables, mask,
+ *       seq_lens and workspace) over layer ranges disjoint from this one, none
+ *       of them with advance_seq_lens != 0, and that nothing this call reads (q,
+ *       k_new, v_new of its layers) is written by them.  The launch then starts
+ *       on its items as soon as SMs come free under the tail of the launches
+ *       before it instead of waiting for them to complete; its own completion
+ *       still implies theirs, so whatever follows on the stream sees plain
+ *       stream order.  The first call of every step passes 0 (it reads the
+ *       seq_lens that the previous step's last call advanced).
+ * A model whose other layers produce q for layer l + 1 from the output of layer
+ * l has a true dependency and passes 0 throughout; the flag is for callers that
+ * hold the inputs of several layers at once (speculative or batched layer
+ * execution, benchmarks of the attention stack).
+ * Every layer owns its partial slots and launch counters in the workspace, which
+ * therefore must have lt_workspace_bytes_layers bytes (zeroed once with
+ * lt_workspace_init); LT_ERR_WORKSPACE otherwise.  Results are bit-identical to
+ * the same sequence of calls with independent_of_previous = 0.
+ */
+lt_status lt_decode_step_layers(const lt_shape* shape, const void* q /* dev */, const void* k_new /* dev */,
+                                const void* v_new /* dev */, void* const* k_full, void* const* v_full,
+                                void* const* k_stream, void* const* v_stream /* host tables */,
+                                const uint8_t* layer_mask /* dev */, int32_t* seq_lens /* dev [B] */,
+                                void* out /* dev */, int32_t out_dtype, int32_t layer_begin, int32_t layer_count,
+                                int32_t advance_seq_lens, int32_t independent_of_previous, void* ws /* dev */,
+                                size_t ws_bytes, void* stream);
 
 /*
  * lt_decode_step for a caller whose step inputs and outputs live in HOST

@@ -132,6 +132,11 @@ def lib() -> C.CDLL:
     L.lt_decode_step.restype = i32
     L.lt_decode_step.argtypes = [shp, vp, vp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
     L.lt_decode_step_host.restype = i32
+    L.lt_decode_step_layers.restype = i32
+    L.lt_workspace_bytes_layers.restype = i32
+    L.lt_decode_step_layers.argtypes = [shp, vp, vp, vp, tab, tab, tab, tab, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz,
+                                        vp]
+    L.lt_workspace_bytes_layers.argtypes = [shp, i32, i32, C.POINTER(sz)]
     L.lt_decode_step_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, tab, tab, tab, tab, vp, vp, i32, vp, sz, vp]
     _LIB = L
     return L
@@ -302,6 +307,27 @@ def decode_step(shape: Shape, q, k_new, v_new, tables: LayerTables, layer_mask, 
                              tables.k_stream, tables.v_stream, _ptr(layer_mask), _ptr(seq_lens), _ptr(out), out_dtype,
                              layer_begin, cnt, 1 if advance_seq_lens else 0, _ptr(ws),
                              ws.numel() * ws.element_size(), _stream(stream)), "lt_decode_step")
+
+
+def decode_step_layers(shape: Shape, q, k_new, v_new, tables: LayerTables, layer_mask, seq_lens, out, ws,
+                       layer_begin: int, layer_count: int = 1, advance_seq_lens: bool = False,
+                       independent_of_previous: bool = False, out_dtype: int | None = None, stream=None):
+    """lt_decode_step_layers: one launch of a step that comes as several launches over disjoint layer ranges."""
+    import torch
+    if out_dtype is None:
+        out_dtype = LT_F32 if out.dtype == torch.float32 else LT_BF16
+    _ok(lib().lt_decode_step_layers(C.byref(shape.c()), _ptr(q), _ptr(k_new), _ptr(v_new), tables.k_full,
+                                    tables.v_full, tables.k_stream, tables.v_stream, _ptr(layer_mask), _ptr(seq_lens),
+                                    _ptr(out), out_dtype, layer_begin, layer_count, 1 if advance_seq_lens else 0,
+                                    1 if independent_of_previous else 0, _ptr(ws), ws.numel() * ws.element_size(),
+                                    _stream(stream)), "lt_decode_step_layers")
+
+
+def workspace_bytes_layers(shape: Shape, n_ctx_max: int = 0, w_last_max: int = 0) -> int:
+    out = C.c_size_t(0)
+    _ok(lib().lt_workspace_bytes_layers(C.byref(shape.c()), n_ctx_max, w_last_max, C.byref(out)),
+        "lt_workspace_bytes_layers")
+    return out.value
 
 
 def decode_step_host(shape: Shape, q_host, k_new_host, v_new_host, out_host, q_dev, k_new_dev, v_new_dev, out_dev,

@@ -67,6 +67,13 @@ DecodePlan make_decode_plan(const lt_shape& s) {
   if (cap > shortest) cap = shortest;
   if (cap > (int64_t)0x7fffffff) cap = 0x7fffffff;
   p.items_cap = (int)cap;
+  // One layer's share of any launch: chunk >= ceil(keys / target) gives at most target + units items, a chunk
+  // clamped from above is at least mid_chunk long; a launch over k layers has at most k times this.
+  const int64_t units_l = (int64_t)s.batch * s.n_kv_heads;
+  int64_t lcap = units_l * ((n_max + p.mid_chunk - 1) / p.mid_chunk);
+  if (lcap < p.target_items + units_l) lcap = p.target_items + units_l;
+  if (lcap * s.n_layers > (int64_t)0x7fffffff) lcap = 0x7fffffff / s.n_layers;
+  p.layer_items_cap = (int)lcap;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int gp = G;  // heads per partial slot
   p.ml_floats = (size_t)cap * gp * 2;
@@ -134,8 +141,15 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
 }
 
 size_t ws_prefix_bytes(const lt_shape& s) {
-  const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads + 2) * sizeof(int);
+  const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads + 2 * (size_t)s.n_layers) * sizeof(int);
   return kWsHeaderBytes + round_up(counters, kWsAlign);
+}
+
+size_t layered_decode_bytes(const lt_shape& s) {
+  const DecodePlan dp = make_decode_plan(s);
+  const size_t slots = (size_t)dp.layer_items_cap * s.n_layers;
+  const size_t G = s.n_q_heads / s.n_kv_heads;
+  return round_up(slots * G * 2 * 4, kWsAlign) + round_up(slots * G * s.head_dim * 4, kWsAlign);
 }
 
 int sm_count_of_current_device() {
@@ -228,6 +242,14 @@ lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w
     score_bytes = round_up((sp.stat_floats > sw.stat_floats ? sp.stat_floats : sw.stat_floats) * 4, kWsAlign);
   }
   *bytes_out = ws_prefix_bytes(*shape) + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
+  return LT_OK;
+}
+
+lt_status lt_workspace_bytes_layers(const lt_shape* shape, int32_t n_ctx_max, int32_t w_last_max, size_t* bytes_out) {
+  lt_status st = lt_workspace_bytes(shape, n_ctx_max, w_last_max, bytes_out);
+  if (st != LT_OK) return st;
+  const size_t layered = ws_prefix_bytes(*shape) + layered_decode_bytes(*shape);
+  if (layered > *bytes_out) *bytes_out = layered;
   return LT_OK;
 }
 
@@ -437,7 +459,7 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
                              const void* const* k_full, const void* const* v_full, const void* const* k_stream,
                              const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
                              int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
-                             void* ws, size_t ws_bytes) {
+                             void* ws, size_t ws_bytes, int layered, int independent) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q || !layer_mask || !seq_lens || !out) return LT_ERR_INVALID_ARG;
@@ -457,8 +479,12 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
 
   DecodePlan dp = make_decode_plan(*shape);
   const size_t prefix = ws_prefix_bytes(*shape);
-  const size_t ml_bytes = round_up(dp.ml_floats * 4, kWsAlign);
-  const size_t o_bytes = round_up(dp.o_floats * 4, kWsAlign);
+  // layered: every layer owns layer_items_cap partial slots, so that launches over different layers can be in
+  // flight together; otherwise every launch starts at slot 0
+  const size_t slots = layered ? (size_t)dp.layer_items_cap * shape->n_layers : (size_t)dp.items_cap;
+  const size_t G = shape->n_q_heads / shape->n_kv_heads;
+  const size_t ml_bytes = round_up(slots * G * 2 * 4, kWsAlign);
+  const size_t o_bytes = round_up(slots * G * shape->head_dim * 4, kWsAlign);
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   if (ws_bytes < prefix + ml_bytes + o_bytes) return LT_ERR_WORKSPACE;
 
@@ -476,7 +502,9 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.max_chunk = dp.max_chunk;
   a.mid_chunk = dp.mid_chunk;
   a.target_items = dp.target_items;
-  a.items_cap = dp.items_cap;
+  a.items_cap = layered ? dp.layer_items_cap : dp.items_cap;  // layered: per layer, scaled by decode_launch
+  a.overlap = (layered && independent) ? 1 : 0;
+  a.slot_base = layered ? 1 : 0;  // layered: turned into layer_begin * layer_items_cap by decode_launch
   a.fused = fused;
   a.advance = advance;
   // A call over part of the stack is one of several launches of a step (a model calls layer by layer):
@@ -485,7 +513,8 @@ lt_status lt::decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q
   a.layer_begin = layer_begin;
   a.layer_count = layer_count;
   a.unit_counters = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
-  a.done_counter = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;
+  a.launch_counters = a.unit_counters + (size_t)shape->n_layers * shape->batch * shape->n_kv_heads;
+  a.done_counter = a.launch_counters + 2 * (size_t)layer_begin;
   a.work_counter = a.done_counter + 1;
   a.part_ml = reinterpret_cast<float*>((char*)ws + prefix);
   a.part_o = reinterpret_cast<float*>((char*)ws + prefix + ml_bytes);
@@ -502,11 +531,22 @@ lt_status lt::decode_launch(const DecodeCall& c, void* stream) {
   const int layer_begin = c.a.layer_begin, layer_count = c.a.layer_count;
   const int layers_per_launch = kMaxWorkEntries / a.s.batch;
   const bool mma = decode_mma_supported(a.s);
+  const bool layered = c.a.slot_base != 0;
   for (int done = 0; done < layer_count; done += layers_per_launch) {
     a.layer_begin = layer_begin + done;
     a.layer_count = layer_count - done < layers_per_launch ? layer_count - done : layers_per_launch;
     a.advance = (c.a.advance && done + a.layer_count == layer_count) ? 1 : 0;
     if (layer_count > layers_per_launch) a.pdl = 1;  // a stack that is split here is several launches too
+    a.done_counter = a.launch_counters + 2 * (size_t)a.layer_begin;
+    a.work_counter = a.done_counter + 1;
+    if (layered) {
+      a.slot_base = a.layer_begin * c.a.items_cap;
+      a.items_cap = a.layer_count * c.a.items_cap;
+      // the later launches of a split call share nothing with the ones before them either; only the tensor-core
+      // kernel starts without waiting
+      a.overlap = (mma && (c.a.overlap || done > 0)) ? 1 : 0;
+      a.pdl = 1;
+    }
     cudaError_t e = mma ? launch_decode_mma(a, c.kf, c.vf, c.ks, c.vs, cs) : launch_decode_generic(a, c.kf, c.vf, c.ks, c.vs, cs);
     if (e != cudaSuccess) return LT_ERR_CUDA;
   }
@@ -546,6 +586,22 @@ lt_status lt_decode_step(const lt_shape* shape, const void* q, const void* k_new
   return decode_impl(shape, q, k_new, v_new, (const void* const*)k_full, (const void* const*)v_full,
                      (const void* const*)k_stream, (const void* const*)v_stream, layer_mask, seq_lens, out, out_dtype,
                      layer_begin, layer_count, 1, advance_seq_lens ? 1 : 0, ws, ws_bytes, stream);
+}
+
+lt_status lt_decode_step_layers(const lt_shape* shape, const void* q, const void* k_new, const void* v_new,
+                                void* const* k_full, void* const* v_full, void* const* k_stream,
+                                void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
+                                int32_t out_dtype, int32_t layer_begin, int32_t layer_count,
+                                int32_t advance_seq_lens, int32_t independent_of_previous, void* ws, size_t ws_bytes,
+                                void* stream) {
+  DecodeCall c;
+  const lt_status st = decode_prepare(&c, shape, q, k_new, v_new, (const void* const*)k_full,
+                                      (const void* const*)v_full, (const void* const*)k_stream,
+                                      (const void* const*)v_stream, layer_mask, seq_lens, out, out_dtype, layer_begin,
+                                      layer_count, 1, advance_seq_lens ? 1 : 0, ws, ws_bytes, 1,
+                                      independent_of_previous ? 1 : 0);
+  if (st != LT_OK) return st;
+  return decode_launch(c, stream);
 }
 
 lt_status lt_decode_step_host(const lt_shape* shape, const void* q_host, const void* k_new_host,

@@ -31,6 +31,16 @@ namespace lt {
 // seq_lens (advanced by a step's last launch), the launch counters and the partial slots of the
 // workspace - is touched only after the wait, which is the first statement of the kernels.  Without the
 // attribute both calls are no-ops.
+//
+// A launch with DecodeArgs::overlap set does not wait at its start: the caller has vouched that it shares
+// nothing with the launches before it (another layer range of the same step, none of which advances
+// seq_lens), its counters and partial slots are those of its own layers, and so its CTAs start on their
+// items as soon as SMs come free under the previous launch's tail.  Two rules keep stream order intact.
+// A launch lets its successor in only after every one of its CTAs has read seq_lens (the trigger follows
+// the work-list build), so a successor that advances seq_lens at its end cannot be read too early by
+// anyone: by induction every earlier launch has all its CTAs past that read.  And the last CTA of an
+// overlapped launch waits for the prior grid before it retires, so the completion of a launch still
+// implies the completion of everything before it.
 __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_allow_next_grid() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
@@ -199,7 +209,9 @@ struct WorkList {
 };
 
 // Slot of the partials of (layer, b, kv head, chunk): the item's own index.
-__device__ __forceinline__ long long partial_unit(const DecodeArgs&, const WorkItem& w) { return w.slot0 + w.c; }
+__device__ __forceinline__ long long partial_unit(const DecodeArgs& a, const WorkItem& w) {
+  return (long long)a.slot_base + w.slot0 + w.c;
+}
 
 // Staging buffer (shared memory) for the (max, sum) pairs of a unit's chunks
 // while they are merged; units with more pairs read them from global memory.
@@ -239,7 +251,7 @@ __device__ __forceinline__ void combine_unit(const DecodeArgs& a, const WorkItem
   const int G = s.n_q_heads / s.n_kv_heads, D = s.head_dim;
   const int GP = G;             // heads per partial slot
   const int Gn = G;
-  const long long unit0 = w.slot0;
+  const long long unit0 = (long long)a.slot_base + w.slot0;
   const long long cs_ml = GP;   // float2s between the slots of consecutive chunks
   const int pairs = w.nc * Gn;
   const bool staged = pairs <= kCombineStagePairs;
@@ -306,6 +318,7 @@ __device__ __forceinline__ void finish_launch(const DecodeArgs& a) {
     __threadfence();
     const int prev = atomicAdd(a.done_counter, 1);
     if (prev == (int)gridDim.x - 1) {
+      if (a.overlap) pdl_wait_prior_grid();  // this launch is complete only when the ones before it are
       *a.done_counter = 0;
       *a.work_counter = 0;
       if (a.fused && a.advance)

@@ -195,11 +195,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   float* sm_buf = reinterpret_cast<float*>(smem + RING_BYTES);  // [2][8][head_dim]
   float* sm_m = sm_buf + 2 * 8 * kD;                            // [WARPS][8]
   float* sm_l = sm_m + WARPS * 8;                               // [WARPS][8]
-  pdl_wait_prior_grid();   // the previous launch of the stream is complete: lengths, counters and partial slots are ours
-  pdl_allow_next_grid();   // the next launch may take SMs as this one's CTAs retire (it waits the same way)
+  // the previous launch of the stream is complete: lengths, counters and partial slots are ours (an overlapped
+  // launch has its own and starts at once)
+  if (!a.overlap) pdl_wait_prior_grid();
   WorkList wl;
   wl.carve(smem + RING_BYTES + MERGE_BYTES, a.layer_count, s.batch);
   wl.build(a, kf, vf, ks, vs);
+  pdl_allow_next_grid();   // seq_lens has been read: the next launch may take SMs as this one's CTAs retire
   const int n_items = wl.total(a);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

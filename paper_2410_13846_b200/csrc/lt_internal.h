@@ -19,8 +19,9 @@ struct LayerTable {
 // [region used by the running call: split-KV partials or scoring statistics].
 constexpr size_t kWsHeaderBytes = 256;
 constexpr size_t kWsAlign = 256;
-// Bytes of header + counters ([L][B][Hkv] unit counters, then the two launch
-// counters); everything here must be zero between calls (lt_workspace_init).
+// Bytes of header + counters ([L][B][Hkv] unit counters, then two launch
+// counters per layer: a launch uses the pair of its first layer); everything
+// here must be zero between calls (lt_workspace_init).
 size_t ws_prefix_bytes(const lt_shape& s);
 
 // Split-KV plan of the decode step; a function of the shape alone so that the
@@ -30,6 +31,8 @@ struct DecodePlan {
   int mid_chunk;             // upper end of the range for launches with few keys (see make_decode_plan)
   int target_items;          // items a launch aims for when its keys allow (a few per CTA)
   int items_cap;             // most items (= partial slots) any launch over this shape can have
+  int layer_items_cap;       // most items per layer of any launch (a launch over k layers has at most k times this):
+                             // what a step issued as concurrent per-layer launches reserves for every layer
   size_t ml_floats;          // [items_cap][G][2]
   size_t o_floats;           // [items_cap][G][D]
 };
@@ -109,12 +112,16 @@ struct DecodeArgs {
   int min_chunk, mid_chunk, max_chunk, target_items, items_cap;
   int fused, advance;
   int pdl;   // launch with the programmatic-serialization attribute (the step comes as several launches)
+  int overlap;    // the caller vouches that this launch shares nothing with the launches before it on the stream
+                  // (another layer range of the same step): it does not wait for them before it starts
+  int slot_base;  // first partial slot of this launch (0, or the launch's own region when launches may overlap)
   float cs;  // softmax scale * log2(e)
   float* part_ml;
   float* part_o;
   int* unit_counters;  // [L][B][Hkv], zero between launches
-  int* done_counter;   // zero between launches
-  int* work_counter;   // zero between launches: dynamic item hand-out
+  int* launch_counters;  // [L][2], zero between launches; the two below are the pair of layer_begin
+  int* done_counter;     // zero between launches
+  int* work_counter;     // zero between launches: dynamic item hand-out
   uint32_t* dev_err;
 };
 // Most (layer, batch row) pairs one launch can take (its work list lives in
@@ -160,7 +167,9 @@ lt_status decode_prepare(DecodeCall* c, const lt_shape* shape, const void* q, co
                          const void* const* k_full, const void* const* v_full, const void* const* k_stream,
                          const void* const* v_stream, const uint8_t* layer_mask, int32_t* seq_lens, void* out,
                          int32_t out_dtype, int32_t layer_begin, int32_t layer_count, int fused, int advance,
-                         void* ws, size_t ws_bytes);
+                         void* ws, size_t ws_bytes, int layered = 0, int independent = 0);
+// Bytes of the split-KV region when every layer has partial slots of its own (lt_decode_step_layers).
+size_t layered_decode_bytes(const lt_shape& s);
 lt_status decode_launch(const DecodeCall& c, void* stream);
 
 struct ScoreArgs {

@@ -10,7 +10,9 @@ launches of at least 2 x target x max keys; a (layer, batch row) has
 ceil(n / chunk) chunks, at least one, per kv head) and swept over lengths, batch
 sizes, layer ranges, masks and both pairs of maximum chunk lengths (2048 / 4096
 for 16-bit caches, 8192 / 8192 for 8-bit ones); the real library's workspace size
-must cover it every time.
+must cover it every time.  The same sweep checks the per-layer bound behind
+lt_decode_step_layers: a launch over k layers never has more than k times the
+slots that the layered workspace keeps for every layer.
 """
 import numpy as np
 import pytest
@@ -43,7 +45,7 @@ def slots_in_workspace(shape):
     G = shape.n_q_heads // shape.n_kv_heads
     nbytes = lt.workspace_bytes(shape, 0, 0)
     units = shape.n_layers * shape.batch * shape.n_kv_heads
-    prefix = HEADER + _round_up((units + 2) * 4, ALIGN)
+    prefix = HEADER + _round_up((units + 2 * shape.n_layers) * 4, ALIGN)   # unit counters + a counter pair per layer
     per_slot = G * 2 * 4 + G * shape.head_dim * 4      # a slot holds (max, sum) and O of every head of the group
     # two regions of 4-byte words, each rounded up to the alignment (at most ALIGN - 4 bytes of padding each):
     # slots * per_slot >= bytes - prefix - 2 * (ALIGN - 4)
@@ -73,6 +75,13 @@ def test_workspace_covers_every_launch(fp8):
                 def data_ptr(self): return 0x1000
             shape.kv_scales = _Fake()
         lo_slots, _ = slots_in_workspace(shape)
+        # lt_decode_step_layers gives every layer its own slots: most items per layer of any launch
+        n_max = max(cap, S + R)
+        per_layer = max(TARGET_ITEMS + B * Hkv, B * Hkv * -(-n_max // mid_chunk))
+        units = L * B * Hkv
+        layered_need = (HEADER + _round_up((units + 2 * L) * 4, ALIGN) + _round_up(per_layer * L * G * 2 * 4, ALIGN)
+                        + _round_up(per_layer * L * G * 128 * 4, ALIGN))
+        assert lt.workspace_bytes_layers(shape, 0, 0) >= max(layered_need, lt.workspace_bytes(shape, 0, 0))
         C = S + R
         layers_per_launch = max(1, MAX_ENTRIES // B)
         for _ in range(6):
@@ -95,6 +104,7 @@ def test_workspace_covers_every_launch(fp8):
                     n_vis = [min(int(n), C if mask[l] else cap) for l in layers for n in lens]
                     items, chunk = items_of_launch(n_vis, Hkv, grid, max_chunk, mid_chunk)
                     assert items <= lo_slots, (trial, L, B, Hkv, G, cap, C, chunk, items, lo_slots)
+                    assert items <= per_layer * len(layers), (trial, L, B, Hkv, cap, C, chunk, items, per_layer)
                     worst = max(worst, items / max(lo_slots, 1))
     assert worst > 0.5          # the sweep does get near the bound: the bound is not vacuous
 
