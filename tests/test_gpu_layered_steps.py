@@ -1,7 +1,6 @@
 """GPU parity of lt_decode_step_layers: a step issued as launches over disjoint layer ranges that may run under
 one another's tails.  Bit-identical to the same launches in plain stream order (lt_decode_step layer by
 layer), and equal to the oracle (O1 / O2 on the logical history) on units sampled at the last step."""
-import numpy as np
 import pytest
 import torch
 
@@ -127,3 +126,63 @@ def test_layered_entry_refuses_a_workspace_without_per_layer_slots():
     with pytest.raises(lt.LtError) as e:
         lt.decode_step_layers(st.shape, q, k, k, st.tables, st.mask, st.seq_lens, out, small, layer_begin=0)
     assert e.value.status == 3      # LT_ERR_WORKSPACE: nothing was enqueued
+
+
+def test_captured_overlapped_step_replays():
+    """A step of overlapped per-layer launches captured as one CUDA graph and replayed back to back: every
+    replay equals an eager whole-stack step, bit for bit (the programmatic edges between the kernel nodes are
+    part of the graph; a replay's first launch waits for the replay before it)."""
+    torch.manual_seed(41)
+    L, B, Hq, Hkv, D, S, R, n0, steps = 6, 2, 8, 2, 128, 4, 28, 700, 12
+    cap = n0 + steps + 2
+    mask = [0, 1, 0, 1, 0, 0]
+    eager = Stack(L, B, Hq, Hkv, D, S, R, cap)
+    graph = Stack(L, B, Hq, Hkv, D, S, R, cap)
+    for st in (eager, graph):
+        st.set_mask(mask); st.set_seq_lens([n0, n0 - 300])
+    for l in range(L):
+        k0 = torch.randn(B, Hkv, cap, D).bfloat16().cuda(); v0 = torch.randn(B, Hkv, cap, D).bfloat16().cuda()
+        for st in (eager, graph):
+            st.k_full[l].copy_(k0); st.v_full[l].copy_(v0)
+    for st in (eager, graph):
+        lt.stream_init(st.shape, st.mask, st.tables, st.seq_lens, ws=st.ws)
+    _layered_ws(graph)
+    sq = torch.zeros(L, B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    sk = torch.zeros(L, B, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    sv = torch.zeros_like(sk)
+    so = torch.zeros(L, B, Hq, D, dtype=torch.float32, device="cuda")
+
+    def layered_step(st):
+        for l in range(L):
+            lt.decode_step_layers(st.shape, sq, sk, sv, st.tables, st.mask, st.seq_lens, so, st.ws, layer_begin=l,
+                                  advance_seq_lens=(l == L - 1), independent_of_previous=(l > 0))
+
+    warm = Stack(L, B, Hq, Hkv, D, S, R, cap)                    # per-device lookups happen outside the capture
+    warm.set_seq_lens([1, 1])
+    _layered_ws(warm)
+    layered_step(warm)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            layered_step(graph)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    refs, gots = [], []
+    for step in range(steps):
+        q = torch.randn(L, B, Hq, D).bfloat16().cuda()
+        k = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        v = torch.randn(L, B, Hkv, D).bfloat16().cuda()
+        ref = torch.zeros_like(so)
+        lt.decode_step(eager.shape, q, k, v, eager.tables, eager.mask, eager.seq_lens, ref, eager.ws)
+        sq.copy_(q); sk.copy_(k); sv.copy_(v)
+        g.replay()
+        refs.append(ref); gots.append(so.clone())               # stream-ordered: no host synchronisation in the loop
+    torch.cuda.synchronize()
+    for step in range(steps):
+        assert torch.equal(gots[step], refs[step]), step
+    assert torch.equal(graph.seq_lens, eager.seq_lens) and lt.check(graph.ws) == 0
+    for l in range(L):
+        assert torch.equal(graph.k_full[l], eager.k_full[l]) and torch.equal(graph.k_stream[l], eager.k_stream[l])
