@@ -92,7 +92,10 @@ static int host_score_splits(const lt_shape& s, int n_ctx, int w_last, bool wind
     if (w0 < S) w0 = S;
     span = n_ctx - w0;
   }
-  int64_t most = (span + 1023) / 1024;
+  // shortest split: 1024 keys on the tensor-core path; the CUDA-core kernel walks a split tile by tile in one CTA,
+  // so small problems are cut finer there to fill the GPU
+  const int shortest = scores_umma_supported(s, w_last) ? 1024 : 128;
+  int64_t most = (span + shortest - 1) / shortest;
   if (want > most) want = most;
   if (want < 1) want = 1;
   int len = (int)((span + want - 1) / want);

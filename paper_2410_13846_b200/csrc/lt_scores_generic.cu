@@ -1,16 +1,29 @@
-// Lazy ratio (Eq. 1), reference-quality CUDA-core path (any dtype, head_dim 64
-// or 128), the merge kernel shared by all scoring paths, and the selection.
+// Lazy ratio (Eq. 1), CUDA-core path (fp32 stacks; head_dim 64 or 128), the merge
+// kernel shared by all scoring paths, and the selection.
 //
 // Partial statistics of one tail row (layer, b, hq, t) over one key split, log2
 // domain with t_j = scale * log2(e) * (q . k_j):
 //   M = max_j t_j,  A = sum_j 2^(t_j - M),  W = sum_{j in window} 2^(t_j - M)
 // over the visible keys j <= n_ctx - w_last + t of the split; the window is
 // {j < n_sink} U {j >= n_ctx - n_recent}.
+//
+// One CTA of 128 threads per (layer, batch row, kv head, key split).  It serves the G * w_last query rows of
+// the kv head in blocks of 32 rows; for each block it walks the split in tiles of 16 KB of K rows (two tiles in
+// shared memory, the next one copied under the arithmetic of this one):
+//   scores      a thread owns one key of the tile and a share of the block's rows.  It walks its K row starting
+//               at element `key` and wrapping around (the 32 rows of a warp, a multiple of 128 bytes apart,
+//               fall into 32 banks); one K element feeds every row of the thread, q (times scale * log2 e)
+//               comes from shared memory at the same rotated index.
+//   statistics  a warp per query row: tile maximum, new running maximum, the tile's sums of 2^(t - M) over all
+//               visible keys and over the window keys, folded into the row's running (M, A, W).
+// A K row is read from memory once per block of rows (from L2 after the first block) instead of once per row.
 #include <cuda_bf16.h>
 
 #include "lt_internal.h"
 
 namespace lt {
+
+namespace {
 
 template <typename T>
 __device__ __forceinline__ float ld_f32(const T* p);
@@ -23,73 +36,176 @@ __device__ __forceinline__ float ld_f32<__nv_bfloat16>(const __nv_bfloat16* p) {
   return __bfloat162float(*p);
 }
 
-// grid (w_last * n_splits, B * Hq, L); block 128.
+__device__ __forceinline__ void copy16_async(void* smem_dst, const void* src, int src_bytes) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void copy_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void copy_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+constexpr int kSgThreads = 128;
+constexpr int kSgRows = 32;           // query rows per pass over the split
+constexpr int kSgTileBytes = 16384;   // K rows of one tile
+
+}  // namespace
+
+// grid (n_splits, B * Hkv, layers of the call); block 128.
 template <typename T, int D>
-__global__ void scores_generic_kernel(ScoreArgs a, LayerTable kf) {
+__global__ void __launch_bounds__(kSgThreads) scores_generic_kernel(ScoreArgs a, LayerTable kf) {
+  constexpr int RB = kSgRows;
+  constexpr int TK = kSgTileBytes / (D * (int)sizeof(T));  // keys per tile: 32, 64 or 128
+  constexpr int ROW = D * (int)sizeof(T), VEC = ROW / 16;
+  constexpr int NRG = kSgThreads / TK;                      // row shares in the score phase
+  constexpr int RPT = RB / NRG;                             // rows per thread
+  static_assert(TK >= 32 && TK <= kSgThreads && kSgThreads % TK == 0 && RB % NRG == 0, "geometry");
+  extern __shared__ __align__(16) uint8_t sg_smem[];
+  uint8_t* tiles = sg_smem;                                             // [2][TK rows of K]
+  float* q_s = reinterpret_cast<float*>(sg_smem + 2 * kSgTileBytes);    // [RB][D] the block's query rows, times scale * log2 e
+  float* sc = q_s + RB * D;                                             // [RB][TK] scores of the tile
+  float* st_M = sc + RB * TK;                                           // [RB] running (M, A, W) of the block's rows
+  float* st_A = st_M + RB;
+  float* st_W = st_A + RB;
   const lt_shape& s = a.s;
-  const int t = blockIdx.x / a.n_splits, sp = blockIdx.x % a.n_splits;
-  const int b = blockIdx.y / s.n_q_heads, hq = blockIdx.y % s.n_q_heads;
+  const int sp = blockIdx.x;
+  const int b = blockIdx.y / s.n_kv_heads, h = blockIdx.y % s.n_kv_heads;
   const int l = a.layer_begin + blockIdx.z;
-  const int G = s.n_q_heads / s.n_kv_heads;
-  const int h = hq / G;
-  __shared__ float qs[D];
-  __shared__ float red[3][128];
-  const T* qp = (const T*)a.q_tail + ((((long long)l * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * D;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) qs[d] = ld_f32<T>(qp + d);
-  __syncthreads();
-  const int i = a.n_ctx - a.w_last + t;  // position of this query; sees keys 0..i
+  const int G = s.n_q_heads / s.n_kv_heads, T_ = a.w_last;
+  const int n_rows = G * T_;  // rows of this kv head: row = g * w_last + t, contiguous in q_tail
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int j0, j1;
-  score_split_range(a, sp, &j0, &j1);
-  j1 = min(i + 1, j1);
+  score_split_range(a, sp, &j0, &j1);  // keys [j0, j1) of this split (j1 <= n_ctx)
+  const int n_tiles = j1 > j0 ? (j1 - j0 + TK - 1) / TK : 0;
   const T* Kl = (const T*)kf.p[l];
-  const int win_lo = s.recent_per_row ? i - s.n_recent + 1 : a.n_ctx - s.n_recent;  // first recent key of this row
-  float M = -INFINITY, A = 0.f, W = 0.f;
-  for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
-    const T* kr = Kl + full_cache_row(s, b, h, j) * D;
-    float dot = 0.f;
-#pragma unroll 8
-    for (int d = 0; d < D; ++d) dot += qs[d] * ld_f32<T>(kr + d);
-    const float tj = dot * a.cs;
-    const float Mn = fmaxf(M, tj);
-    const float corr = exp2f(M - Mn), p = exp2f(tj - Mn);
-    A = A * corr + p;
-    W = W * corr + ((j < s.n_sink || j >= win_lo) ? p : 0.f);
-    M = Mn;
-  }
-  red[0][threadIdx.x] = M;
-  red[1][threadIdx.x] = A;
-  red[2][threadIdx.x] = W;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float Mx = -INFINITY;
-    for (int k = 0; k < 128; ++k) Mx = fmaxf(Mx, red[0][k]);
-    float As = 0.f, Ws = 0.f;
-    if (Mx > -INFINITY) {
-      for (int k = 0; k < 128; ++k) {
-        const float w = exp2f(red[0][k] - Mx);
-        As += w * red[1][k];
-        Ws += w * red[2][k];
-      }
+  const T* qbase = (const T*)a.q_tail + (((long long)l * s.batch + b) * s.n_q_heads + (long long)h * G) * T_ * D;
+  auto fetch_tile = [&](int it) {
+    uint8_t* kt = tiles + (it & 1) * kSgTileBytes;
+    for (int i = tid; i < TK * VEC; i += kSgThreads) {
+      const int r = i / VEC, p = i - r * VEC;
+      const int j = j0 + it * TK + r;
+      const bool valid = j < j1;
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(Kl + full_cache_row(s, b, h, valid ? j : j0) * D);
+      copy16_async(kt + r * ROW + p * 16, src + p * 16, valid ? 16 : 0);
     }
-    float* st = a.stats +
-                ((((((long long)blockIdx.z * s.batch + b) * s.n_q_heads + hq) * a.w_last + t) * a.n_splits) + sp) * 3;
-    st[0] = Mx;
-    st[1] = As;
-    st[2] = Ws;
+  };
+  for (int r0 = 0; r0 < n_rows; r0 += RB) {
+    const int RBn = min(RB, n_rows - r0);
+    for (int i = tid; i < RB * D; i += kSgThreads) q_s[i] = i < RBn * D ? ld_f32<T>(qbase + (long long)r0 * D + i) * a.cs : 0.f;
+    if (tid < RB) {
+      st_M[tid] = -INFINITY;
+      st_A[tid] = 0.f;
+      st_W[tid] = 0.f;
+    }
+    if (n_tiles > 0) fetch_tile(0);
+    copy_commit();
+    for (int it = 0; it < n_tiles; ++it) {
+      if (it + 1 < n_tiles) fetch_tile(it + 1);
+      copy_commit();
+      copy_wait<1>();
+      __syncthreads();  // tile `it` has landed; the block's q rows and state are visible
+      const int tile_j0 = j0 + it * TK;
+      // ---- scores -------------------------------------------------------------------
+      {
+        const int key = tid % TK, rg = tid / TK;
+        if (rg * RPT < RBn) {
+          const T* krow = reinterpret_cast<const T*>(tiles + (it & 1) * kSgTileBytes) + key * D;
+          const float* qr = q_s + rg * RPT * D;
+          float t[RPT];
+#pragma unroll
+          for (int i = 0; i < RPT; ++i) t[i] = 0.f;
+#pragma unroll 4
+          for (int dd = 0; dd < D; ++dd) {
+            const int d = (dd + key) & (D - 1);
+            const float kv = ld_f32<T>(krow + d);
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) t[i] = fmaf(kv, qr[i * D + d], t[i]);
+          }
+          const int j = tile_j0 + key;
+#pragma unroll
+          for (int i = 0; i < RPT; ++i) {
+            const int row = r0 + rg * RPT + i;
+            const int pos = a.n_ctx - T_ + row % T_;  // position of this query: it sees keys 0 .. pos
+            sc[(rg * RPT + i) * TK + key] = (j < j1 && j <= pos) ? t[i] : -INFINITY;
+          }
+        }
+      }
+      __syncthreads();
+      // ---- statistics: a warp per row ---------------------------------------------------
+      for (int r = warp; r < RBn; r += kSgThreads / 32) {
+        const int pos = a.n_ctx - T_ + (r0 + r) % T_;
+        const int win_lo = s.recent_per_row ? pos - s.n_recent + 1 : a.n_ctx - s.n_recent;  // first recent key of this row
+        float v[TK / 32];
+        float m = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) {
+          v[c] = sc[r * TK + lane + 32 * c];
+          m = fmaxf(m, v[c]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (m > -INFINITY) {  // the row sees at least one key of this tile (uniform over the warp)
+          const float Mo = st_M[r];
+          const float Mn = fmaxf(Mo, m);
+          float sa = 0.f, sw = 0.f;
+#pragma unroll
+          for (int c = 0; c < TK / 32; ++c) {
+            const int j = tile_j0 + lane + 32 * c;
+            const float p = exp2f(v[c] - Mn);
+            sa += p;
+            sw += (j < s.n_sink || j >= win_lo) ? p : 0.f;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            sa += __shfl_xor_sync(0xffffffffu, sa, o);
+            sw += __shfl_xor_sync(0xffffffffu, sw, o);
+          }
+          if (lane == 0) {
+            const float corr = exp2f(Mo - Mn);  // 0 while the row has seen nothing yet
+            st_M[r] = Mn;
+            st_A[r] = st_A[r] * corr + sa;
+            st_W[r] = st_W[r] * corr + sw;
+          }
+        }
+      }
+      __syncthreads();  // the stage and the scores are free for the tile after next
+    }
+    copy_wait<0>();
+    if (tid < RBn) {
+      const int row = r0 + tid;
+      const int hq = h * G + row / T_, t = row % T_;
+      float* st = a.stats +
+                  ((((((long long)blockIdx.z * s.batch + b) * s.n_q_heads + hq) * T_ + t) * a.n_splits) + sp) * 3;
+      st[0] = st_M[tid];
+      st[1] = st_A[tid];
+      st[2] = st_W[tid];
+    }
+    __syncthreads();  // q and the state are rewritten by the next block of rows
   }
 }
 
+template <typename T, int D>
+static cudaError_t launch_scores_generic_variant(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
+  constexpr int TK = kSgTileBytes / (D * (int)sizeof(T));
+  constexpr int smem = 2 * kSgTileBytes + (kSgRows * D + kSgRows * TK + 3 * kSgRows) * 4;
+  auto kern = scores_generic_kernel<T, D>;
+  // the same value on every call, so concurrent first calls from several host threads agree
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(a.n_splits, a.s.batch * a.s.n_kv_heads, a.layer_count);
+  kern<<<grid, kSgThreads, smem, st>>>(a, kf);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
-  dim3 grid(a.w_last * a.n_splits, a.s.batch * a.s.n_q_heads, a.layer_count);
   const bool bf = a.s.dtype == LT_BF16;
   if (a.s.head_dim == 128) {
-    if (bf) scores_generic_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(a, kf);
-    else scores_generic_kernel<float, 128><<<grid, 128, 0, st>>>(a, kf);
-  } else {
-    if (bf) scores_generic_kernel<__nv_bfloat16, 64><<<grid, 128, 0, st>>>(a, kf);
-    else scores_generic_kernel<float, 64><<<grid, 128, 0, st>>>(a, kf);
+    return bf ? launch_scores_generic_variant<__nv_bfloat16, 128>(a, kf, st)
+              : launch_scores_generic_variant<float, 128>(a, kf, st);
   }
-  return cudaGetLastError();
+  return bf ? launch_scores_generic_variant<__nv_bfloat16, 64>(a, kf, st)
+            : launch_scores_generic_variant<float, 64>(a, kf, st);
 }
 
 // One warp per (layer, b, hq): lane t, t + 32, ... merges the statistics slots of its tail rows and takes the
