@@ -460,7 +460,8 @@ def run_ours(args):
 def run_variants(wl, mask_hybrid):
     """The same decode step on the same stack shape with (a) paged full caches
     (128-token pages behind a shuffled block table) and (b) FP8 E4M3 caches with
-    per-layer scales.  Contents are random: the work does not depend on them.
+    per-layer scales; also with head_dim 64, with a query group of 16 and with fp32 caches
+    (the CUDA-core kernels).  Contents are random: the work does not depend on them.
     Reported in `detail`; the headline stays the contiguous bf16 stack."""
     cfg, lt, dev = wl.cfg, wl.lt, wl.device
     L, B, Hq, Hkv, D = cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
@@ -579,6 +580,48 @@ def run_variants(wl, mask_hybrid):
     b16 = algorithmic_bytes_decode(cfg16, n_mean, cfg.n_lazy)
     res["group_16"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b16 / (ms * 1e-3) / 1e9}
     del k16, v16, ks16, vs16, ws16, tables16
+    # (e) fp32 caches (8 layers of the same head shape, every other one lazy): the CUDA-core kernels
+    L32 = 8
+    cfg32 = cfg.scaled(n_layers=L32, dtype="f32")
+    shape32 = lt.Shape(L32, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_F32)
+    mk32 = lambda n: [torch.randn((B, Hkv, n, D), device=dev) for _ in range(L32)]  # noqa: E731
+    k32, v32, ks32, vs32 = mk32(cap), mk32(cap), mk32(C), mk32(C)
+    tables32 = lt.LayerTables(shape32, k32, v32, ks32, vs32)
+    ws32 = torch.empty(lt.workspace_bytes(shape32, cfg.n_ctx, T), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws32)
+    q32 = torch.randn((L32, B, Hq, D), device=dev)
+    kn32 = torch.randn((L32, B, Hkv, D), device=dev)
+    out32 = torch.zeros((L32, B, Hq, D), device=dev)
+    mask32 = torch.zeros(L32, dtype=torch.uint8, device=dev)
+    mask32[1::2] = 1
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
+    for _ in range(2):
+        lt.decode_step(shape32, q32, kn32, kn32, tables32, mask32, seq, out32, ws32)
+    torch.cuda.synchronize()
+    seq.fill_(cfg.n_ctx)
+    e0.record()
+    for _ in range(8):
+        lt.decode_step(shape32, q32, kn32, kn32, tables32, mask32, seq, out32, ws32)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws32) == 0
+    ms = e0.elapsed_time(e1) / 8
+    b32 = algorithmic_bytes_decode(cfg32, cfg.n_ctx + 4.5, L32 // 2)
+    res["fp32_caches_8_layers"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b32 / (ms * 1e-3) / 1e9,
+                                   "frac_of_nominal_8TBs": b32 / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
+    qt32 = torch.randn((L32, B, Hq, T, D), device=dev)
+    sc32 = torch.zeros((L32, B, Hq), dtype=torch.float32, device=dev)
+    lt.lazy_scores(shape32, qt32, tables32, cfg.n_ctx, T, sc32, ws32)
+    torch.cuda.synchronize()
+    e0.record()
+    lt.lazy_scores(shape32, qt32, tables32, cfg.n_ctx, T, sc32, ws32)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws32) == 0
+    ms = e0.elapsed_time(e1)
+    res["fp32_caches_8_layers"]["lazy_scores_ms"] = ms
+    res["fp32_caches_8_layers"]["lazy_scores_fp32_tflops"] = 2.0 * L32 * B * Hq * T * cfg.n_ctx * D / (ms * 1e-3) / 1e12
+    del k32, v32, ks32, vs32, ws32, tables32, qt32
     return res
 
 
