@@ -355,7 +355,7 @@ def run_ours(args):
     del lse
 
     # ---- the scoring kernel alone against its three roofs (HBM, tensor, MUFU) -------------
-    n_it = 80
+    n_it = 400                         # about 2.4 s: long enough for the 200 ms clock and power samples to see the loop alone
     s_sampler = ClockSampler(gpu_index)
     torch.cuda.synchronize()
     s_sampler.start()
