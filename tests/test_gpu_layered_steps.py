@@ -186,3 +186,52 @@ def test_captured_overlapped_step_replays():
     assert torch.equal(graph.seq_lens, eager.seq_lens) and lt.check(graph.ws) == 0
     for l in range(L):
         assert torch.equal(graph.k_full[l], eager.k_full[l]) and torch.equal(graph.k_stream[l], eager.k_stream[l])
+
+
+def test_overlapped_launches_with_paged_fp8_caches_and_per_prompt_masks():
+    """The deployment options together (block tables, 8-bit caches, a mask row per prompt): overlapped per-layer
+    launches still equal the plain-order chain bit for bit (their parity with the oracle is covered where each
+    option is tested on its own)."""
+    torch.manual_seed(51)
+    L, B, Hq, Hkv, D, S, R, page, pps = 6, 3, 16, 2, 128, 4, 60, 128, 40
+    cap, n_pages, steps = page * pps, 3 * 40 + 5, 8
+    lens = [4990, 2100, 129]
+    scales = torch.full((L, 2), 0.03, dtype=torch.float32, device="cuda")
+    table = torch.randperm(n_pages)[: B * pps].view(B, pps).to(torch.int32).cuda().contiguous()
+    mask = torch.tensor([[0, 1, 0, 0, 1, 0], [1, 0, 0, 1, 0, 0], [0, 0, 1, 1, 0, 1]], dtype=torch.uint8).cuda()
+    pools = [torch.randint(0, 120, (n_pages, Hkv, page, D), dtype=torch.uint8) for _ in range(2 * L)]
+    rings = [torch.randint(0, 120, (B, Hkv, S + R, D), dtype=torch.uint8) for _ in range(2 * L)]
+    shape = lt.Shape(L, B, Hq, Hkv, D, S, R, cap, lt.LT_BF16, 0.0, per_sequence_mask=1, page_size=page, pages_per_seq=pps,
+                     n_pages=n_pages, block_table=table, kv_fp8=1, kv_scales=scales)
+    state = []
+    for layered in (False, True):
+        kf = [p.clone().cuda() for p in pools[:L]]; vf = [p.clone().cuda() for p in pools[L:]]
+        ks = [p.clone().cuda() for p in rings[:L]]; vs = [p.clone().cuda() for p in rings[L:]]
+        tabs = lt.LayerTables(shape, kf, vf, ks, vs)
+        nbytes = lt.workspace_bytes_layers(shape) if layered else lt.workspace_bytes(shape)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda"); lt.workspace_init(ws)
+        seq = torch.tensor(lens, dtype=torch.int32, device="cuda")
+        state.append((kf, vf, ks, vs, tabs, ws, seq))
+    g = torch.Generator().manual_seed(52)
+    outs = ([], [])
+    for t in range(steps):
+        q = torch.randn(L, B, Hq, D, generator=g).bfloat16().cuda()
+        k = torch.randn(L, B, Hkv, D, generator=g).bfloat16().cuda()
+        v = torch.randn(L, B, Hkv, D, generator=g).bfloat16().cuda()
+        for which, (kf, vf, ks, vs, tabs, ws, seq) in enumerate(state):
+            out = torch.full((L, B, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
+            for l in range(L):
+                if which:
+                    lt.decode_step_layers(shape, q, k, v, tabs, mask, seq, out, ws, layer_begin=l,
+                                          advance_seq_lens=(l == L - 1), independent_of_previous=(l > 0))
+                else:
+                    lt.decode_step(shape, q, k, v, tabs, mask, seq, out, ws, layer_begin=l, layer_count=1,
+                                   advance_seq_lens=(l == L - 1))
+            outs[which].append(out)
+    torch.cuda.synchronize()
+    for t in range(steps):
+        assert torch.isfinite(outs[0][t]).all() and torch.equal(outs[1][t], outs[0][t]), t
+    for a, b in zip(state[0][:4], state[1][:4]):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    assert torch.equal(state[0][6], state[1][6]) and lt.check(state[0][5]) == 0 and lt.check(state[1][5]) == 0
