@@ -580,6 +580,30 @@ def run_variants(wl, mask_hybrid):
     b16 = algorithmic_bytes_decode(cfg16, n_mean, cfg.n_lazy)
     res["group_16"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b16 / (ms * 1e-3) / 1e9}
     del k16, v16, ks16, vs16, ws16, tables16
+    # ... and a group of 32 (64 q / 2 kv heads): the four warps share every tile and serve eight heads each
+    cfg32g = cfg.scaled(n_q_heads=64, n_kv_heads=2)
+    shape32g = lt.Shape(L, B, 64, 2, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16)
+    k16, v16, ks16, vs16 = mk16(cap), mk16(cap), mk16(C), mk16(C)
+    tables32g = lt.LayerTables(shape32g, k16, v16, ks16, vs16)
+    ws32g = torch.empty(lt.workspace_bytes(shape32g), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws32g)
+    q32g = torch.randn((L, B, 64, D), device=dev).bfloat16()
+    out32g = torch.zeros_like(q32g)
+    seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        lt.decode_step(shape32g, q32g, kn16, kn16, tables32g, mask_hybrid, seq, out32g, ws32g)
+    torch.cuda.synchronize()
+    seq.fill_(cfg.n_ctx)
+    e0.record()
+    for _ in range(16):
+        lt.decode_step(shape32g, q32g, kn16, kn16, tables32g, mask_hybrid, seq, out32g, ws32g)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws32g) == 0
+    ms = e0.elapsed_time(e1) / 16
+    b32g = algorithmic_bytes_decode(cfg32g, n_mean, cfg.n_lazy)
+    res["group_32"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs": b32g / (ms * 1e-3) / 1e9}
+    del k16, v16, ks16, vs16, ws32g, tables32g
     # (e) fp32 caches (8 layers of the same head shape, every other one lazy): the CUDA-core kernels
     L32 = 8
     cfg32 = cfg.scaled(n_layers=L32, dtype="f32")

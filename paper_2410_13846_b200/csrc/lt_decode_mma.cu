@@ -1,5 +1,5 @@
-// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 16 (groups above 8 by
-// warp pairs: template branch PAIR);
+// Decode step, bandwidth path: bf16 activations, head_dim 128 or 64, GQA group <= 32 (groups above 8 by
+// warps that share a tile ring and serve eight heads each: template parameter ROLES);
 // caches in bf16 or (template branch FP8, head_dim 128) in E4M3 bytes.
 //
 // A persistent launch (two CTAs per SM) walks the flattened work list of
@@ -162,16 +162,21 @@ struct TileSrc {
 // 16-byte column c of K row r sits at column c ^ (r & 7), of V row r at
 // c ^ (r & 7) ^ (4 * ((r >> 3) & 1)): the eight rows of either ldmatrix phase fall into eight different bank groups.
 //
-// PAIR = true (query groups of 9..16 heads): the four warps work as two pairs.  The warps of a pair walk the same
+// ROLES = 2 (query groups of 9..16 heads): the four warps work as two pairs.  The warps of a pair walk the same
 // tiles through one shared ring (each copies half of every tile, a 64-thread named barrier per tile makes the
 // copies visible and frees the stage that is refilled), warp 0 of the pair serves heads 0-7 of the group and warp
 // 1 heads 8-15, so the chunk still crosses HBM, L2 and shared memory once.
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, bool PAIR>
+// ROLES = 4 (groups of 17..32 heads, 16-bit caches): all four warps walk one ring of twice the depth (a quarter of
+// every tile each, one 128-thread named barrier per tile); warp w serves heads 8w .. 8w + 7 - a warp beyond the
+// group's last head computes on zeros and stores nothing - and no sums cross warps.
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, int ROLES>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
   static_assert(DH == 128 || (DH == 64 && !FP8), "head_dim 128, or 64 with 16-bit caches");
-  constexpr int STREAMS = PAIR ? WARPS / 2 : WARPS;   // independent tile streams of the CTA
+  static_assert(ROLES == 1 || ROLES == 2 || (ROLES == 4 && !FP8), "one, two or four warps per tile stream");
+  constexpr bool PAIR = ROLES > 1;                    // several warps share a ring, eight heads of the group each
+  constexpr int STREAMS = WARPS / ROLES;              // independent tile streams of the CTA
   constexpr int RSTAGES = NSTAGE;                     // ring stages of a stream
   constexpr int kD = DH;                       // head_dim
   constexpr int kSrcRowBytes = kD * 2;         // one row of q, k_new, v_new (bf16)
@@ -206,11 +211,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gp = lane >> 2, c = lane & 3;  // fragment row / column-pair index
-  const int stream = PAIR ? warp >> 1 : warp;  // tile stream of this warp
-  const int role = PAIR ? warp & 1 : 0;        // pair: which eight heads of the group this warp serves
+  const int stream = warp / ROLES;  // tile stream of this warp
+  const int role = warp % ROLES;    // which eight heads of the group this warp serves
   const uint32_t wsm = smem_u32(smem) + stream * STREAM_BYTES;
   auto stream_sync = [&]() {  // the threads that share a ring: the warp, or the 64 threads of a pair
-    if constexpr (PAIR) {
+    if constexpr (ROLES == 4) {
+      asm volatile("bar.sync 1, 128;\n" ::: "memory");
+    } else if constexpr (ROLES == 2) {
       if (stream == 0) asm volatile("bar.sync 1, 64;\n" ::: "memory");
       else asm volatile("bar.sync 2, 64;\n" ::: "memory");
     } else {
@@ -283,7 +290,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   // offset of every pass is the first one xor a constant.
   constexpr int VPRX = FP8 ? 8 : VPR;             // 16-byte vectors of a cached row
   constexpr int RPI = 32 / VPRX;
-  constexpr int FROWS = PAIR ? TILE / 2 : TILE;   // rows of a tile this warp copies (a pair's warps: half each)
+  constexpr int FROWS = TILE / ROLES;             // rows of a tile this warp copies (the warps of a ring share them out)
   const int f_row = role * FROWS + lane / VPRX;
   const int f_p = lane % VPRX;
   const uint32_t f_goff = f_row * kRowBytes + f_p * 16;
@@ -331,7 +338,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
         }
       }
     } else {
-      constexpr int ROWS = PAIR ? TILE / 2 : TILE;  // a pair's warps copy half a tile each
+      constexpr int ROWS = TILE / ROLES;  // the warps of a ring copy an equal share of the tile each
 #pragma unroll
       for (int i = 0; i < ROWS * VPR / 32; ++i) {
         const int r = role * ROWS + (32 / VPR) * i + lane / VPR;
@@ -381,7 +388,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     const int l = w.l, b = w.b, h = w.h;
     // query heads served by this warp: the group, or this warp's eight of a pair's sixteen
     const int g0 = role * 8;
-    const int Gn = PAIR ? min(8, G - role * 8) : G;
+    const int Gn = PAIR ? max(0, min(8, G - role * 8)) : G;
     const int j1 = src_cur.j1;
     int fetched_next = 0;
     if (threadIdx.x == 0) fetched_next = 2 * gridDim.x + atomicAdd(a.work_counter, 1);
@@ -637,8 +644,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     __syncthreads();  // (max, sum) of every warp and the next item index are visible
     const int after_next = s_next;
     // the warps whose results belong to the same heads: all four, or (pairs) the two of this warp's role
-    constexpr int W0_STEP = PAIR ? 2 : 1;
-    const int w_first = PAIR ? role : 0;
+    constexpr int W0_STEP = ROLES;
+    const int w_first = role;
     float Mx0 = -INFINITY, Mx1 = -INFINITY;
 #pragma unroll
     for (int ww = w_first; ww < WARPS; ww += W0_STEP) {
@@ -666,7 +673,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     }
     // rows of heads 2c (and 2c + 1 at + kD) of a warp's O in merge buffer `which`
     auto buf_at = [&](int which, int) { return sm_buf + which * (8 * kD) + (2 * c) * kD; };
-    if (warp >= 2) {
+    // (four roles: every warp holds the whole sum of its own eight heads, nothing to add)
+    if (ROLES < 4 && warp >= 2) {
 #pragma unroll
       for (int dt = 0; dt < NK; ++dt) {
         float* p = buf_at(warp - 2, dt);
@@ -677,7 +685,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       }
     }
     __syncthreads();
-    if (warp < 2) {
+    if (ROLES < 4 && warp < 2) {
 #pragma unroll
       for (int dt = 0; dt < NK; ++dt) {
         const float* p = buf_at(warp, dt);
@@ -702,8 +710,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       __syncthreads();
     }
     const bool single = w.nc <= 1;  // the whole (layer, b, kv head) is this one chunk
-    // the warp that holds the item's sum: warp 0, or (pairs) warps 0 and 1 with eight heads each
-    if (PAIR ? warp < 2 : warp == 0) {
+    // the warps that hold the item's sum: warp 0, or one warp per role with eight heads each
+    if (warp < ROLES) {
       if constexpr (!PAIR) {
 #pragma unroll
         for (int dt = 0; dt < NK; ++dt) {
@@ -777,20 +785,20 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   finish_launch(a);
 }
 bool decode_mma_supported(const lt_shape& s) {
-  // groups of 9..16: two warps per tile, eight heads each
+  // groups of 9..16: two warps per tile, eight heads each; 17..32 (16-bit caches): four warps per tile
   return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
-         (s.n_q_heads / s.n_kv_heads) <= 16;
+         (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 16 : 32);
 }
 
-template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, bool PAIR>
+template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, int ROLES>
 static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st) {
-  constexpr int streams = PAIR ? WARPS / 2 : WARPS;
+  constexpr int streams = WARPS / ROLES;
   constexpr int ring = FP8 ? streams * NSTAGE * TILE * 256 : streams * NSTAGE * TILE * 4 * DH;
   constexpr int merge = 2 * 8 * DH * 4 + 2 * WARPS * 8 * 4;
   static_assert(2 * 8 * DH * 4 >= kCombineStagePairs * 8, "the merge buffers double as the combine staging area");
   const int smem = ring + merge + worklist_smem_bytes(a.layer_count * a.s.batch, a.s.batch);
-  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8, DH, PAIR>;
+  auto kern = decode_mma_kernel<TILE, NSTAGE, WARPS, MINB, FP8, DH, ROLES>;
   // Per device, behind a lock (host threads may issue their first calls concurrently): the dynamic
   // shared-memory limit is raised once to the largest size any launch of this variant can ask for, and
   // the occupancy of each shared-memory size met so far is remembered (host time matters for per-layer callers).
@@ -830,17 +838,22 @@ static cudaError_t launch_variant(const DecodeArgs& a, const LayerTable& kf, con
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf, const LayerTable& ks,
                               const LayerTable& vs, cudaStream_t st) {
-  const bool pair = a.s.n_q_heads / a.s.n_kv_heads > 8;  // groups of 9..16: two warps per tile, eight heads each
+  const int G = a.s.n_q_heads / a.s.n_kv_heads;
+  const bool pair = G > 8;   // groups of 9..16: two warps per tile, eight heads each
+  const bool quad = G > 16;  // groups of 17..32: the four warps share one ring of twice the depth
   // 8-bit caches: raw stages of 32 keys (8 KB); a warp's three stages or a pair's six hold what the 16-bit ring holds
   if (a.s.kv_fp8)
-    return pair ? launch_variant<32, 6, 4, 2, true, 128, true>(a, kf, vf, ks, vs, st)
-                : launch_variant<32, 3, 4, 2, true, 128, false>(a, kf, vf, ks, vs, st);
+    return pair ? launch_variant<32, 6, 4, 2, true, 128, 2>(a, kf, vf, ks, vs, st)
+                : launch_variant<32, 3, 4, 2, true, 128, 1>(a, kf, vf, ks, vs, st);
   // head_dim 64: rows are half as long, so 32-key tiles keep the bytes in flight per warp (24 KB) the same
-  if (a.s.head_dim == 64)
-    return pair ? launch_variant<32, 6, 4, 2, false, 64, true>(a, kf, vf, ks, vs, st)
-                : launch_variant<32, 3, 4, 2, false, 64, false>(a, kf, vf, ks, vs, st);
-  return pair ? launch_variant<32, 3, 4, 2, false, 128, true>(a, kf, vf, ks, vs, st)
-              : launch_variant<16, 3, 4, 2, false, 128, false>(a, kf, vf, ks, vs, st);
+  if (a.s.head_dim == 64) {
+    if (quad) return launch_variant<32, 12, 4, 2, false, 64, 4>(a, kf, vf, ks, vs, st);
+    return pair ? launch_variant<32, 6, 4, 2, false, 64, 2>(a, kf, vf, ks, vs, st)
+                : launch_variant<32, 3, 4, 2, false, 64, 1>(a, kf, vf, ks, vs, st);
+  }
+  if (quad) return launch_variant<32, 6, 4, 2, false, 128, 4>(a, kf, vf, ks, vs, st);
+  return pair ? launch_variant<32, 3, 4, 2, false, 128, 2>(a, kf, vf, ks, vs, st)
+              : launch_variant<16, 3, 4, 2, false, 128, 1>(a, kf, vf, ks, vs, st);
 }
 
 }  // namespace lt

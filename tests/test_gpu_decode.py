@@ -41,14 +41,18 @@ def _oracle_out(st, q, hist_k, hist_v, lens, mask):
 
 
 CASES = [
-    # dtype, D, Hq, Hkv, S, R, lens, scale              (bf16/128/G<=8 -> tensor-core path)
+    # dtype, D, Hq, Hkv, S, R, lens, scale              (bf16, G <= 32 -> tensor-core path)
     (torch.bfloat16, 128, 8, 2, 4, 60, [300, 1, 64, 65, 17], 0.0),          # G=4, ragged, n<S+R, exactly S+R
     (torch.bfloat16, 128, 5, 1, 4, 28, [2049, 2048, 2047, 33], 0.0),        # G=5, chunk boundaries
     (torch.bfloat16, 128, 2, 2, 0, 16, [100, 16, 3], 0.11),                 # G=1, no sink, custom scale
     (torch.bfloat16, 128, 16, 2, 2, 6, [700, 5], 0.0),                      # G=8
     (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40], 0.0),                    # G=16: warp pairs, eight heads per warp
     (torch.bfloat16, 128, 12, 1, 4, 28, [4200, 2049, 65], 0.0),             # G=12: warps of a pair serve 8 and 4 heads, several chunks
-    (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40], 0.0),                    # G=20 -> CUDA-core path
+    (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40], 0.0),                    # G=20: four warps per tile; the third serves 4 heads, the fourth none
+    (torch.bfloat16, 128, 32, 1, 4, 28, [4200, 2049, 65, 0], 0.0),          # G=32: four warps per tile, eight heads each, several chunks
+    (torch.bfloat16, 128, 17, 1, 0, 16, [300, 31], 0.0),                    # G=17: one head in the third warp
+    (torch.bfloat16, 64, 24, 1, 4, 28, [2049, 2047, 33, 4500], 0.0),        # D=64, G=24: four warps over a twelve-stage ring
+    (torch.bfloat16, 128, 40, 1, 4, 12, [130, 40], 0.0),                    # G=40 -> CUDA-core path, five passes of eight heads
     (torch.bfloat16, 64, 4, 2, 4, 60, [257, 90], 0.0),                      # D=64: 32-key tiles of 128-byte rows
     (torch.bfloat16, 64, 8, 1, 4, 28, [2049, 2048, 2047, 33, 4500], 0.0),   # D=64, G=8, chunk boundaries
     (torch.bfloat16, 64, 16, 1, 4, 28, [300, 2100], 0.0),                   # D=64, G=16: warp pairs

@@ -32,7 +32,10 @@ CASES = [
     (torch.bfloat16, 128, 8, 2, 4, 28, [300, 1, 0, 31, 32, 2047], 40),      # tensor-core path; wraps; n = 0 start
     (torch.bfloat16, 128, 5, 1, 0, 16, [2040, 15], 20),                    # G=5, no sink, chunk boundary crossed
     (torch.bfloat16, 128, 32, 2, 4, 12, [130, 40, 2040], 20),              # G=16: warp pairs; the fused append stores the new row once
-    (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40], 20),                    # G=20 -> CUDA-core path
+    (torch.bfloat16, 128, 40, 2, 4, 12, [130, 40, 2040], 20),              # G=20: four warps per tile (8, 8, 4, 0 heads); chunk boundary crossed
+    (torch.bfloat16, 128, 32, 1, 4, 28, [300, 1, 0, 2047], 40),            # G=32: four warps per tile; wraps; the new row is stored once
+    (torch.bfloat16, 64, 32, 1, 0, 16, [2040, 15], 20),                    # head_dim 64, G=32
+    (torch.bfloat16, 128, 40, 1, 4, 12, [130, 40], 20),                    # G=40 -> CUDA-core path
     (torch.bfloat16, 64, 8, 2, 4, 28, [300, 1, 0, 31, 32, 2047], 40),      # head_dim 64 on the tensor-core path; wraps
     (torch.bfloat16, 64, 5, 1, 0, 16, [2040, 15], 20),                     # head_dim 64, G=5, chunk boundary crossed
     (torch.float32, 64, 4, 2, 4, 60, [513, 3], 70),                        # fp32, D=64
