@@ -40,6 +40,11 @@
  *   - A decode step is "append, then attend": the new token attends to itself
  *     (causal mask with i >= j, Appendix E).
  *   - GQA: query head hq reads kv head hq / (n_q_heads / n_kv_heads).
+ *   - Every shape the calls accept is computed on the GPU by this library's own
+ *     kernels.  The bandwidth-bound tensor-core kernels serve bf16 stacks with
+ *     head_dim 64 or 128 (decode: query groups of up to 32 heads, up to 16 with
+ *     8-bit caches; scoring: any group); fp32 stacks and larger groups run on
+ *     tiled CUDA-core kernels, several times slower per byte.
  */
 #ifndef LT_H_
 #define LT_H_
