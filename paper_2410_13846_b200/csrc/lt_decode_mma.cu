@@ -497,6 +497,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
       const uint32_t st = wsm + (consumed % RSTAGES) * RING_STAGE;
       ++consumed;
       const int key_base = src_cur.j0 + (stream + it * STREAMS) * TILE;
+      // a warp whose eight heads lie beyond the group (four roles, groups of 17..24) only copies its share of the tiles
+      if (ROLES == 4 && Gn == 0) continue;
 
       // ---- S^T = K Q^T ------------------------------------------------------
       float sc[MT][4];
