@@ -512,7 +512,24 @@ def run_variants(wl, mask_hybrid):
     ms = time_steps(shape8, tables8, ws8, cfg.n_ctx)
     kv8 = algorithmic_bytes_decode(cfg, n_mean, cfg.n_lazy) / 2          # one byte per cached element
     res["fp8_caches"] = {"step_ms": ms, "decode_tokens_per_s": B / (ms * 1e-3), "gbs_of_8bit_bytes": kv8 / (ms * 1e-3) / 1e9}
-    del k8, v8, ks8, vs8, ws8, tables8
+    # ... and the lazy scores over the whole prompt read from the 8-bit keys (E4M3 MMAs on the stored bytes)
+    del ws8
+    T8 = cfg.w_last
+    ws8 = torch.empty(lt.workspace_bytes(shape8, cfg.n_ctx, T8), dtype=torch.uint8, device=dev)
+    lt.workspace_init(ws8)
+    sc8 = torch.zeros((L, B, Hq), dtype=torch.float32, device=dev)
+    for _ in range(2):
+        lt.lazy_scores(shape8, wl.q_tail, tables8, cfg.n_ctx, T8, sc8, ws8)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        lt.lazy_scores(shape8, wl.q_tail, tables8, cfg.n_ctx, T8, sc8, ws8)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lt.check(ws8) == 0 and bool(torch.isfinite(sc8).all())
+    res["fp8_caches"]["lazy_scores_ms"] = e0.elapsed_time(e1) / 20
+    del k8, v8, ks8, vs8, ws8, tables8, sc8
     # (c) the same stack with head_dim 64 (bf16): half the bytes per token, 32-key tiles of 128-byte rows
     shape64 = lt.Shape(L, B, Hq, Hkv, 64, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16)
     mk64 = lambda n: [torch.randn((B, Hkv, n, 64), device=dev).bfloat16() for _ in range(L)]  # noqa: E731

@@ -115,7 +115,10 @@ typedef struct lt_shape {
      dtype = LT_BF16, head_dim = 128 and a query group of at most 16.  The kernels turn the stored bytes into
      f16 in registers (exact) and multiply on the tensor cores with fp32 accumulation, q as f16 at one
      power-of-two scale per head (exact for bf16 inputs), the probabilities as one f16 term.  lt_lazy_scores and
-     lt_lazy_scores_lse do not read 8-bit keys: score from the prefill's 16-bit keys with a shape whose kv_fp8 is 0. */
+     lt_lazy_scores_lse read 8-bit keys too (k_full holds the E4M3 bytes; q_tail stays bf16): the stored bytes go
+     through E4M3 tensor-core MMAs against q as two E4M3 terms per element at one power-of-two scale per query
+     row (exact for bf16 inputs down to 2^-10 of the row's largest value), which the call writes into the
+     workspace; size the workspace with this shape (lt_workspace_bytes adds the room for it). */
   int32_t kv_fp8;
   int32_t reserved2_;      /* must be 0 */
   const float* kv_scales;  /* dev float [n_layers][2] (K scale, V scale), positive; read during device work */

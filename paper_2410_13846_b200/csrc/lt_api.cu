@@ -143,6 +143,12 @@ ScorePlan make_score_plan(const lt_shape& s, int n_ctx, int w_last, bool window_
   return p;
 }
 
+size_t score_q8_bytes(const lt_shape& s, int w_last) {
+  if (!s.kv_fp8 || w_last < 1) return 0;
+  const size_t rows = (size_t)s.n_layers * s.batch * s.n_q_heads * w_last;
+  return round_up(2 * rows * s.head_dim, kWsAlign) + round_up(rows * sizeof(float), kWsAlign);
+}
+
 size_t ws_prefix_bytes(const lt_shape& s) {
   const size_t counters = ((size_t)s.n_layers * s.batch * s.n_kv_heads + 2 * (size_t)s.n_layers) * sizeof(int);
   return kWsHeaderBytes + round_up(counters, kWsAlign);
@@ -243,6 +249,7 @@ lt_status lt_workspace_bytes(const lt_shape* shape, int32_t n_ctx_max, int32_t w
     const ScorePlan sp = make_score_plan(*shape, n_ctx_max, w_last_max, false);
     const ScorePlan sw = make_score_plan(*shape, n_ctx_max, w_last_max, true);
     score_bytes = round_up((sp.stat_floats > sw.stat_floats ? sp.stat_floats : sw.stat_floats) * 4, kWsAlign);
+    score_bytes += score_q8_bytes(*shape, w_last_max);  // 8-bit keys: the call's two-term copy of q_tail
   }
   *bytes_out = ws_prefix_bytes(*shape) + (decode_bytes > score_bytes ? decode_bytes : score_bytes);
   return LT_OK;
@@ -283,7 +290,8 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   if (st != LT_OK) return st;
   if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
   if (window_only && !lse) return LT_ERR_INVALID_ARG;
-  if (shape->kv_fp8) return LT_ERR_UNSUPPORTED;  // scoring reads 16- or 32-bit keys only
+  // 8-bit keys are scored by the tensor-core kernel only (E4M3 MMAs on the stored bytes)
+  if (shape->kv_fp8 && !scores_umma_supported(*shape, w_last)) return LT_ERR_UNSUPPORTED;
   if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
   if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0) return LT_ERR_INVALID_ARG;
   if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
@@ -316,7 +324,8 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   }
   if (!ws || ((uintptr_t)ws % kWsAlign) != 0) return LT_ERR_WORKSPACE;
   const size_t prefix = ws_prefix_bytes(*shape);
-  if (ws_bytes < prefix + round_up(sp.stat_floats * 4, kWsAlign)) return LT_ERR_WORKSPACE;
+  const size_t stat_bytes = round_up(sp.stat_floats * 4, kWsAlign);
+  if (ws_bytes < prefix + stat_bytes + score_q8_bytes(*shape, w_last)) return LT_ERR_WORKSPACE;
   a.s = *shape;
   a.q_tail = q_tail;
   a.lse = lse;
@@ -331,6 +340,11 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   a.scores = scores;
   a.cs = resolved_scale(*shape) * 1.4426950408889634f;
   a.dev_err = err_word(ws);
+  if (shape->kv_fp8) {
+    a.q8_rows = (long long)shape->n_layers * shape->batch * shape->n_q_heads * w_last;
+    a.q8 = reinterpret_cast<uint8_t*>((char*)ws + prefix + stat_bytes);
+    a.q8_scale = reinterpret_cast<float*>(a.q8 + round_up(2 * (size_t)a.q8_rows * shape->head_dim, kWsAlign));
+  }
   cudaStream_t cs = (cudaStream_t)stream;
   cudaError_t e = umma ? launch_scores_umma(a, kf, cs) : launch_scores_generic(a, kf, cs);
   if (e != cudaSuccess) return LT_ERR_CUDA;

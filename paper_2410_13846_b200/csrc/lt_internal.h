@@ -193,7 +193,14 @@ struct ScoreArgs {
   float* stats;  // workspace
   float* scores;
   uint32_t* dev_err;
+  // 8-bit keys (tensor-core path): q_tail as two E4M3 terms per element, q = q8_scale[row] * (hi + lo), made by
+  // the call itself in the workspace: q8 holds the hi rows [q8_rows][head_dim], then the lo rows
+  uint8_t* q8;
+  float* q8_scale;     // [q8_rows]
+  long long q8_rows;   // n_layers * batch * n_q_heads * w_last
 };
+// Workspace bytes of the two-term query copy for w_last tail queries (0 unless the caches are 8-bit).
+size_t score_q8_bytes(const lt_shape& s, int w_last);
 // Key range [*k0, *k1) of split sp (see ScorePlan).
 __host__ __device__ inline void score_split_range(const ScoreArgs& a, int sp, int* k0, int* k1) {
   if (!a.window_only) {

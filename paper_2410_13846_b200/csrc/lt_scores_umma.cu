@@ -61,6 +61,8 @@
 // is freed and the kernel returns.
 #include <cuda.h>  // CUtensorMap and its enums; the encoder is looked up at run time, nothing links to libcuda
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 
 #include "lt_internal.h"
 
@@ -80,13 +82,18 @@ constexpr int kBarBytes = 256;
 constexpr int kMergeBytes = 2 * 128 * 3 * 4;      // (reference, sum, windowed sum) of 128 rows x two key halves
 // Geometry that depends on the head dimension DH (128 or 64): a row has DH / 64 halves of 128 bytes; the K ring
 // holds 128 KB either way (2 stages of 64 KB, or 4 of 32 KB).
-template <int DH>
+// K8 (8-bit keys, head_dim 128): a K row is one 128-byte span of E4M3 bytes and a tile 32 KB (four stages); the
+// query block comes as two E4M3 terms (q = scale * (hi + lo), see q_split_kernel) of 32 KB each, which take the
+// places of the two 64-d halves of a 16-bit query block, and the contraction runs as four 32-wide k-steps per term.
+template <int DH, bool K8 = false>
 struct Geo {
-  static constexpr int kHalves = DH / 64;
-  static constexpr int kQBytes = kHalves * kQHalfBytes;      // 64 KB or 32 KB
-  static constexpr int kStageBytes = kHalves * kKHalfBytes;  // 64 KB or 32 KB
-  static constexpr int kStages = 4 / kHalves;
-  static constexpr int kKSteps = DH / 16;                    // 16-wide k-steps of the contraction
+  static_assert(!K8 || DH == 128, "8-bit keys: head_dim 128");
+  static constexpr int kHalves = DH / 64;                               // 128-byte spans of a 16-bit row; K8: terms of q
+  static constexpr int kKHalves = K8 ? 1 : kHalves;                     // 128-byte spans of a K row
+  static constexpr int kQBytes = kHalves * kQHalfBytes;                 // 64 KB or 32 KB
+  static constexpr int kStageBytes = kKHalves * kKHalfBytes;            // 64 KB or 32 KB
+  static constexpr int kStages = 4 / kKHalves;
+  static constexpr int kKSteps = DH / 16;                               // MMAs per row block and tile (K8: 2 terms x 4)
   static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kMergeBytes + 1024;  // + alignment slack
 };
 constexpr int kStatWarps = 16;
@@ -165,6 +172,19 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) | ((128u >> 4) << 24);
 
+// The same with A and B in E4M3 (format code 0 in both fields), for tcgen05.mma.kind::f8f6f4: K = 32 per instruction.
+constexpr uint32_t kIdesc8 = (1u << 4) | ((uint32_t)(kBlockN >> 3) << 17) | ((128u >> 4) << 24);
+
+// D[tmem] (+)= A[smem] . B[smem]^T over 32 E4M3 values per row: A a 128-row slice of one term of the query block,
+// B a 256-key slice of the K tile.
+__device__ __forceinline__ void umma_e4m3_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(kIdesc8), "r"(accumulate)
+      : "memory");
+}
 // D[tmem] (+)= A[smem] . B[smem]^T: A a 128-row x 16-d slice of the query block, B a 256-key x 16-d slice of the K tile.
 __device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
   asm volatile(
@@ -377,11 +397,12 @@ __device__ __forceinline__ bool next_piece(const ScoreArgs& a, long long& cursor
   return true;
 }
 
-template <int DH>
+template <int DH, bool K8>
 __global__ void __launch_bounds__(kThreads, 1)
     scores_umma_kernel(ScoreArgs a, const __grid_constant__ KeyMaps maps) {
-  constexpr int kHalves = Geo<DH>::kHalves, kQBytes = Geo<DH>::kQBytes, kStageBytes = Geo<DH>::kStageBytes;
-  constexpr int kStages = Geo<DH>::kStages, kKSteps = Geo<DH>::kKSteps;
+  using G_ = Geo<DH, K8>;
+  constexpr int kHalves = G_::kHalves, kKHalves = G_::kKHalves, kQBytes = G_::kQBytes, kStageBytes = G_::kStageBytes;
+  constexpr int kStages = G_::kStages, kKSteps = G_::kKSteps;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern of the MMA is a function of address bits 4..9
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -463,7 +484,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_expect_tx(bar_qfull, kQBytes);
             const int yq = ((p.l * s.batch + p.b) * s.n_q_heads + p.h * G) * T + p.rb * kBlockM;
 #pragma unroll
-            for (int hf = 0; hf < kHalves; ++hf) tma_load_2d(sQ + hf * kQHalfBytes, &maps.q, 64 * hf, yq, bar_qfull);
+            for (int hf = 0; hf < kHalves; ++hf) {
+              // 16-bit queries: the two 64-d halves of the rows; 8-bit keys: the rows of the two E4M3 terms of q
+              if constexpr (K8) tma_load_2d(sQ + hf * kQHalfBytes, &maps.q, 0, hf * a.q8_rows + yq, bar_qfull);
+              else tma_load_2d(sQ + hf * kQHalfBytes, &maps.q, 64 * hf, yq, bar_qfull);
+            }
             ++q_loads;
             prev_unit = p.unit;
           }
@@ -488,7 +513,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 y = (page * s.n_kv_heads + p.h) * s.page_size + j % s.page_size;
               }
 #pragma unroll
-              for (int hf = 0; hf < kHalves; ++hf)
+              for (int hf = 0; hf < kKHalves; ++hf)
                 tma_load_2d(dst + hf * kKHalfBytes + rh * (128 * 128), map, 64 * hf, y, bar);
             }
           }
@@ -541,8 +566,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
               for (int ks = 0; ks < kKSteps; ++ks) {
                 const uint32_t a_addr = sQ + (ks >> 2) * kQHalfBytes + j * (128 * 128) + (ks & 3) * 32;
-                const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
-                umma_bf16_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
+                if constexpr (K8) {
+                  // term ks >> 2 of q against the tile's 32 bytes ks & 3: both terms add into the same scores
+                  const uint32_t b_addr = sK + st * kStageBytes + (ks & 3) * 32;
+                  umma_e4m3_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
+                } else {
+                  const uint32_t b_addr = sK + st * kStageBytes + (ks >> 2) * kKHalfBytes + (ks & 3) * 32;
+                  umma_bf16_ss(d_tmem, umma_desc(a_addr), umma_desc(b_addr), ks > 0 ? 1u : 0u);
+                }
               }
               umma_commit(bar_sfull + 8 * acc);
             }
@@ -561,7 +592,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int mb = (sw >> 2) & 1;    // statistics group = accumulator of this warp
     const int ch = sw >> 3;          // half of the tile's 256 keys that this warp reads
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + mb * 256 + ch * 128;
-    const float cs = a.cs;
     const int S = s.n_sink;
 
     bool ok = true;
@@ -585,6 +615,12 @@ __global__ void __launch_bounds__(kThreads, 1)
       const long long rowid =
           (((long long)(p.l - a.layer_begin) * s.batch + p.b) * s.n_q_heads + p.h * G + g) * T + tq;
       float* stp = a.stats + (rowid * a.n_splits + 2 * p.slot + ch) * 3;
+      float cs = a.cs;
+      if constexpr (K8) {
+        // scores come out in units of (row's q scale) x (layer's K scale)
+        const long long qrow = (((long long)p.l * s.batch + p.b) * s.n_q_heads + p.h * G + g) * T + tq;
+        cs = a.cs * s.kv_scales[2 * p.l] * (row_valid ? a.q8_scale[qrow] : 1.f);
+      }
       if (!active || p.n_tiles == 0) {
         // nothing to read: an idle row block, or an empty key range (its slots still get neutral statistics)
         if (active && row_valid && (!alt || mb == 0)) {
@@ -754,46 +790,96 @@ EncodeTiledFn encode_tiled_fn() {
 }
 }  // namespace
 
+// 8-bit keys: the tail queries as two E4M3 terms.  A warp per query row of 128 values: the row's scale is the power
+// of two that puts its largest magnitude into [128, 256) (inside E4M3's range of 448), hi = E4M3 nearest to
+// q / scale, lo = E4M3 nearest to q / scale - hi.  A bf16 value has eight significant bits and each term four, so
+// hi + lo is exact unless the value is more than 2^10 below the row's largest, where what is dropped is below
+// 2^-17 of that largest value.
+__global__ void q_split_kernel(const __nv_bfloat16* __restrict__ q_tail, long long row_begin, long long row_end,
+                               long long rows_total, uint8_t* __restrict__ q8, float* __restrict__ q8_scale) {
+  const long long row = row_begin + (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= row_end) return;  // whole warps leave together
+  const int lane = threadIdx.x & 31;
+  const uint2 raw = *reinterpret_cast<const uint2*>(q_tail + row * 128 + lane * 4);
+  float x[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u), __uint_as_float(raw.y << 16),
+                __uint_as_float(raw.y & 0xffff0000u)};
+  float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  const int e2 = (amax > 0.f && amax < INFINITY) ? ilogbf(amax) - 7 : 0;
+  const float scale = exp2f((float)e2), inv = exp2f((float)-e2);
+  uint32_t hi = 0, lo = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float y = x[i] * inv;  // exact: a power of two
+    const __nv_fp8_storage_t h = __nv_cvt_float_to_fp8(y, __NV_SATFINITE, __NV_E4M3);
+    const float hf = __half2float(__half(__nv_cvt_fp8_to_halfraw(h, __NV_E4M3)));
+    const __nv_fp8_storage_t l = __nv_cvt_float_to_fp8(y - hf, __NV_SATFINITE, __NV_E4M3);
+    hi |= (uint32_t)h << (8 * i);
+    lo |= (uint32_t)l << (8 * i);
+  }
+  *reinterpret_cast<uint32_t*>(q8 + row * 128 + lane * 4) = hi;
+  *reinterpret_cast<uint32_t*>(q8 + (rows_total + row) * 128 + lane * 4) = lo;
+  if (lane == 0) q8_scale[row] = scale;
+}
+
 // grid = a.grid CTAs (fixed with the plan, so that the merge kernel finds the pieces of a unit); block 576.
-template <int DH>
+template <int DH, bool K8>
 static cudaError_t launch_scores_umma_dh(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return cudaErrorNotSupported;
+  constexpr int kElem = K8 ? 1 : 2;  // bytes of a cached key element
+  const CUtensorMapDataType dt = K8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   const cuuint64_t rows_total = a.s.page_size > 0 ? (cuuint64_t)a.s.n_pages * a.s.n_kv_heads * a.s.page_size
                                                   : (cuuint64_t)a.s.batch * a.s.n_kv_heads * a.s.full_capacity;
   const cuuint64_t gdim[2] = {(cuuint64_t)DH, rows_total};
-  const cuuint64_t gstride[1] = {(cuuint64_t)(2 * DH)};
-  const cuuint32_t box[2] = {64u, 128u};
+  const cuuint64_t gstride[1] = {(cuuint64_t)(kElem * DH)};
+  const cuuint32_t box[2] = {K8 ? 128u : 64u, 128u};  // 128 bytes x 128 keys either way
   const cuuint32_t estride[2] = {1u, 1u};
   KeyMaps local;
-  {
+  const cuuint64_t q_rows = (cuuint64_t)a.s.n_layers * a.s.batch * a.s.n_q_heads * (cuuint64_t)a.w_last;
+  if (K8) {
+    // this call's layers of q_tail as two E4M3 terms, then one matrix of 2 x q_rows rows of 128 bytes over them
+    const long long per_layer = (long long)a.s.batch * a.s.n_q_heads * a.w_last;
+    const long long r0 = a.layer_begin * per_layer, r1 = r0 + a.layer_count * per_layer;
+    q_split_kernel<<<(unsigned)((r1 - r0 + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)a.q_tail, r0, r1,
+                                                                    (long long)q_rows, a.q8, a.q8_scale);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const cuuint64_t qdim[2] = {128u, 2 * q_rows};
+    const cuuint32_t qbox[2] = {128u, (cuuint32_t)kBlockM};
+    const CUresult r = encode(&local.q, dt, 2, a.q8, qdim, gstride, qbox, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  } else {
     // the tail queries of the whole stack as one matrix of head_dim-element rows; a box is 64 d of a unit's 256 rows
-    const cuuint64_t qdim[2] = {(cuuint64_t)DH,
-                                (cuuint64_t)a.s.n_layers * a.s.batch * a.s.n_q_heads * (cuuint64_t)a.w_last};
+    const cuuint64_t qdim[2] = {(cuuint64_t)DH, q_rows};
     const cuuint32_t qbox[2] = {64u, (cuuint32_t)kBlockM};
-    const CUresult r = encode(&local.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.q_tail), qdim, gstride,
-                              qbox, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    const CUresult r = encode(&local.q, dt, 2, const_cast<void*>(a.q_tail), qdim, gstride, qbox, estride,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   const int l_end = a.layer_begin + a.layer_count;
   for (int l = a.layer_begin; l < l_end; ++l) {
-    const CUresult r = encode(&local.m[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kf.p[l]), gdim,
-                              gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    const CUresult r = encode(&local.m[l], dt, 2, const_cast<void*>(kf.p[l]), gdim, gstride, box, estride,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   for (int l = 0; l < LT_MAX_LAYERS; ++l)
     if (l < a.layer_begin || l >= l_end) local.m[l] = local.m[a.layer_begin];
-  constexpr int smem = Geo<DH>::kSmemBytes;
-  cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  constexpr int smem = Geo<DH, K8>::kSmemBytes;
+  cudaError_t e = cudaFuncSetAttribute(scores_umma_kernel<DH, K8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  scores_umma_kernel<DH><<<a.grid, kThreads, smem, st>>>(a, local);
+  scores_umma_kernel<DH, K8><<<a.grid, kThreads, smem, st>>>(a, local);
   return cudaGetLastError();
 }
 
 cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st) {
-  return a.s.head_dim == 64 ? launch_scores_umma_dh<64>(a, kf, st) : launch_scores_umma_dh<128>(a, kf, st);
+  if (a.s.kv_fp8) return launch_scores_umma_dh<128, true>(a, kf, st);
+  return a.s.head_dim == 64 ? launch_scores_umma_dh<64, false>(a, kf, st) : launch_scores_umma_dh<128, false>(a, kf, st);
 }
 
 }  // namespace lt

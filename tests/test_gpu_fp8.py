@@ -93,20 +93,68 @@ def test_fp8_caches_append_codes_and_attention(Hq, Hkv, S, R, lens, steps):
                         assert np.array_equal(st.k_full[l][b, h, :n + steps].cpu().numpy(), hist)
 
 
-def test_fp8_shape_is_validated_and_scoring_refuses_8bit_keys():
+def test_fp8_shape_is_validated():
     sc = torch.full((2, 2), 0.02, dtype=torch.float32, device="cuda")
     ok = lt.Shape(2, 1, 8, 2, 128, 4, 12, 64, lt.LT_BF16, 0.0, kv_fp8=1, kv_scales=sc)
     assert lt.workspace_bytes(ok) > 0
+    # scoring with 8-bit keys keeps a two-term copy of the tail queries in the workspace
+    assert lt.workspace_bytes(ok, 64, 8) >= lt.workspace_bytes(ok) + 2 * (2 * 1 * 8 * 8) * 128
     for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=34)):
         d = dict(ok.__dict__); d.update(kw)
         with pytest.raises(lt.LtError):
             lt.workspace_bytes(lt.Shape(**d))
-    k8 = [torch.zeros((1, 2, 64, 128), dtype=torch.uint8, device="cuda") for _ in range(2)]
-    ws = torch.empty(lt.workspace_bytes(ok, 64, 8), dtype=torch.uint8, device="cuda")
-    with pytest.raises(lt.LtError) as e:
-        lt.lazy_scores(ok, torch.zeros((2, 1, 8, 8, 128), dtype=torch.bfloat16, device="cuda"), k8, 64, 8,
-                       torch.zeros((2, 1, 8), device="cuda"), ws)
-    assert e.value.status == 2
+
+
+@pytest.mark.parametrize("Hq,Hkv,T,n,S,R,per_row", [
+    (8, 2, 64, 1500, 4, 60, 0),        # 256 query rows per kv head: both accumulators per tile; ragged last tile
+    (5, 1, 16, 700, 4, 28, 0),         # 80 rows: one row block, tiles alternate between the accumulators
+    (16, 2, 64, 900, 0, 100, 1),       # two query blocks per kv head; no sink; per-row window
+    (8, 2, 32, 300, 4, 400, 0),        # the window covers every key: every score is 1
+])
+def test_fp8_keys_lazy_scores_match_eq1(Hq, Hkv, T, n, S, R, per_row):
+    """Scoring from 8-bit keys (E4M3 MMAs on the stored bytes, q as two E4M3 terms) against Eq. 1 on the
+    dequantised keys; the route with the log-sum-exp given must agree as well."""
+    from tests.gpu_util import SCORE_ABS
+    torch.manual_seed(41)
+    g = np.random.default_rng(41)
+    L, B, D = 2, 2, 128
+    scales = g.uniform(0.015, 0.04, size=(L, 2)).astype(np.float32)
+    sc = torch.from_numpy(scales).cuda().contiguous()
+    shape = lt.Shape(L, B, Hq, Hkv, D, S, R, n, lt.LT_BF16, 0.0, recent_per_row=per_row, kv_fp8=1, kv_scales=sc)
+    q_tail = torch.randn(L, B, Hq, T, D).bfloat16()
+    q_tail[:, :, :, :, :3] *= 6.0                                              # a few large coordinates: the values of a row span several binades
+    k8, kvals = [], []
+    for l in range(L):
+        hk = torch.randn(B, Hkv, n, D).bfloat16()
+        hk[:, :, :max(S, 1)] += 0.3 * q_tail[l, :, ::Hq // Hkv].float().mean(2, keepdim=True).bfloat16()   # some mass on the first keys
+        kc, kval = O.quantize_e4m3(f64(hk), scales[l, 0])
+        k8.append(torch.from_numpy(kc).cuda()); kvals.append(kval)
+    tables = lt.LayerTables(shape, k8, k8, None, None)
+    ws = torch.empty(lt.workspace_bytes(shape, n, T), dtype=torch.uint8, device="cuda")
+    lt.workspace_init(ws)
+    scores = torch.full((L, B, Hq), float("nan"), device="cuda")
+    lt.lazy_scores(shape, q_tail.cuda(), tables, n, T, scores, ws)
+    ref = np.zeros((L, B, Hq)); lse = np.zeros((L, B, Hq, T))
+    fn = O.lazy_scores_per_row_window if per_row else O.lazy_scores
+    for l in range(L):
+        for b in range(B):
+            ref[l, b] = fn(f64(q_tail[l, b]), kvals[l][b], S, R)
+            lse[l, b] = O.causal_lse(f64(q_tail[l, b]), kvals[l][b])
+    assert lt.check(ws) == 0
+    err = np.abs(f64(scores) - ref).max()
+    assert err <= SCORE_ABS, err
+    if S + R >= n:
+        assert np.abs(ref - 1.0).max() < 1e-12
+    scores2 = torch.full((L, B, Hq), float("nan"), device="cuda")
+    lt.lazy_scores_lse(shape, q_tail.cuda(), tables, torch.from_numpy(lse).float().cuda(), n, T, scores2, ws)
+    assert lt.check(ws) == 0
+    err2 = np.abs(f64(scores2) - ref).max()
+    assert err2 <= SCORE_ABS, err2
+    # one layer at a time writes the same bits into that layer's slice
+    one = torch.full((L, B, Hq), float("nan"), device="cuda")
+    for l in range(L):
+        lt.lazy_scores(shape, q_tail.cuda(), tables, n, T, one, ws, layer_begin=l, layer_count=1)
+    assert np.abs(f64(one) - ref).max() <= SCORE_ABS
 
 
 def test_fp8_with_paged_full_caches():
