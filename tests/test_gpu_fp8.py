@@ -248,3 +248,38 @@ def test_fp8_long_context_sampled_units():
         ref = O.streaming_attention(qh, K, V, S, R) if mask[l] else O.full_attention(qh, K, V)
         mx, rel = attn_errors(f64(out[l, b, h * G:(h + 1) * G]), ref)
         assert rel <= ATTN_REL_L2 and mx <= ATTN_MAX_ABS * max(1.0, float(np.abs(ref).max())), (l, b, h, mx, rel)
+
+
+def test_fp8_keys_lazy_scores_with_paged_pools():
+    """Scoring from E4M3 page pools behind a block table: a 128-key box of a tile never straddles a page."""
+    from tests.gpu_util import SCORE_ABS
+    torch.manual_seed(43)
+    g = np.random.default_rng(43)
+    L, B, Hq, Hkv, D, S, R, page, pps, T = 2, 2, 8, 2, 128, 4, 60, 128, 9, 64
+    cap, n = page * pps, 1100
+    scales = g.uniform(0.015, 0.04, size=(L, 2)).astype(np.float32)
+    n_pages = B * pps + 3
+    table = torch.randperm(n_pages)[: B * pps].view(B, pps).to(torch.int32).cuda().contiguous()
+    shape = lt.Shape(L, B, Hq, Hkv, D, S, R, cap, lt.LT_BF16, 0.0, page_size=page, pages_per_seq=pps, n_pages=n_pages,
+                     block_table=table, kv_fp8=1, kv_scales=torch.from_numpy(scales).cuda().contiguous())
+    pools = [torch.full((n_pages, Hkv, page, D), 0x7E, dtype=torch.uint8, device="cuda") for _ in range(L)]   # 448 where nothing is stored
+    q_tail = torch.randn(L, B, Hq, T, D).bfloat16()
+    kvals, tab = [], table.cpu()
+    for l in range(L):
+        hk = torch.randn(B, Hkv, n, D).bfloat16()
+        kc, kval = O.quantize_e4m3(f64(hk), scales[l, 0])
+        kvals.append(kval)
+        for b in range(B):
+            for p in range(pps):
+                lo, hi = p * page, min((p + 1) * page, n)
+                if lo < hi:
+                    pools[l][int(tab[b, p]), :, : hi - lo] = torch.from_numpy(kc[b, :, lo:hi]).cuda()
+    tables = lt.LayerTables(shape, pools, pools, None, None)
+    ws = torch.empty(lt.workspace_bytes(shape, n, T), dtype=torch.uint8, device="cuda")
+    lt.workspace_init(ws)
+    scores = torch.full((L, B, Hq), float("nan"), device="cuda")
+    lt.lazy_scores(shape, q_tail.cuda(), tables, n, T, scores, ws)
+    assert lt.check(ws) == 0
+    ref = np.stack([np.stack([O.lazy_scores(f64(q_tail[l, b]), kvals[l][b], S, R) for b in range(B)]) for l in range(L)])
+    err = np.abs(f64(scores) - ref).max()
+    assert err <= SCORE_ABS and 0.0 < ref.min() and ref.max() < 0.9, (err, ref.min(), ref.max())
