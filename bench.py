@@ -1028,9 +1028,9 @@ def run_profile_case(args):
 
 
 def run_profile_case_fp8(args):
-    """Small case of the decode step with FP8 caches for profiler captures: 4
-    layers (2 lazy) of the benchmark's stack shape, byte caches with random
-    codes (2.3 GB on the device), a few decode steps, nothing else."""
+    """Small case with FP8 caches for profiler captures: 4 layers (2 lazy) of the
+    benchmark's stack shape, byte caches with random codes (2.3 GB on the device),
+    two scoring passes from the 8-bit keys and a few decode steps, nothing else."""
     assert torch.cuda.is_available()
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
@@ -1045,14 +1045,18 @@ def run_profile_case_fp8(args):
     shape = lt.Shape(L, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, cap, lt.LT_BF16, kv_fp8=1, kv_scales=scales)
     mk = lambda n: [torch.randint(0, 120, (B, Hkv, n, D), dtype=torch.uint8, device=dev) for _ in range(L)]
     tables = lt.LayerTables(shape, mk(cap), mk(cap), mk(C), mk(C))
-    ws = torch.empty(lt.workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    ws = torch.empty(lt.workspace_bytes(shape, cfg.n_ctx, cfg.w_last), dtype=torch.uint8, device=dev)
     lt.workspace_init(ws)
     mask = torch.tensor([0, 1, 1, 0], dtype=torch.uint8, device=dev)
     seq = torch.full((B,), cfg.n_ctx, dtype=torch.int32, device=dev)
     q = torch.randn((L, B, Hq, D), device=dev).bfloat16()
     k = torch.randn((L, B, Hkv, D), device=dev).bfloat16()
     out = torch.zeros_like(q)
+    q_tail = torch.randn((L, B, Hq, cfg.w_last, D), device=dev).bfloat16()
+    scores = torch.zeros((L, B, Hq), dtype=torch.float32, device=dev)
     t0 = time.perf_counter()
+    for _ in range(2):      # the scoring pass from the 8-bit keys (the second launch is the warm one)
+        lt.lazy_scores(shape, q_tail, tables, cfg.n_ctx, cfg.w_last, scores, ws)
     for _ in range(args.profile_case_fp8):
         lt.decode_step(shape, q, k, k, tables, mask, seq, out, ws)
     torch.cuda.synchronize()
