@@ -225,7 +225,7 @@ __host__ __device__ inline void score_split_range(const ScoreArgs& a, int sp, in
   *k1 = (*k0 + a.split_len < a.n_ctx) ? *k0 + a.split_len : a.n_ctx;
 }
 cudaError_t launch_scores_generic(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
-// bf16, head_dim 128: tcgen05 / TMEM path.
+// bf16 queries, head_dim 128 or 64 (8-bit keys: 128): tcgen05 / TMEM path.
 bool scores_umma_supported(const lt_shape& s, int w_last);
 cudaError_t launch_scores_umma(const ScoreArgs& a, const LayerTable& kf, cudaStream_t st);
 cudaError_t launch_scores_finish(const ScoreArgs& a, cudaStream_t st);

@@ -1,4 +1,6 @@
-// Lazy ratio (Eq. 1), Blackwell tensor-core path: bf16, head_dim 128 or 64.
+// Lazy ratio (Eq. 1), Blackwell tensor-core path: bf16 queries, head_dim 128 or 64; keys in bf16, or (head_dim 128,
+// template branch K8) as the E4M3 bytes of an 8-bit cache, which go through tcgen05.mma kind::f8f6f4 against the
+// queries as two E4M3 terms (see Geo and q_split_kernel).
 //
 // S = Q K^T is a real dense contraction here (G * w_last query rows against
 // every prompt key), so it runs on the 5th-generation tensor cores:
