@@ -95,6 +95,18 @@ def test_host_side_errors_come_before_any_launch():
     assert L.lt_kv_append(C.byref(cs), fake, fake, fake, fake, None, None, None, None, 0, 2, 1, None, None) == 1
     assert L.lt_stream_init(C.byref(cs), fake, tab, tab, fake, None, tab, None, None) == 1
     assert L.lt_workspace_init(None, 0, None) == 3
+    # the layered step: same checks as lt_decode_step, and its workspace must have a slot region per layer
+    need, need_l = C.c_size_t(0), C.c_size_t(0)
+    big = lt.Shape(8, 2, 8, 2, 128, 4, 60, 40000)
+    assert L.lt_workspace_bytes(C.byref(big.c()), 0, 0, C.byref(need)) == 0
+    assert L.lt_workspace_bytes_layers(C.byref(big.c()), 0, 0, C.byref(need_l)) == 0 and need_l.value > need.value
+    assert L.lt_workspace_bytes_layers(C.byref(big.c()), 0, 0, None) == 1
+    tab8 = (C.c_void_p * 8)(*[0x1000 * (i + 1) for i in range(8)])
+    args = lambda ws_bytes, begin=0, count=1, q=fake: (C.byref(big.c()), q, fake, fake, tab8, tab8, None, None, fake, fake, fake,
+                                                        0, begin, count, 0, 1, C.c_void_p(0x1000), ws_bytes, None)
+    assert L.lt_decode_step_layers(*args(need.value)) == 3                      # plain workspace: no per-layer slots
+    assert L.lt_decode_step_layers(*args(need_l.value, begin=8)) == 1           # layer range
+    assert L.lt_decode_step_layers(*args(need_l.value, q=None)) == 1            # null q
 
 
 def test_binding_refuses_cpu_tensors():
