@@ -283,3 +283,52 @@ def test_fp8_keys_lazy_scores_with_paged_pools():
     ref = np.stack([np.stack([O.lazy_scores(f64(q_tail[l, b]), kvals[l][b], S, R) for b in range(B)]) for l in range(L)])
     err = np.abs(f64(scores) - ref).max()
     assert err <= SCORE_ABS and 0.0 < ref.min() and ref.max() < 0.9, (err, ref.min(), ref.max())
+
+
+def test_fp8_32k_stack_scoring_from_8bit_keys_sampled_units():
+    """The benchmark stack's shape with its keys stored as E4M3 (torch's cast makes the input codes, one scale per
+    layer): scores from the 8-bit keys against Eq. 1 on the dequantised keys of sampled (layer, batch row, kv head)
+    units - every kv head, first and last batch row, planted and unplanted layers - and the planted layers recovered."""
+    import gc
+    from synth import CONFIGS, make_layer, planted_layers
+    from tests.gpu_util import SCORE_ABS
+    gc.collect(); torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 30 * 2**30:
+        pytest.skip("needs ~15 GB of free device memory")
+    cfg = CONFIGS["llama3_8b_32k"]
+    L, B, Hq, Hkv, D, n, T, G = (cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_ctx,
+                                 cfg.w_last, cfg.group)
+    planted = planted_layers(cfg)
+    scales = np.full((L, 2), 0.03, dtype=np.float32)                     # |k| up to 448 x 0.03 = 13 is representable
+    shape = lt.Shape(L, B, Hq, Hkv, D, cfg.n_sink, cfg.n_recent, n, lt.LT_BF16, 0.0, kv_fp8=1,
+                     kv_scales=torch.from_numpy(scales).cuda().contiguous())
+    q_tail = torch.empty((L, B, Hq, T, D), dtype=torch.bfloat16, device="cuda")
+    k8 = []
+    for l in range(L):
+        qt, K, V = make_layer(cfg, l, l in planted, "cuda", capacity=n)
+        q_tail[l].copy_(qt)
+        k8.append((K.float() / 0.03).to(torch.float8_e4m3fn).view(torch.uint8).contiguous())
+        del qt, K, V
+    tables = lt.LayerTables(shape, k8, k8, None, None)
+    ws = torch.empty(lt.workspace_bytes(shape, n, T), dtype=torch.uint8, device="cuda")
+    lt.workspace_init(ws)
+    scores = torch.zeros((L, B, Hq), dtype=torch.float32, device="cuda")
+    lt.lazy_scores(shape, q_tail, tables, n, T, scores, ws)
+    assert lt.check(ws) == 0
+    sc = f64(scores)
+    assert np.isfinite(sc).all() and sc.min() >= 0 and sc.max() <= 1 + 1e-6
+    table = O.e4m3_values()                                              # code -> value, the oracle's own table
+    unplanted = [l for l in range(L) if l not in planted]
+    units = [(planted[0], 0, 0), (unplanted[0], B - 1, 1), (planted[-1], B - 1, 2), (unplanted[-1], 0, 3),
+             (planted[len(planted) // 2], B // 2, 4), (unplanted[len(unplanted) // 2], 1, 5),
+             (planted[1], B - 1, 6), (unplanted[1], 0, 7)]
+    assert {u[2] for u in units} == set(range(Hkv))
+    for l, b, h in units:
+        Kd = table[k8[l][b, h].cpu().numpy()] * float(scales[l, 0])        # [n, D] dequantised keys of the unit
+        ref = O.lazy_scores(f64(q_tail[l, b, h * G:(h + 1) * G]), Kd[None], cfg.n_sink, cfg.n_recent)
+        assert np.max(np.abs(sc[l, b, h * G:(h + 1) * G] - ref)) <= SCORE_ABS, (l, b, h)
+    mask = torch.zeros(L, dtype=torch.uint8, device="cuda")
+    lt.select_lazy(scores, L, B, Hq, cfg.n_lazy, mask)
+    assert sorted(np.nonzero(mask.cpu().numpy())[0].tolist()) == planted
+    assert np.array_equal(mask.cpu().numpy(), O.select_lazy(sc, cfg.n_lazy)[0])
