@@ -195,6 +195,21 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail /* dev */,
                          size_t ws_bytes, void* stream);
 
 /*
+ * lt_lazy_scores that also hands out the denominators it computed (Table 1:
+ * the `lse` that the prefill's attention returns next to its output):
+ *   lse_out  dev float [L][B][Hq][w_last]: natural logarithm of
+ *            sum_{j <= i} exp(scale * q_i . k_j) for the tail rows
+ *            i = n_ctx - w_last .. n_ctx - 1; only the scored layers' slices are
+ *            written.  It is the input lt_lazy_scores_lse expects, for callers
+ *            whose prefill does not export it.
+ * Everything else as lt_lazy_scores (same pass over the keys, same scores).
+ */
+lt_status lt_lazy_scores_with_lse(const lt_shape* shape, const void* q_tail /* dev */,
+                                  const void* const* k_full /* host table */, int32_t n_ctx, int32_t w_last,
+                                  int32_t layer_begin, int32_t layer_count, float* scores /* dev */,
+                                  float* lse_out /* dev */, void* ws /* dev */, size_t ws_bytes, void* stream);
+
+/*
  * Lazy ratio with the denominator given (Section 5.1: FlashAttention's prefill
  * already produced the log-sum-exp of every attention row, so only the product of
  * the tail queries with the kept keys is left to compute, a constant-size one; Table 1).

@@ -111,6 +111,8 @@ def lib() -> C.CDLL:
     L.lt_check.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     L.lt_lazy_scores.restype = i32
     L.lt_lazy_scores.argtypes = [shp, vp, tab, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.lt_lazy_scores_with_lse.restype = i32
+    L.lt_lazy_scores_with_lse.argtypes = [shp, vp, tab, i32, i32, i32, i32, vp, vp, vp, sz, vp]
     L.lt_lazy_scores_lse.restype = i32
     L.lt_lazy_scores_lse.argtypes = [shp, vp, tab, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.lt_select_lazy.restype = i32
@@ -228,6 +230,16 @@ def lazy_scores(shape: Shape, q_tail, k_full, n_ctx: int, w_last: int, scores, w
     cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
     _ok(lib().lt_lazy_scores(C.byref(shape.c()), _ptr(q_tail), tab, n_ctx, w_last, layer_begin, cnt, _ptr(scores),
                              _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "lt_lazy_scores")
+
+
+def lazy_scores_with_lse(shape: Shape, q_tail, k_full, n_ctx: int, w_last: int, scores, lse_out, ws, layer_begin: int = 0,
+                         layer_count: int | None = None, stream=None):
+    """lt_lazy_scores_with_lse: Eq. 1 plus the tail rows' log-sum-exp that the same pass computed."""
+    tab = k_full.k_full if isinstance(k_full, LayerTables) else _table(k_full, shape.n_layers)
+    cnt = shape.n_layers - layer_begin if layer_count is None else layer_count
+    _ok(lib().lt_lazy_scores_with_lse(C.byref(shape.c()), _ptr(q_tail), tab, n_ctx, w_last, layer_begin, cnt,
+                                      _ptr(scores), _ptr(lse_out), _ptr(ws), ws.numel() * ws.element_size(),
+                                      _stream(stream)), "lt_lazy_scores_with_lse")
 
 
 def lazy_scores_lse(shape: Shape, q_tail, k_full, lse, n_ctx: int, w_last: int, scores, ws, layer_begin: int = 0,

@@ -285,7 +285,8 @@ lt_status lt_check(void* ws, uint32_t* flags_out, void* stream) {
 // Shared body of lt_lazy_scores (lse == NULL) and lt_lazy_scores_lse.
 static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,
                              int window_only, int32_t n_ctx, int32_t w_last, int32_t layer_begin,
-                             int32_t layer_count, float* scores, void* ws, size_t ws_bytes, void* stream) {
+                             int32_t layer_count, float* scores, void* ws, size_t ws_bytes, void* stream,
+                             float* lse_out = nullptr) {
   lt_status st = validate_shape(shape);
   if (st != LT_OK) return st;
   if (!q_tail || !k_full || !scores) return LT_ERR_INVALID_ARG;
@@ -293,7 +294,8 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   // 8-bit keys are scored by the tensor-core kernel only (E4M3 MMAs on the stored bytes)
   if (shape->kv_fp8 && !scores_umma_supported(*shape, w_last)) return LT_ERR_UNSUPPORTED;
   if (w_last < 1 || w_last > n_ctx || n_ctx > shape->full_capacity) return LT_ERR_INVALID_ARG;
-  if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0) return LT_ERR_INVALID_ARG;
+  if (((uintptr_t)q_tail & 15u) != 0 || ((uintptr_t)lse & 3u) != 0 || ((uintptr_t)lse_out & 3u) != 0)
+    return LT_ERR_INVALID_ARG;
   if ((st = check_layer_range(shape, layer_begin, layer_count)) != LT_OK) return st;
   LayerTable kf;
   if ((st = fill_table_range(&kf, k_full, layer_begin, layer_count)) != LT_OK) return st;
@@ -329,6 +331,7 @@ static lt_status scores_impl(const lt_shape* shape, const void* q_tail, const vo
   a.s = *shape;
   a.q_tail = q_tail;
   a.lse = lse;
+  a.lse_out = lse_out;
   a.n_ctx = n_ctx;
   a.w_last = w_last;
   a.layer_begin = layer_begin;
@@ -357,6 +360,14 @@ lt_status lt_lazy_scores(const lt_shape* shape, const void* q_tail, const void* 
                          size_t ws_bytes, void* stream) {
   return scores_impl(shape, q_tail, k_full, nullptr, 0, n_ctx, w_last, layer_begin, layer_count, scores, ws, ws_bytes,
                      stream);
+}
+
+lt_status lt_lazy_scores_with_lse(const lt_shape* shape, const void* q_tail, const void* const* k_full, int32_t n_ctx,
+                                  int32_t w_last, int32_t layer_begin, int32_t layer_count, float* scores,
+                                  float* lse_out, void* ws, size_t ws_bytes, void* stream) {
+  if (!lse_out) return LT_ERR_INVALID_ARG;
+  return scores_impl(shape, q_tail, k_full, nullptr, 0, n_ctx, w_last, layer_begin, layer_count, scores, ws, ws_bytes,
+                     stream, lse_out);
 }
 
 lt_status lt_lazy_scores_lse(const lt_shape* shape, const void* q_tail, const void* const* k_full, const float* lse,

@@ -176,6 +176,7 @@ struct ScoreArgs {
   lt_shape s;
   const void* q_tail;
   const float* lse;  // window_only: natural-log denominators [L][B][Hq][T]
+  float* lse_out;    // full pass only, may be NULL: receives the denominators it computed, same layout
   int n_ctx, w_last;
   int layer_begin, layer_count;  // layers scored by this call; q_tail, stats and scores keep their whole-stack indexing
   int window_only;

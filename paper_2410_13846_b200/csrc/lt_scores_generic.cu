@@ -251,6 +251,8 @@ __global__ void scores_finish_kernel(ScoreArgs a) {
         W += w * st[sp * 3 + 2];
       }
       sum += W / A;
+      // the row's log-sum-exp over its visible keys, as a prefill's attention kernel would hand it over
+      if (a.lse_out) a.lse_out[idx * T + t] = (Mx + log2f(A)) * 0.6931471805599453f;
     }
   }
 #pragma unroll

@@ -167,3 +167,38 @@ def test_both_scoring_routes_give_the_same_mask_on_a_planted_stack():
     ma = torch.zeros(L, dtype=torch.uint8, device="cuda"); mb = torch.zeros_like(ma)
     lt.select_lazy(a, L, B, Hq, cfg.n_lazy, ma); lt.select_lazy(b, L, B, Hq, cfg.n_lazy, mb)
     assert torch.equal(ma, mb) and sorted(torch.nonzero(ma).flatten().tolist()) == planted
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv,S,R,n_ctx,T", [
+    (torch.float32, 64, 4, 2, 4, 60, 512, 16),           # CUDA-core kernel
+    (torch.bfloat16, 128, 8, 2, 4, 60, 1777, 64),        # tensor-core kernel, several pieces per unit
+    (torch.bfloat16, 64, 5, 1, 0, 28, 900, 8),           # one row block, tiles alternate between the accumulators
+])
+def test_scores_pass_hands_out_the_log_sum_exp(dtype, D, Hq, Hkv, S, R, n_ctx, T):
+    """lt_lazy_scores_with_lse: the denominators of the same pass against the oracle's causal log-sum-exp (what
+    Table 1 takes from the prefill), the scores unchanged, and the pair (lse, kept keys) through the constant-size
+    route reproducing Eq. 1."""
+    torch.manual_seed(15)
+    L, B = 3, 2
+    st = Stack(L, B, Hq, Hkv, D, S, R, n_ctx, dtype, n_ctx_max=n_ctx, w_last_max=T)
+    for l in range(L):
+        st.k_full[l][:, :, :n_ctx] = torch.randn(B, Hkv, n_ctx, D).to(dtype).cuda()
+    q_tail = (1.3 * torch.randn(L, B, Hq, T, D)).to(dtype).cuda()
+    plain = _run_scores(st, q_tail, n_ctx, T)
+    scores = torch.full_like(plain, float("nan"))
+    lse = torch.full((L, B, Hq, T), float("nan"), dtype=torch.float32, device="cuda")
+    lt.lazy_scores_with_lse(st.shape, q_tail, st.tables, n_ctx, T, scores, lse, st.ws)
+    assert torch.equal(scores, plain)
+    ref_lse = np.stack([np.stack([O.causal_lse(f64(q_tail[l, b]), f64(st.k_full[l][b, :, :n_ctx])) for b in range(B)])
+                        for l in range(L)])
+    assert np.max(np.abs(f64(lse) - ref_lse)) <= 1e-4, np.max(np.abs(f64(lse) - ref_lse))
+    # a layer range writes only its slices
+    part = torch.full_like(lse, float("nan"))
+    lt.lazy_scores_with_lse(st.shape, q_tail, st.tables, n_ctx, T, scores, part, st.ws, layer_begin=1, layer_count=1)
+    assert torch.isnan(part[0]).all() and torch.isnan(part[2]).all()
+    assert np.max(np.abs(f64(part[1]) - ref_lse[1])) <= 1e-4
+    # the denominators feed the route that reads the kept keys only
+    again = torch.full_like(plain, float("nan"))
+    lt.lazy_scores_lse(st.shape, q_tail, st.tables, lse, n_ctx, T, again, st.ws)
+    assert np.max(np.abs(f64(again) - _oracle_scores(st, q_tail, n_ctx))) <= SCORE_ABS
+    assert lt.check(st.ws) == 0
