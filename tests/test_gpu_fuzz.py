@@ -92,3 +92,59 @@ def test_random_option_combinations_against_the_oracle(seed):
                 for h in range(Hkv):
                     ek, valid = O.stream_cache_after(hist[h], S, R)
                     assert np.array_equal(bits(st.k_stream[l][b, h, :valid]), ek[:valid]), (c, l, b, h)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_scoring_combinations_against_eq1(seed):
+    """Eq. 1 through both routes (full denominator; log-sum-exp given) on seeded random shapes: group sizes, tail
+    lengths from one query to several row blocks, windows smaller and larger than the prompt, both readings of
+    X_recent, paged caches, and both scoring kernels."""
+    from tests.gpu_util import SCORE_ABS
+    g = np.random.default_rng(3000 + seed)
+    torch.manual_seed(4000 + seed)
+    dtype = torch.float32 if g.random() < 0.2 else torch.bfloat16
+    D = int(g.choice([64, 128]))
+    Hkv = int(g.choice([1, 2]))
+    G = int(g.choice([1, 2, 4, 5, 8, 16]))
+    T = int(g.choice([1, 5, 16, 64]))
+    n = int(g.choice([T, T + 1, 130, 257, 700, 1500, 2600]))
+    n = max(n, T)
+    S = int(g.choice([0, 1, 4]))
+    R = int(g.choice([1, 16, 60, 300, 4000]))
+    per_row = int(g.random() < 0.3)
+    paged = bool(g.random() < 0.4) and dtype == torch.bfloat16
+    L, B, Hq = 2, 2, Hkv * G
+    if paged:
+        page = 128
+        pps = -(-n // page)
+        st = PagedStack(L, B, Hq, Hkv, D, S, R, page, pps, dtype, seed=seed, recent_per_row=per_row)
+        cap = page * pps
+    else:
+        cap = n
+        st = Stack(L, B, Hq, Hkv, D, S, R, cap, dtype, n_ctx_max=n, w_last_max=T)
+        st.shape = lt.Shape(L, B, Hq, Hkv, D, S, R, cap, st.shape.dtype, 0.0, recent_per_row=per_row)
+    hk = [torch.randn(B, Hkv, cap, D).to(dtype) for _ in range(L)]
+    for l in range(L):
+        if paged:
+            st.scatter(l, hk[l], hk[l])
+        else:
+            st.k_full[l].copy_(hk[l])
+    q_tail = (1.2 * torch.randn(L, B, Hq, T, D)).to(dtype)
+    fn = O.lazy_scores_per_row_window if per_row else O.lazy_scores
+    ref = np.zeros((L, B, Hq)); lse = np.zeros((L, B, Hq, T))
+    for l in range(L):
+        for b in range(B):
+            ref[l, b] = fn(f64(q_tail[l, b]), f64(hk[l][b, :, :n]), S, R)
+            lse[l, b] = O.causal_lse(f64(q_tail[l, b]), f64(hk[l][b, :, :n]))
+    ws = torch.empty(lt.workspace_bytes(st.shape, n, T), dtype=torch.uint8, device="cuda")
+    lt.workspace_init(ws)
+    a = torch.full((L, B, Hq), float("nan"), device="cuda")
+    b2 = torch.full((L, B, Hq), float("nan"), device="cuda")
+    lse_out = torch.full((L, B, Hq, T), float("nan"), device="cuda")
+    lt.lazy_scores_with_lse(st.shape, q_tail.cuda(), st.tables, n, T, a, lse_out, ws)
+    lt.lazy_scores_lse(st.shape, q_tail.cuda(), st.tables, torch.from_numpy(lse).float().cuda(), n, T, b2, ws)
+    assert lt.check(ws) == 0
+    what = (seed, dtype, D, Hkv, G, T, n, S, R, per_row, paged)
+    assert np.max(np.abs(f64(a) - ref)) <= SCORE_ABS, what
+    assert np.max(np.abs(f64(b2) - ref)) <= SCORE_ABS, what
+    assert np.max(np.abs(f64(lse_out) - lse)) <= 2e-4, what
