@@ -42,8 +42,8 @@
  *   - GQA: query head hq reads kv head hq / (n_q_heads / n_kv_heads).
  *   - Every shape the calls accept is computed on the GPU by this library's own
  *     kernels.  The bandwidth-bound tensor-core kernels serve bf16 stacks with
- *     head_dim 64 or 128 (decode: query groups of up to 32 heads, up to 16 with
- *     8-bit caches; scoring: any group); fp32 stacks and larger groups run on
+ *     head_dim 64 or 128 (decode: query groups of up to 32 heads; scoring: any
+ *     group); fp32 stacks and larger groups run on
  *     tiled CUDA-core kernels, several times slower per byte.
  */
 #ifndef LT_H_
@@ -112,7 +112,7 @@ typedef struct lt_shape {
      v_new and out stay in `dtype`.  A stored byte c of layer l means E4M3(c) * kv_scales[l][0] for K and
      * kv_scales[l][1] for V; lt_kv_append / lt_decode_step store code(x) = E4M3 nearest to
      float32(x) / scale (float32 division, round to nearest even, saturating at +-448).  Needs
-     dtype = LT_BF16, head_dim = 128 and a query group of at most 16.  The kernels turn the stored bytes into
+     dtype = LT_BF16, head_dim = 128 and a query group of at most 32.  The kernels turn the stored bytes into
      f16 in registers (exact) and multiply on the tensor cores with fp32 accumulation, q as f16 at one
      power-of-two scale per head (exact for bf16 inputs), the probabilities as one f16 term.  lt_lazy_scores and
      lt_lazy_scores_lse read 8-bit keys too (k_full holds the E4M3 bytes; q_tail stays bf16): the stored bytes go

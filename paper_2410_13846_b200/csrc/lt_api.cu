@@ -28,7 +28,7 @@ lt_status validate_shape(const lt_shape* s) {
   if (s->kv_fp8 & ~1) return LT_ERR_INVALID_ARG;
   if (s->kv_fp8) {
     if (!s->kv_scales) return LT_ERR_INVALID_ARG;
-    if (s->dtype != LT_BF16 || s->head_dim != 128 || s->n_q_heads / s->n_kv_heads > 16) return LT_ERR_UNSUPPORTED;
+    if (s->dtype != LT_BF16 || s->head_dim != 128 || s->n_q_heads / s->n_kv_heads > 32) return LT_ERR_UNSUPPORTED;
   }
   if (s->page_size > 0) {
     if (s->page_size % 128 != 0) return LT_ERR_UNSUPPORTED;

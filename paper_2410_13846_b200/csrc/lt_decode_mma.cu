@@ -166,7 +166,7 @@ struct TileSrc {
 // tiles through one shared ring (each copies half of every tile, a 64-thread named barrier per tile makes the
 // copies visible and frees the stage that is refilled), warp 0 of the pair serves heads 0-7 of the group and warp
 // 1 heads 8-15, so the chunk still crosses HBM, L2 and shared memory once.
-// ROLES = 4 (groups of 17..32 heads, 16-bit caches): all four warps walk one ring of twice the depth (a quarter of
+// ROLES = 4 (groups of 17..32 heads): all four warps walk one ring of twice the depth (a quarter of
 // every tile each, one 128-thread named barrier per tile); warp w serves heads 8w .. 8w + 7 - a warp beyond the
 // group's last head computes on zeros and stores nothing - and no sums cross warps.
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, int ROLES>
@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
     decode_mma_kernel(DecodeArgs a, LayerTable kf, LayerTable vf, LayerTable ks, LayerTable vs) {
   static_assert(WARPS == 4, "the merge tree below is written for four warps");
   static_assert(DH == 128 || (DH == 64 && !FP8), "head_dim 128, or 64 with 16-bit caches");
-  static_assert(ROLES == 1 || ROLES == 2 || (ROLES == 4 && !FP8), "one, two or four warps per tile stream");
+  static_assert(ROLES == 1 || ROLES == 2 || ROLES == 4, "one, two or four warps per tile stream");
   constexpr bool PAIR = ROLES > 1;                    // several warps share a ring, eight heads of the group each
   constexpr int STREAMS = WARPS / ROLES;              // independent tile streams of the CTA
   constexpr int RSTAGES = NSTAGE;                     // ring stages of a stream
@@ -787,9 +787,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB)
   finish_launch(a);
 }
 bool decode_mma_supported(const lt_shape& s) {
-  // groups of 9..16: two warps per tile, eight heads each; 17..32 (16-bit caches): four warps per tile
+  // groups of 9..16: two warps per tile, eight heads each; 17..32: four warps per tile
   return s.dtype == LT_BF16 && (s.head_dim == 128 || s.head_dim == 64) &&
-         (s.n_q_heads / s.n_kv_heads) <= (s.kv_fp8 ? 16 : 32);
+         (s.n_q_heads / s.n_kv_heads) <= 32;
 }
 
 template <int TILE, int NSTAGE, int WARPS, int MINB, bool FP8, int DH, int ROLES>
@@ -844,9 +844,11 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const L
   const bool pair = G > 8;   // groups of 9..16: two warps per tile, eight heads each
   const bool quad = G > 16;  // groups of 17..32: the four warps share one ring of twice the depth
   // 8-bit caches: raw stages of 32 keys (8 KB); a warp's three stages or a pair's six hold what the 16-bit ring holds
-  if (a.s.kv_fp8)
+  if (a.s.kv_fp8) {
+    if (quad) return launch_variant<32, 12, 4, 2, true, 128, 4>(a, kf, vf, ks, vs, st);
     return pair ? launch_variant<32, 6, 4, 2, true, 128, 2>(a, kf, vf, ks, vs, st)
                 : launch_variant<32, 3, 4, 2, true, 128, 1>(a, kf, vf, ks, vs, st);
+  }
   // head_dim 64: rows are half as long, so 32-key tiles keep the bytes in flight per warp (24 KB) the same
   if (a.s.head_dim == 64) {
     if (quad) return launch_variant<32, 12, 4, 2, false, 64, 4>(a, kf, vf, ks, vs, st);

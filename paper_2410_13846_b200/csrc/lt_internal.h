@@ -151,7 +151,7 @@ inline cudaError_t launch_decode_kernel(Kern kern, int grid, int threads, int sm
 }
 cudaError_t launch_decode_generic(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                                   const LayerTable& ks, const LayerTable& vs, cudaStream_t st);
-// bf16, head_dim 128 or 64, group size <= 32 (<= 16 with 8-bit caches): tensor-core path.
+// bf16, head_dim 128 or 64, group size <= 32: tensor-core path.
 bool decode_mma_supported(const lt_shape& s);
 cudaError_t launch_decode_mma(const DecodeArgs& a, const LayerTable& kf, const LayerTable& vf,
                               const LayerTable& ks, const LayerTable& vs, cudaStream_t st);

@@ -32,6 +32,8 @@ class Fp8Stack:
     (16, 2, 3, 9, [5, 0], 14),                     # G = 8, starts (almost) empty
     (32, 2, 4, 28, [300, 2047, 33], 36),           # G = 16: warp pairs on the byte path, ring wraps, chunk boundary
     (12, 1, 2, 12, [4200, 64], 6),                 # G = 12: the second warp of a pair serves four heads; several chunks
+    (32, 1, 4, 28, [300, 2047, 33], 36),           # G = 32: four warps per tile on the byte path, ring wraps
+    (20, 1, 0, 12, [4200, 64, 0], 6),              # G = 20: the third warp serves four heads, the fourth none; several chunks
 ])
 def test_fp8_caches_append_codes_and_attention(Hq, Hkv, S, R, lens, steps):
     torch.manual_seed(33)
@@ -99,7 +101,7 @@ def test_fp8_shape_is_validated():
     assert lt.workspace_bytes(ok) > 0
     # scoring with 8-bit keys keeps a two-term copy of the tail queries in the workspace
     assert lt.workspace_bytes(ok, 64, 8) >= lt.workspace_bytes(ok) + 2 * (2 * 1 * 8 * 8) * 128
-    for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=34)):
+    for kw in (dict(kv_scales=None), dict(head_dim=64), dict(dtype=lt.LT_F32), dict(n_q_heads=66)):
         d = dict(ok.__dict__); d.update(kw)
         with pytest.raises(lt.LtError):
             lt.workspace_bytes(lt.Shape(**d))
