@@ -135,7 +135,8 @@ def test_fp8_keys_lazy_scores_match_eq1(Hq, Hkv, T, n, S, R, per_row):
     ws = torch.empty(lt.workspace_bytes(shape, n, T), dtype=torch.uint8, device="cuda")
     lt.workspace_init(ws)
     scores = torch.full((L, B, Hq), float("nan"), device="cuda")
-    lt.lazy_scores(shape, q_tail.cuda(), tables, n, T, scores, ws)
+    lse_out = torch.full((L, B, Hq, T), float("nan"), device="cuda")
+    lt.lazy_scores_with_lse(shape, q_tail.cuda(), tables, n, T, scores, lse_out, ws)
     ref = np.zeros((L, B, Hq)); lse = np.zeros((L, B, Hq, T))
     fn = O.lazy_scores_per_row_window if per_row else O.lazy_scores
     for l in range(L):
@@ -145,6 +146,7 @@ def test_fp8_keys_lazy_scores_match_eq1(Hq, Hkv, T, n, S, R, per_row):
     assert lt.check(ws) == 0
     err = np.abs(f64(scores) - ref).max()
     assert err <= SCORE_ABS, err
+    assert np.abs(f64(lse_out) - lse).max() <= 1e-3          # the denominators of the same pass, natural log
     if S + R >= n:
         assert np.abs(ref - 1.0).max() < 1e-12
     scores2 = torch.full((L, B, Hq), float("nan"), device="cuda")
